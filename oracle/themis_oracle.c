@@ -1,0 +1,333 @@
+/*
+ * CPU oracle for the batched pipeline-scaling solver (Themis, arXiv 2407.14843).
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is a plain, slow, scalar restatement of
+ * what the solver computes.  It shares no code with the CUDA library and must
+ * never be called from the product path; only the tests, the smoke check and
+ * the benchmark's CPU-baseline leg use it.
+ *
+ * What is computed, per independent instance (one pipeline, one arrival rate):
+ *
+ *   minimise   sum_s  h_s * c_s                               (Eq. 6, objective)
+ *   subject to sum_s  l_s(b_s, c_s) + q_s(b_s)  <=  SLO       (Eq. 5 / Eq. 6)
+ *              lambda <= thr_s(b_s, c_s) * h_s   for all s     (Eq. 6)
+ *
+ * with h = replicas (the paper's n_s), c = cores per replica, b = batch size,
+ * thr(b, c) = b / l(b, c) the throughput of one replica, and the queuing delay
+ * q(b) = (b - 1) / lambda of Eq. 4 (optionally (b - 1) * h / lambda when every
+ * replica fills its own batch, flag ORACLE_QUEUE_PER_REPLICA).
+ *
+ * Latencies are discretised to buckets of width w: a stage costs
+ * ceil(l / w) + ceil(q / w) buckets and the budget is T = floor(SLO / w).
+ *
+ * Three solvers are provided and pinned against each other by the tests:
+ *   oracle_solve_batch      the stage-by-stage dynamic program of Algorithm 1,
+ *                           with the candidate minimum hoisted out of the
+ *                           budget loop (G_s) and a min-plus combine (F_s);
+ *   oracle_alg1_scatter     Algorithm 1 in the paper's own loop order
+ *                           (stage, budget descending, cores, batch), scattering
+ *                           into best[s][i + l];
+ *   brute_force.c           Eq. 6 by exhaustive enumeration (separate file).
+ *
+ * Readings of the paper taken here (each is pinned by a test):
+ *   - a candidate is skipped iff its replicas cannot sustain lambda or it does
+ *     not fit the remaining budget (the printed condition in Algorithm 1 is
+ *     inverted; the prose under it states the intent);
+ *   - throughput equality (thr * h == lambda) is feasible, as in Eq. 6;
+ *   - the budget test is on i + l, the index actually written;
+ *   - ties: strict '<' in ascending candidate order, so the lowest candidate
+ *     index wins, the lowest stage latency wins in the combine, and the lowest
+ *     total latency wins in the final scan (the paper's loops do the same);
+ *   - cost of a stage is h * c (Eq. 6), which equals Algorithm 1's 'c' when
+ *     every stage has one replica.
+ *
+ * Candidate index: idx = ((h - 1) * c_max + (c - 1)) * n_batch + bi for the
+ * joint problem (h slowest, then c, batch fastest, the loop order of
+ * Algorithm 1 with h added outside); idx = (c - 1) * n_batch + bi when h is
+ * fixed.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_INF INT32_MAX
+#define ORACLE_QUEUE_PER_REPLICA 1u
+
+typedef struct {
+    int32_t n_instances;
+    int32_t n_stages;
+    int32_t n_profiles;
+    int32_t c_max;
+    int32_t n_batch;
+    int32_t batch_sizes[16];
+    int32_t h_max;
+    int32_t slo_us;
+    int32_t bucket_us;
+    uint32_t flags;
+} oracle_problem;
+
+static uint64_t ceil_div_u64(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
+
+/*
+ * One candidate of one stage (the body of Algorithm 1's inner loops).
+ * Returns 1 and sets *ell (latency in buckets) and *cost when the candidate
+ * can sustain the arrival rate; returns 0 otherwise.  *ell may exceed T.
+ *
+ *   l   = profiled latency of a batch of b on c cores          [us]
+ *   q   = (b - 1) / lambda  (times h with the per-replica flag) [us]  (Eq. 4)
+ *   thr = b / l per replica; feasible iff h * thr >= lambda     (Eq. 6)
+ *
+ * lambda is given in milli-requests per second, so
+ *   h * b / (l_us * 1e-6) >= lambda_m * 1e-3   <=>   h * b * 1e9 >= lambda_m * l_us
+ *   q_us = (b - 1) * m * 1e9 / lambda_m.
+ */
+static int score_candidate(int32_t l_us, int32_t h, int32_t c, int32_t b, uint32_t lambda_m,
+                           int32_t bucket_us, uint32_t flags, int64_t *ell, int32_t *cost)
+{
+    uint64_t supply = (uint64_t)h * (uint64_t)b * 1000000000ull;
+    uint64_t demand = (uint64_t)lambda_m * (uint64_t)l_us;
+    if (supply < demand) return 0;
+    uint64_t m = (flags & ORACLE_QUEUE_PER_REPLICA) ? (uint64_t)h : 1ull;
+    uint64_t q_buckets = ceil_div_u64((uint64_t)(b - 1) * m * 1000000000ull,
+                                      (uint64_t)lambda_m * (uint64_t)bucket_us);
+    uint64_t l_buckets = ceil_div_u64((uint64_t)l_us, (uint64_t)bucket_us);
+    *ell = (int64_t)(l_buckets + q_buckets);
+    *cost = h * c;
+    return 1;
+}
+
+/*
+ * Per-bucket minimum over the candidates of one stage:
+ *   G[l]    = min cost over feasible candidates whose latency is exactly l buckets
+ *   Garg[l] = lowest candidate index attaining it (0 where G[l] is INF)
+ * lat_stage is [c_max][n_batch].  h_fixed > 0 selects the vertical variant.
+ */
+void oracle_score_stage(const oracle_problem *p, const int32_t *lat_stage, uint32_t lambda_m,
+                        int32_t h_fixed, int32_t T, int32_t *G, uint16_t *Garg)
+{
+    for (int32_t l = 0; l <= T; ++l) { G[l] = ORACLE_INF; Garg[l] = 0; }
+    int32_t h_lo = h_fixed > 0 ? h_fixed : 1;
+    int32_t h_hi = h_fixed > 0 ? h_fixed : p->h_max;
+    int32_t idx = 0;
+    for (int32_t h = h_lo; h <= h_hi; ++h)
+        for (int32_t c = 1; c <= p->c_max; ++c)
+            for (int32_t bi = 0; bi < p->n_batch; ++bi, ++idx) {
+                int64_t ell; int32_t cost;
+                int32_t l_us = lat_stage[(c - 1) * p->n_batch + bi];
+                if (!score_candidate(l_us, h, c, p->batch_sizes[bi], lambda_m, p->bucket_us,
+                                     p->flags, &ell, &cost))
+                    continue;
+                if (ell > T) continue;
+                if (cost < G[ell]) { G[ell] = cost; Garg[ell] = (uint16_t)idx; }
+            }
+}
+
+/*
+ * Min-plus combine of the prefix with one more stage:
+ *   F[t] = min_{0 <= l <= t} Fprev[t - l] + G[l],  A[t] = lowest l attaining it
+ * (A[t] = 0 where F[t] is INF).
+ */
+void oracle_minplus(int32_t T, const int32_t *Fprev, const int32_t *G, int32_t *F, uint16_t *A)
+{
+    for (int32_t t = 0; t <= T; ++t) {
+        int32_t best = ORACLE_INF; int32_t arg = 0;
+        for (int32_t l = 0; l <= t; ++l) {
+            if (Fprev[t - l] == ORACLE_INF || G[l] == ORACLE_INF) continue;
+            int32_t v = Fprev[t - l] + G[l];
+            if (v < best) { best = v; arg = l; }
+        }
+        F[t] = best; A[t] = (uint16_t)arg;
+    }
+}
+
+static void decode_idx(const oracle_problem *p, int32_t idx, int32_t h_fixed,
+                       int32_t *h, int32_t *c, int32_t *b)
+{
+    int32_t bi = idx % p->n_batch;
+    int32_t r = idx / p->n_batch;
+    *b = p->batch_sizes[bi];
+    *c = r % p->c_max + 1;
+    *h = h_fixed > 0 ? h_fixed : r / p->c_max + 1;
+}
+
+/*
+ * One instance, dynamic program.  Work arrays hold S rows of T+1 entries:
+ *   Gs, Gargs  per-stage candidate minima;  Fs  prefix tables;  As  argmin.
+ * Returns 0 (solved) or 1 (infeasible).
+ */
+static int solve_instance(const oracle_problem *p, const int32_t *lat_pipeline /* [S][C][B] */,
+                          uint32_t lambda_m, const int32_t *replicas /* [S] or NULL */,
+                          int32_t *h_out, int32_t *c_out, int32_t *b_out,
+                          int32_t *cost_out, int32_t *lat_out,
+                          int32_t *Gs, uint16_t *Gargs, int32_t *Fs, uint16_t *As)
+{
+    const int32_t S = p->n_stages, T = p->slo_us / p->bucket_us, W = T + 1;
+    const int32_t stage_words = p->c_max * p->n_batch;
+    for (int32_t s = 0; s < S; ++s)
+        oracle_score_stage(p, lat_pipeline + (size_t)s * stage_words, lambda_m,
+                           replicas ? replicas[s] : 0, T, Gs + (size_t)s * W, Gargs + (size_t)s * W);
+    /* first stage: the whole budget spent so far belongs to it */
+    memcpy(Fs, Gs, sizeof(int32_t) * (size_t)W);
+    memset(As, 0, sizeof(uint16_t) * (size_t)W);
+    for (int32_t s = 1; s < S; ++s)
+        oracle_minplus(T, Fs + (size_t)(s - 1) * W, Gs + (size_t)s * W,
+                       Fs + (size_t)s * W, As + (size_t)s * W);
+    /* final scan: cheapest total, lowest total latency among equals */
+    const int32_t *Fl = Fs + (size_t)(S - 1) * W;
+    int32_t best = ORACLE_INF, tstar = -1;
+    for (int32_t t = 0; t <= T; ++t)
+        if (Fl[t] < best) { best = Fl[t]; tstar = t; }
+    if (tstar < 0) {
+        for (int32_t s = 0; s < S; ++s) { h_out[s] = 0; c_out[s] = 0; b_out[s] = 0; }
+        *cost_out = -1; *lat_out = -1;
+        return 1;
+    }
+    /* walk the argmin tables back from the last stage */
+    int32_t t = tstar;
+    for (int32_t s = S - 1; s >= 0; --s) {
+        int32_t ell = s > 0 ? (int32_t)As[(size_t)s * W + t] : t;
+        int32_t idx = Gargs[(size_t)s * W + ell];
+        decode_idx(p, idx, replicas ? replicas[s] : 0, &h_out[s], &c_out[s], &b_out[s]);
+        t -= ell;
+    }
+    *cost_out = best; *lat_out = tstar;
+    return 0;
+}
+
+/*
+ * Batch driver.  All pointers are host memory.
+ *   lat_us      [P][S][c_max][n_batch]
+ *   profile_id  [N] or NULL (all 0)
+ *   lambda_mrps [N]
+ *   replicas    [N][S] (vertical variant) or NULL (joint)
+ *   h, c, b     [N][S];  total_cost, latency_buckets, status  [N]
+ * Optional dumps (NULL to skip), row-major with rows of T+1 entries:
+ *   dump_G int32 [N][S][T+1], dump_Garg uint16 [N][S][T+1],
+ *   dump_F int32 [N][S][T+1], dump_A uint16 [N][S][T+1]  (A row 0 is zero).
+ * n_threads <= 0 uses every core OpenMP sees.  Returns the thread count used,
+ * or -1 on allocation failure.
+ */
+int oracle_solve_batch(const oracle_problem *p, const int32_t *lat_us, const int32_t *profile_id,
+                       const uint32_t *lambda_mrps, const int32_t *replicas,
+                       int32_t *h, int32_t *c, int32_t *b,
+                       int32_t *total_cost, int32_t *latency_buckets, int32_t *status,
+                       int32_t *dump_G, uint16_t *dump_Garg, int32_t *dump_F, uint16_t *dump_A,
+                       int n_threads)
+{
+    const int32_t N = p->n_instances, S = p->n_stages;
+    const size_t W = (size_t)(p->slo_us / p->bucket_us) + 1;
+    const size_t rows = (size_t)S * W;
+    const size_t pipeline_words = (size_t)S * p->c_max * p->n_batch;
+    int used = 1, failed = 0;
+#ifdef _OPENMP
+    if (n_threads <= 0) n_threads = omp_get_max_threads();
+    used = n_threads;
+#pragma omp parallel num_threads(n_threads)
+#endif
+    {
+        int32_t *Gs = (int32_t *)malloc(sizeof(int32_t) * rows);
+        int32_t *Fs = (int32_t *)malloc(sizeof(int32_t) * rows);
+        uint16_t *Gargs = (uint16_t *)malloc(sizeof(uint16_t) * rows);
+        uint16_t *As = (uint16_t *)malloc(sizeof(uint16_t) * rows);
+        if (!Gs || !Fs || !Gargs || !As) {
+#ifdef _OPENMP
+#pragma omp atomic write
+#endif
+            failed = 1;
+        } else {
+#ifdef _OPENMP
+#pragma omp for schedule(dynamic, 1)
+#endif
+            for (int32_t n = 0; n < N; ++n) {
+                int32_t pid = profile_id ? profile_id[n] : 0;
+                status[n] = solve_instance(p, lat_us + (size_t)pid * pipeline_words, lambda_mrps[n],
+                                           replicas ? replicas + (size_t)n * S : NULL,
+                                           h + (size_t)n * S, c + (size_t)n * S, b + (size_t)n * S,
+                                           &total_cost[n], &latency_buckets[n], Gs, Gargs, Fs, As);
+                if (dump_G) memcpy(dump_G + (size_t)n * rows, Gs, sizeof(int32_t) * rows);
+                if (dump_F) memcpy(dump_F + (size_t)n * rows, Fs, sizeof(int32_t) * rows);
+                if (dump_Garg) memcpy(dump_Garg + (size_t)n * rows, Gargs, sizeof(uint16_t) * rows);
+                if (dump_A) memcpy(dump_A + (size_t)n * rows, As, sizeof(uint16_t) * rows);
+            }
+        }
+        free(Gs); free(Fs); free(Gargs); free(As);
+    }
+    return failed ? -1 : used;
+}
+
+/*
+ * Algorithm 1 in the paper's loop order, one instance: for each stage, for the
+ * budget already spent i from T down to 0, for each candidate (replicas,
+ * cores, batch), extend the reachable state (s-1, i) to (s, i + l) when the
+ * candidate sustains lambda and i + l <= T, keeping the cheaper total under a
+ * strict '<'.  The first stage extends the empty prefix (i = 0 only).
+ * best_* hold, per state, the running total, the stage latency used and the
+ * candidate index, from which the configuration is read back recursively.
+ * Returns 0 (solved) or 1 (infeasible); outputs as in oracle_solve_batch.
+ */
+int oracle_alg1_scatter(const oracle_problem *p, const int32_t *lat_pipeline, uint32_t lambda_m,
+                        const int32_t *replicas, int32_t *h_out, int32_t *c_out, int32_t *b_out,
+                        int32_t *cost_out, int32_t *lat_out)
+{
+    const int32_t S = p->n_stages, T = p->slo_us / p->bucket_us, W = T + 1;
+    const size_t cells = (size_t)S * W;
+    uint8_t *dp = (uint8_t *)calloc(cells, 1);
+    int32_t *best_total = (int32_t *)malloc(sizeof(int32_t) * cells);
+    int32_t *best_ell = (int32_t *)malloc(sizeof(int32_t) * cells);
+    int32_t *best_idx = (int32_t *)malloc(sizeof(int32_t) * cells);
+    if (!dp || !best_total || !best_ell || !best_idx) {
+        free(dp); free(best_total); free(best_ell); free(best_idx);
+        return -1;
+    }
+    for (int32_t s = 0; s < S; ++s) {
+        const int32_t *lat_stage = lat_pipeline + (size_t)s * p->c_max * p->n_batch;
+        int32_t h_lo = replicas ? replicas[s] : 1, h_hi = replicas ? replicas[s] : p->h_max;
+        for (int32_t i = T; i >= 0; --i) {
+            int reachable = (s == 0) ? (i == 0) : dp[(size_t)(s - 1) * W + i];
+            if (!reachable) continue;
+            int32_t idx = 0;
+            for (int32_t h = h_lo; h <= h_hi; ++h)
+                for (int32_t c = 1; c <= p->c_max; ++c)
+                    for (int32_t bi = 0; bi < p->n_batch; ++bi, ++idx) {
+                        int64_t ell; int32_t cost;
+                        if (!score_candidate(lat_stage[(c - 1) * p->n_batch + bi], h, c,
+                                             p->batch_sizes[bi], lambda_m, p->bucket_us, p->flags,
+                                             &ell, &cost))
+                            continue;
+                        if ((int64_t)i + ell > T) continue;
+                        int32_t total = cost + (s == 0 ? 0 : best_total[(size_t)(s - 1) * W + i]);
+                        size_t dst = (size_t)s * W + (size_t)(i + ell);
+                        if (!dp[dst] || total < best_total[dst]) {
+                            dp[dst] = 1;
+                            best_total[dst] = total;
+                            best_ell[dst] = (int32_t)ell;
+                            best_idx[dst] = idx;
+                        }
+                    }
+        }
+    }
+    int32_t least = ORACLE_INF, ind = -1;
+    for (int32_t i = 0; i <= T; ++i) {
+        size_t k = (size_t)(S - 1) * W + i;
+        if (dp[k] && best_total[k] < least) { least = best_total[k]; ind = i; }
+    }
+    int rc = 1;
+    if (ind < 0) {
+        for (int32_t s = 0; s < S; ++s) { h_out[s] = 0; c_out[s] = 0; b_out[s] = 0; }
+        *cost_out = -1; *lat_out = -1;
+    } else {
+        int32_t t = ind;
+        for (int32_t s = S - 1; s >= 0; --s) {
+            size_t k = (size_t)s * W + t;
+            decode_idx(p, best_idx[k], replicas ? replicas[s] : 0, &h_out[s], &c_out[s], &b_out[s]);
+            t -= best_ell[k];
+        }
+        *cost_out = least; *lat_out = ind;
+        rc = 0;
+    }
+    free(dp); free(best_total); free(best_ell); free(best_idx);
+    return rc;
+}
