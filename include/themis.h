@@ -1,0 +1,202 @@
+/*
+ * libthemis: batched solver for the joint horizontal + vertical scaling problem
+ * of multi-model inference pipelines (Themis, arXiv 2407.14843), for NVIDIA B200.
+ *
+ * One "instance" is one pipeline of S stages under one arrival rate lambda.  For
+ * every stage the solver picks replicas h (the paper's n_s), cores per replica c
+ * and batch size b, minimising  sum_s h_s * c_s  (Eq. 6) subject to
+ *     sum_s  l_s(b_s, c_s) + q_s(b_s)  <=  SLO            (Eq. 5)
+ *     lambda <= h_s * thr_s(b_s, c_s),  thr = b / l(b, c)   (Eq. 6)
+ * where l is the profiled processing latency and q the queuing delay of Eq. 4,
+ * q = (b - 1) / lambda.  Latencies are discretised to buckets of bucket_us:
+ * a stage occupies ceil(l / w) + ceil(q / w) buckets out of T = floor(SLO / w).
+ * Instances are independent and solved in one batch.
+ *
+ * Method (Algorithm 1, restructured): per stage the candidates are reduced to a
+ * per-bucket minimum cost G_s[l]; stages are combined by the recurrence
+ *     F_0 = G_0,   F_s[t] = min_{0<=l<=t} F_{s-1}[t-l] + G_s[l]
+ * and the configuration is read back from the argmin tables.  Ties resolve to
+ * the lowest index everywhere (lowest total latency, then lowest latency of the
+ * last stage, ..., then lowest candidate index per stage), which is what
+ * Algorithm 1's strict '<' in ascending loop order yields.
+ *
+ * Conventions for every entry point:
+ *  - returns THEMIS_OK or a negative THEMIS_E_* code; never throws;
+ *  - "d_" pointers are DEVICE memory, "h_" pointers are HOST memory; all are
+ *    owned by the caller and must stay valid until the stream work completes;
+ *  - nothing is allocated on the device; scratch comes from the caller's
+ *    workspace (see themis_workspace_bytes);
+ *  - work is enqueued on the given CUDA stream (a cudaStream_t passed as void*,
+ *    NULL = default stream) and the call returns without synchronising, except
+ *    themis_solve_batch_host, which synchronises the stream before returning;
+ *  - scalar arguments are validated on the host before anything is launched;
+ *    bad array contents (lambda = 0, latency <= 0, replicas < 1) are detected on
+ *    the device and reported per instance in status[n];
+ *  - an instance with no feasible configuration is not an error: status[n] = 1
+ *    (Algorithm 1's "no solution" branch).
+ */
+#ifndef THEMIS_H_
+#define THEMIS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define THEMIS_VERSION 100
+
+/* problem limits */
+#define THEMIS_MAX_BATCH_SIZES 16
+#define THEMIS_MAX_STAGES 64
+#define THEMIS_MAX_T 16383        /* budget in buckets (argmin tables are 14-bit) */
+#define THEMIS_MAX_CANDIDATES 65535 /* per stage (candidate index is uint16) */
+#define THEMIS_MAX_TOTAL_COST 131070 /* n_stages * h_max * c_max must not exceed it */
+
+/* themis_problem_t.flags */
+#define THEMIS_QUEUE_PER_REPLICA 1u /* q = (b-1) * h / lambda: every replica fills
+                                       its own batch.  Clear: q = (b-1)/lambda, Eq. 4 */
+
+/* return codes */
+#define THEMIS_OK 0
+#define THEMIS_E_INVALID_ARG (-1)
+#define THEMIS_E_UNSUPPORTED_SIZE (-2)
+#define THEMIS_E_WORKSPACE_TOO_SMALL (-3)
+#define THEMIS_E_CUDA (-4)
+
+/* per-instance status */
+#define THEMIS_STATUS_OK 0
+#define THEMIS_STATUS_INFEASIBLE 1
+#define THEMIS_STATUS_BAD_INPUT (-1)   /* lambda = 0, a latency <= 0 or replicas < 1 */
+#define THEMIS_STATUS_TIMEOUT (-2)     /* a bounded on-device wait expired */
+
+/* value of an empty bucket in the G table of the workspace */
+#define THEMIS_G_INF INT32_MAX
+
+typedef struct {
+    int32_t n_instances;   /* N >= 1 */
+    int32_t n_stages;      /* S in 1..THEMIS_MAX_STAGES */
+    int32_t n_profiles;    /* P >= 1 distinct pipelines (sets of latency tables) */
+    int32_t c_max;         /* cores per replica range over 1..c_max */
+    int32_t n_batch;       /* number of batch sizes, 1..THEMIS_MAX_BATCH_SIZES */
+    int32_t batch_sizes[THEMIS_MAX_BATCH_SIZES]; /* strictly increasing, 1..65536 */
+    int32_t h_max;         /* joint: replicas range over 1..h_max; vertical: ignored */
+    int32_t slo_us;        /* SLO in microseconds */
+    int32_t bucket_us;     /* bucket width w; T = slo_us / bucket_us, 1 <= T <= THEMIS_MAX_T */
+    uint32_t flags;        /* THEMIS_QUEUE_PER_REPLICA or 0 */
+} themis_problem_t;
+
+/* Result arrays, caller-owned and caller-sized.  Device pointers for the d_
+ * entry points, host pointers for themis_solve_batch_host. */
+typedef struct {
+    int32_t *h;               /* [N][S] row-major; 0 where unsolved */
+    int32_t *c;               /* [N][S] */
+    int32_t *b;               /* [N][S] */
+    int32_t *total_cost;      /* [N] sum_s h*c; -1 where unsolved */
+    int32_t *latency_buckets; /* [N] sum of stage latencies in buckets (<= T); -1 where unsolved */
+    int32_t *status;          /* [N] THEMIS_STATUS_* */
+} themis_result_t;
+
+/* Where the intermediate tables live inside a workspace (byte offsets from its
+ * start; rows are row_pitch entries long, entries beyond T are padding).
+ *   G    int32  [N][S][row_pitch]  per-bucket minimum cost, THEMIS_G_INF if empty
+ *   Garg uint16 [N][S][row_pitch]  lowest candidate index attaining G (0 if empty)
+ *   A    uint16 [N][S][row_pitch]  A[s][t] = lowest l attaining F_s[t] (row 0 unused,
+ *                                  0 where F_s[t] is unreachable)
+ *   F    int32  [N][row_pitch]     last prefix table F_{S-1}, THEMIS_G_INF if unreachable
+ * Candidate index: idx = ((h-1)*c_max + (c-1))*n_batch + bi (joint),
+ *                  idx = (c-1)*n_batch + bi (vertical). */
+typedef struct {
+    size_t g_offset, garg_offset, a_offset, f_offset, flag_offset;
+    size_t total_bytes;
+    int32_t row_pitch;
+    int32_t T;
+} themis_workspace_layout_t;
+
+/* Device workspace needed by the d_ entry points for this problem
+ * (8 * N * S * row_pitch bytes plus small terms).  vertical != 0 selects the
+ * h-fixed variant.  Fails with INVALID_ARG / UNSUPPORTED_SIZE like the solvers. */
+int themis_workspace_bytes(const themis_problem_t *problem, int vertical, size_t *out_bytes);
+int themis_workspace_layout(const themis_problem_t *problem, int vertical,
+                            themis_workspace_layout_t *out_layout);
+
+/*
+ * Joint solver (Eq. 6 over h in 1..h_max, c in 1..c_max, b in batch_sizes).
+ *   d_lat_us       [P][S][c_max][n_batch] int32, batch index fastest: profiled
+ *                  latency of one batch in microseconds, >= 1
+ *   d_profile_id   [N] int32 in 0..P-1, or NULL (every instance uses profile 0)
+ *   d_lambda_mrps  [N] uint32 arrival rate in milli-requests per second, >= 1
+ *   out            device result arrays
+ *   d_workspace    device scratch, 256-byte aligned, >= themis_workspace_bytes
+ * Runs the candidate-scoring kernel, then the min-plus/backtrack kernel.
+ */
+int themis_solve_batch(const themis_problem_t *problem, const int32_t *d_lat_us,
+                       const int32_t *d_profile_id, const uint32_t *d_lambda_mrps,
+                       themis_result_t out, void *d_workspace, size_t workspace_bytes,
+                       void *cuda_stream);
+
+/*
+ * In-place vertical-only variant (Algorithm 1): replicas are fixed,
+ *   d_replicas     [N][S] int32, >= 1
+ * candidates range over (c, b) only and a stage costs replicas * c.
+ */
+int themis_solve_vertical_batch(const themis_problem_t *problem, const int32_t *d_lat_us,
+                                const int32_t *d_profile_id, const uint32_t *d_lambda_mrps,
+                                const int32_t *d_replicas, themis_result_t out,
+                                void *d_workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * The two halves of the solvers, for checking and timing each step on its own.
+ * themis_score_batch fills G and Garg of the workspace (candidate scoring: the
+ * inner loops of Algorithm 1 with Eq. 4 and the throughput test of Eq. 6);
+ * themis_minplus_batch consumes them (recurrence, final scan, backtrack) and
+ * fills A, F and the result arrays.  d_replicas = NULL selects the joint problem.
+ * Calling them back to back on one stream equals the corresponding solver.
+ */
+int themis_score_batch(const themis_problem_t *problem, const int32_t *d_lat_us,
+                       const int32_t *d_profile_id, const uint32_t *d_lambda_mrps,
+                       const int32_t *d_replicas, void *d_workspace, size_t workspace_bytes,
+                       void *cuda_stream);
+int themis_minplus_batch(const themis_problem_t *problem, const int32_t *d_replicas,
+                         themis_result_t out, void *d_workspace, size_t workspace_bytes,
+                         void *cuda_stream);
+
+/*
+ * Host-buffer variant: inputs and results are HOST arrays (pinned memory makes
+ * the copies asynchronous).  Copies the inputs into the workspace, solves, copies
+ * the results back and synchronises the stream.  h_replicas = NULL selects the
+ * joint problem.  The workspace must hold themis_host_workspace_bytes.
+ */
+int themis_host_workspace_bytes(const themis_problem_t *problem, int vertical, size_t *out_bytes);
+int themis_solve_batch_host(const themis_problem_t *problem, const int32_t *h_lat_us,
+                            const int32_t *h_profile_id, const uint32_t *h_lambda_mrps,
+                            const int32_t *h_replicas, themis_result_t h_out,
+                            void *d_workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Integer-ALU throughput probe (not part of the method): every thread runs
+ * `iters` rounds of 16 independent add-then-min updates, the operation pair of
+ * the recurrence, in one of three instruction forms:
+ *   mode 0: separate 32-bit add and unsigned min;
+ *   mode 1: the fused add-min instruction (one instruction per update);
+ *   mode 2: one add per update and one three-input min per two updates.
+ * Launches `blocks` x `threads` and writes one word per thread to d_sink
+ * (blocks*threads uint32).  Updates performed = blocks*threads*iters*16.
+ */
+int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_sink,
+                     void *cuda_stream);
+
+/* Tuning knob of the min-plus kernel: consecutive budget cells per thread
+ * (8 or 16); 0 restores the built-in choice.  Results do not depend on it. */
+int themis_set_minplus_tile(int cells_per_thread);
+
+/* Text for a return code; for THEMIS_E_CUDA includes the last CUDA error seen by
+ * the calling thread.  The pointer stays valid until the thread's next call. */
+const char *themis_strerror(int code);
+int themis_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* THEMIS_H_ */

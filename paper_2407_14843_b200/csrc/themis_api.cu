@@ -1,0 +1,310 @@
+// C ABI of libthemis: argument validation, workspace carving, kernel launches.
+#include <stdio.h>
+#include <string.h>
+
+#include "themis_internal.h"
+
+namespace themis {
+namespace {
+
+thread_local cudaError_t t_last_cuda = cudaSuccess;
+thread_local char t_msg[256];
+int g_tile = 0;   // min-plus cells per thread; 0 = built-in choice
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+int fail_cuda(cudaError_t e)
+{
+    t_last_cuda = e;
+    return THEMIS_E_CUDA;
+}
+
+// Host-side validation of the scalar description.  Fills T, K.
+int validate(const themis_problem_t *pr, int vertical, int32_t *T_out, int32_t *K_out)
+{
+    if (!pr) return THEMIS_E_INVALID_ARG;
+    if (pr->n_instances < 1 || pr->n_stages < 1 || pr->n_profiles < 1 || pr->c_max < 1 || pr->n_batch < 1)
+        return THEMIS_E_INVALID_ARG;
+    if (pr->slo_us < 1 || pr->bucket_us < 1) return THEMIS_E_INVALID_ARG;
+    if (pr->flags & ~THEMIS_QUEUE_PER_REPLICA) return THEMIS_E_INVALID_ARG;
+    if (!vertical && pr->h_max < 1) return THEMIS_E_INVALID_ARG;
+    if (pr->n_batch > THEMIS_MAX_BATCH_SIZES) return THEMIS_E_UNSUPPORTED_SIZE;
+    for (int i = 0; i < pr->n_batch; ++i) {
+        if (pr->batch_sizes[i] < 1 || pr->batch_sizes[i] > 65536) return THEMIS_E_INVALID_ARG;
+        if (i > 0 && pr->batch_sizes[i] <= pr->batch_sizes[i - 1]) return THEMIS_E_INVALID_ARG;
+    }
+    if (pr->n_stages > THEMIS_MAX_STAGES) return THEMIS_E_UNSUPPORTED_SIZE;
+    const int64_t T = pr->slo_us / pr->bucket_us;
+    if (T < 1) return THEMIS_E_INVALID_ARG;
+    if (T > THEMIS_MAX_T) return THEMIS_E_UNSUPPORTED_SIZE;
+    const int64_t h = vertical ? 1 : pr->h_max;
+    const int64_t K = h * pr->c_max * pr->n_batch;
+    if (K > THEMIS_MAX_CANDIDATES) return THEMIS_E_UNSUPPORTED_SIZE;
+    // joint: the largest possible total must stay below the "unreachable" cost;
+    // vertical: the same bound is checked on the device against replicas[].
+    if (!vertical && (int64_t)pr->n_stages * pr->h_max * pr->c_max > THEMIS_MAX_TOTAL_COST)
+        return THEMIS_E_UNSUPPORTED_SIZE;
+    if (vertical && (int64_t)pr->n_stages * pr->c_max > THEMIS_MAX_TOTAL_COST) return THEMIS_E_UNSUPPORTED_SIZE;
+    // shared-memory tables of the scoring kernel: n_batch * h entries, two tables
+    if ((int64_t)pr->n_batch * h > 8192) return THEMIS_E_UNSUPPORTED_SIZE;
+    *T_out = (int32_t)T;
+    *K_out = (int32_t)K;
+    return THEMIS_OK;
+}
+
+int layout_of(const themis_problem_t *pr, int vertical, themis_workspace_layout_t *L)
+{
+    int32_t T, K;
+    int rc = validate(pr, vertical, &T, &K);
+    if (rc != THEMIS_OK) return rc;
+    const size_t pitch = (size_t)(T + 1 + kRowAlign - 1) / kRowAlign * kRowAlign;
+    const size_t rows = (size_t)pr->n_instances * pr->n_stages;
+    size_t off = 0;
+    L->g_offset = off;    off = align_up(off + rows * pitch * sizeof(int32_t));
+    L->garg_offset = off; off = align_up(off + rows * pitch * sizeof(uint16_t));
+    L->a_offset = off;    off = align_up(off + rows * pitch * sizeof(uint16_t));
+    L->f_offset = off;    off = align_up(off + (size_t)pr->n_instances * pitch * sizeof(int32_t));
+    L->flag_offset = off; off = align_up(off + (size_t)pr->n_instances * sizeof(int32_t));
+    L->total_bytes = off;
+    L->row_pitch = (int32_t)pitch;
+    L->T = T;
+    return THEMIS_OK;
+}
+
+int make_params(const themis_problem_t *pr, int vertical, void *ws, size_t ws_bytes, Params *P)
+{
+    themis_workspace_layout_t L;
+    int rc = layout_of(pr, vertical, &L);
+    if (rc != THEMIS_OK) return rc;
+    if (!ws || ((uintptr_t)ws & (kAlign - 1))) return THEMIS_E_INVALID_ARG;
+    if (ws_bytes < L.total_bytes) return THEMIS_E_WORKSPACE_TOO_SMALL;
+    memset(P, 0, sizeof(*P));
+    P->prob = *pr;
+    P->T = L.T;
+    P->pitch = L.row_pitch;
+    P->vertical = vertical ? 1 : 0;
+    P->K = (vertical ? 1 : pr->h_max) * pr->c_max * pr->n_batch;
+    char *base = static_cast<char *>(ws);
+    P->G = reinterpret_cast<int32_t *>(base + L.g_offset);
+    P->Garg = reinterpret_cast<uint16_t *>(base + L.garg_offset);
+    P->A = reinterpret_cast<uint16_t *>(base + L.a_offset);
+    P->F = reinterpret_cast<int32_t *>(base + L.f_offset);
+    P->inst_flag = reinterpret_cast<int32_t *>(base + L.flag_offset);
+    return THEMIS_OK;
+}
+
+bool result_ok(const themis_result_t &o)
+{
+    return o.h && o.c && o.b && o.total_cost && o.latency_buckets && o.status;
+}
+
+int score_impl(const themis_problem_t *pr, const int32_t *lat, const int32_t *pid, const uint32_t *lam,
+               const int32_t *rep, int vertical, void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    Params P;
+    int rc = make_params(pr, vertical, ws, ws_bytes, &P);
+    if (rc != THEMIS_OK) return rc;
+    if (!lat || !lam || (vertical && !rep)) return THEMIS_E_INVALID_ARG;
+    P.lat_us = lat; P.profile_id = pid; P.lambda_mrps = lam; P.replicas = rep;
+    cudaError_t e = launch_score(P, st);
+    return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
+}
+
+int minplus_impl(const themis_problem_t *pr, const int32_t *rep, int vertical, themis_result_t out, void *ws,
+                 size_t ws_bytes, cudaStream_t st)
+{
+    Params P;
+    int rc = make_params(pr, vertical, ws, ws_bytes, &P);
+    if (rc != THEMIS_OK) return rc;
+    if (!result_ok(out) || (vertical && !rep)) return THEMIS_E_INVALID_ARG;
+    P.replicas = rep; P.out = out;
+    cudaError_t e = launch_minplus(P, g_tile, st);
+    return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
+}
+
+int solve_impl(const themis_problem_t *pr, const int32_t *lat, const int32_t *pid, const uint32_t *lam,
+               const int32_t *rep, int vertical, themis_result_t out, void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    int32_t T, K;
+    int rc = validate(pr, vertical, &T, &K);
+    if (rc != THEMIS_OK) return rc;
+    if (!result_ok(out)) return THEMIS_E_INVALID_ARG;
+    rc = score_impl(pr, lat, pid, lam, rep, vertical, ws, ws_bytes, st);
+    if (rc != THEMIS_OK) return rc;
+    return minplus_impl(pr, rep, vertical, out, ws, ws_bytes, st);
+}
+
+// Staging area appended to the solver workspace by the host-buffer variant.
+struct HostStage {
+    size_t lat, pid, lam, rep, h, c, b, cost, latb, status, total;
+};
+
+int host_stage_of(const themis_problem_t *pr, int vertical, size_t base, HostStage *H)
+{
+    const size_t N = pr->n_instances, S = pr->n_stages;
+    size_t off = align_up(base);
+    H->lat = off; off = align_up(off + (size_t)pr->n_profiles * S * pr->c_max * pr->n_batch * 4);
+    H->pid = off; off = align_up(off + N * 4);
+    H->lam = off; off = align_up(off + N * 4);
+    H->rep = off; off = align_up(off + (vertical ? N * S * 4 : 0));
+    H->h = off; off = align_up(off + N * S * 4);
+    H->c = off; off = align_up(off + N * S * 4);
+    H->b = off; off = align_up(off + N * S * 4);
+    H->cost = off; off = align_up(off + N * 4);
+    H->latb = off; off = align_up(off + N * 4);
+    H->status = off; off = align_up(off + N * 4);
+    H->total = off;
+    return THEMIS_OK;
+}
+
+}  // namespace
+}  // namespace themis
+
+using namespace themis;
+
+extern "C" {
+
+int themis_version(void) { return THEMIS_VERSION; }
+
+const char *themis_strerror(int code)
+{
+    switch (code) {
+        case THEMIS_OK: return "ok";
+        case THEMIS_E_INVALID_ARG: return "invalid argument";
+        case THEMIS_E_UNSUPPORTED_SIZE: return "problem size outside the supported limits";
+        case THEMIS_E_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case THEMIS_E_CUDA:
+            snprintf(t_msg, sizeof(t_msg), "CUDA error: %s", cudaGetErrorString(t_last_cuda));
+            return t_msg;
+        default: return "unknown error code";
+    }
+}
+
+int themis_workspace_layout(const themis_problem_t *problem, int vertical, themis_workspace_layout_t *out_layout)
+{
+    if (!out_layout) return THEMIS_E_INVALID_ARG;
+    return layout_of(problem, vertical, out_layout);
+}
+
+int themis_workspace_bytes(const themis_problem_t *problem, int vertical, size_t *out_bytes)
+{
+    if (!out_bytes) return THEMIS_E_INVALID_ARG;
+    themis_workspace_layout_t L;
+    int rc = layout_of(problem, vertical, &L);
+    if (rc == THEMIS_OK) *out_bytes = L.total_bytes;
+    return rc;
+}
+
+int themis_solve_batch(const themis_problem_t *problem, const int32_t *d_lat_us, const int32_t *d_profile_id,
+                       const uint32_t *d_lambda_mrps, themis_result_t out, void *d_workspace,
+                       size_t workspace_bytes, void *cuda_stream)
+{
+    return solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, nullptr, 0, out, d_workspace,
+                      workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int themis_solve_vertical_batch(const themis_problem_t *problem, const int32_t *d_lat_us,
+                                const int32_t *d_profile_id, const uint32_t *d_lambda_mrps,
+                                const int32_t *d_replicas, themis_result_t out, void *d_workspace,
+                                size_t workspace_bytes, void *cuda_stream)
+{
+    if (!d_replicas) return THEMIS_E_INVALID_ARG;
+    return solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, d_replicas, 1, out, d_workspace,
+                      workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int themis_score_batch(const themis_problem_t *problem, const int32_t *d_lat_us, const int32_t *d_profile_id,
+                       const uint32_t *d_lambda_mrps, const int32_t *d_replicas, void *d_workspace,
+                       size_t workspace_bytes, void *cuda_stream)
+{
+    return score_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, d_replicas, d_replicas != nullptr,
+                      d_workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int themis_minplus_batch(const themis_problem_t *problem, const int32_t *d_replicas, themis_result_t out,
+                         void *d_workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    return minplus_impl(problem, d_replicas, d_replicas != nullptr, out, d_workspace, workspace_bytes,
+                        static_cast<cudaStream_t>(cuda_stream));
+}
+
+int themis_host_workspace_bytes(const themis_problem_t *problem, int vertical, size_t *out_bytes)
+{
+    if (!out_bytes) return THEMIS_E_INVALID_ARG;
+    themis_workspace_layout_t L;
+    int rc = layout_of(problem, vertical, &L);
+    if (rc != THEMIS_OK) return rc;
+    HostStage H;
+    host_stage_of(problem, vertical, L.total_bytes, &H);
+    *out_bytes = H.total;
+    return THEMIS_OK;
+}
+
+int themis_solve_batch_host(const themis_problem_t *problem, const int32_t *h_lat_us, const int32_t *h_profile_id,
+                            const uint32_t *h_lambda_mrps, const int32_t *h_replicas, themis_result_t h_out,
+                            void *d_workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    const int vertical = h_replicas != nullptr;
+    themis_workspace_layout_t L;
+    int rc = layout_of(problem, vertical, &L);
+    if (rc != THEMIS_OK) return rc;
+    if (!h_lat_us || !h_lambda_mrps || !result_ok(h_out)) return THEMIS_E_INVALID_ARG;
+    if (!d_workspace || ((uintptr_t)d_workspace & (kAlign - 1))) return THEMIS_E_INVALID_ARG;
+    HostStage H;
+    host_stage_of(problem, vertical, L.total_bytes, &H);
+    if (workspace_bytes < H.total) return THEMIS_E_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char *base = static_cast<char *>(d_workspace);
+    const size_t N = problem->n_instances, S = problem->n_stages;
+    const size_t lat_bytes = (size_t)problem->n_profiles * S * problem->c_max * problem->n_batch * 4;
+    cudaError_t e;
+#define THEMIS_COPY(dst, src, bytes, kind)                                    \
+    do {                                                                      \
+        e = cudaMemcpyAsync((dst), (src), (bytes), (kind), st);               \
+        if (e != cudaSuccess) return fail_cuda(e);                            \
+    } while (0)
+    THEMIS_COPY(base + H.lat, h_lat_us, lat_bytes, cudaMemcpyHostToDevice);
+    if (h_profile_id) THEMIS_COPY(base + H.pid, h_profile_id, N * 4, cudaMemcpyHostToDevice);
+    THEMIS_COPY(base + H.lam, h_lambda_mrps, N * 4, cudaMemcpyHostToDevice);
+    if (vertical) THEMIS_COPY(base + H.rep, h_replicas, N * S * 4, cudaMemcpyHostToDevice);
+    themis_result_t d_out;
+    d_out.h = reinterpret_cast<int32_t *>(base + H.h);
+    d_out.c = reinterpret_cast<int32_t *>(base + H.c);
+    d_out.b = reinterpret_cast<int32_t *>(base + H.b);
+    d_out.total_cost = reinterpret_cast<int32_t *>(base + H.cost);
+    d_out.latency_buckets = reinterpret_cast<int32_t *>(base + H.latb);
+    d_out.status = reinterpret_cast<int32_t *>(base + H.status);
+    rc = solve_impl(problem, reinterpret_cast<const int32_t *>(base + H.lat),
+                    h_profile_id ? reinterpret_cast<const int32_t *>(base + H.pid) : nullptr,
+                    reinterpret_cast<const uint32_t *>(base + H.lam),
+                    vertical ? reinterpret_cast<const int32_t *>(base + H.rep) : nullptr, vertical, d_out,
+                    d_workspace, L.total_bytes, st);
+    if (rc != THEMIS_OK) return rc;
+    THEMIS_COPY(h_out.h, d_out.h, N * S * 4, cudaMemcpyDeviceToHost);
+    THEMIS_COPY(h_out.c, d_out.c, N * S * 4, cudaMemcpyDeviceToHost);
+    THEMIS_COPY(h_out.b, d_out.b, N * S * 4, cudaMemcpyDeviceToHost);
+    THEMIS_COPY(h_out.total_cost, d_out.total_cost, N * 4, cudaMemcpyDeviceToHost);
+    THEMIS_COPY(h_out.latency_buckets, d_out.latency_buckets, N * 4, cudaMemcpyDeviceToHost);
+    THEMIS_COPY(h_out.status, d_out.status, N * 4, cudaMemcpyDeviceToHost);
+#undef THEMIS_COPY
+    e = cudaStreamSynchronize(st);
+    return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
+}
+
+int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_sink, void *cuda_stream)
+{
+    if (mode < 0 || mode > 4 || blocks < 1 || threads < 32 || threads > 1024 || iters < 1 || !d_sink)
+        return THEMIS_E_INVALID_ARG;
+    cudaError_t e = launch_alu_probe(mode, blocks, threads, iters, d_sink, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
+}
+
+int themis_set_minplus_tile(int cells_per_thread)
+{
+    if (cells_per_thread != 0 && cells_per_thread != 8 && cells_per_thread != 16) return THEMIS_E_INVALID_ARG;
+    g_tile = cells_per_thread;
+    return THEMIS_OK;
+}
+
+}  // extern "C"

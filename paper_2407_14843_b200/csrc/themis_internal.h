@@ -1,0 +1,47 @@
+// Internal declarations shared by the translation units of libthemis.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "themis.h"
+
+namespace themis {
+
+// Cost field of a packed key: 17 bits.  Valid totals are <= THEMIS_MAX_TOTAL_COST
+// = kInfCost - 1, so the sum of two fields (<= 2^18 - 2) plus a 14-bit index still
+// fits an unsigned 32-bit word and "unreachable" never needs a branch.
+constexpr uint32_t kIdxBits = 14;
+constexpr uint32_t kIdxMask = (1u << kIdxBits) - 1u;
+constexpr uint32_t kInfCost = (1u << 17) - 1u;
+constexpr uint32_t kInfKey = kInfCost << kIdxBits;
+
+// Rows of the workspace tables are padded to a multiple of this many entries,
+// so every row starts 64-byte aligned (uint16) / 128-byte aligned (int32) and
+// bulk copies of whole rows meet the 16-byte rule.
+constexpr int kRowAlign = 32;
+
+struct Params {
+    themis_problem_t prob;
+    int32_t T;          // budget in buckets
+    int32_t pitch;      // row pitch of G / Garg / A / F in entries
+    int32_t vertical;   // 1: h fixed per stage from replicas[]
+    int32_t K;          // candidates per stage
+    const int32_t *lat_us;
+    const int32_t *profile_id;
+    const uint32_t *lambda_mrps;
+    const int32_t *replicas;
+    int32_t *G;
+    uint16_t *Garg;
+    uint16_t *A;
+    int32_t *F;
+    int32_t *inst_flag;  // [N] nonzero = bad input seen by the scoring kernel
+    themis_result_t out;
+};
+
+cudaError_t launch_score(const Params &p, cudaStream_t stream);
+cudaError_t launch_minplus(const Params &p, int tile, cudaStream_t stream);
+cudaError_t launch_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *sink,
+                             cudaStream_t stream);
+
+}  // namespace themis

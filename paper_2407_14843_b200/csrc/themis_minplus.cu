@@ -1,0 +1,321 @@
+// Min-plus stage recurrence, final scan and backtrack (Algorithm 1's budget
+// loop with the candidate minimum hoisted out), one thread block per instance:
+//
+//   F_0 = G_0,   F_s[t] = min_{0<=l<=t} F_{s-1}[t-l] + G_s[l],   A_s[t] = lowest such l
+//
+// Arithmetic.  Both operands are kept as packed unsigned keys
+//   Fk[i] = cost << 14                (low 14 bits zero)
+//   Gk[l] = cost << 14 | l
+// so one fused add-min per (t, l) cell carries the argmin along: the smallest
+// sum has the smallest cost and, among equal costs, the smallest l.  The cost
+// field is 17 bits with "unreachable" = 2^17 - 1; the sum of two fields fits 18
+// bits, so no cell needs a branch or can overflow.
+//
+// Tiling.  A thread owns R consecutive budget cells t0..t0+R-1 and walks l
+// upward in chunks of R.  Per chunk it loads R new words of F (its window
+// slides down by R) and R words of G (the same address for every lane of the
+// warp, a broadcast) and performs R*R cell updates from registers.  F is stored
+// in chunks of R words padded to R+4 so that the 16-byte loads of consecutive
+// lanes fall into distinct bank groups; one extra chunk of "unreachable" in
+// front of F[0] stands for every negative index.
+//
+// Staging.  Row s+1 of G is fetched by a bulk asynchronous copy into the other
+// half of a double buffer, completion signalled on an mbarrier, while stage s
+// computes.  Every wait on an mbarrier is bounded; on expiry the block reports
+// THEMIS_STATUS_TIMEOUT for its instance and leaves.
+#include "themis_internal.h"
+
+namespace themis {
+namespace {
+
+constexpr uint32_t kWaitLimit = 1u << 20;   // try_wait attempts before giving up
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
+                 : "memory");
+}
+
+// One-dimensional bulk asynchronous copy global -> this block's shared memory.
+// Both addresses 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_load(void *dst_smem, const void *src_gmem, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+            smem_addr(dst_smem)),
+        "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar))
+        : "memory");
+}
+
+// Bounded wait for the given phase parity; false if the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+{
+    const uint32_t a = smem_addr(bar);
+    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(a), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+template <int R>
+struct Tile {
+    static constexpr int kChunkStride = R + 4;   // words between chunk starts in shared F
+};
+
+// One chunk step: loads the next-lower chunk of F into w_lo and R keys of G, then
+// updates acc[r] = min(acc[r], F[t0 + r - (l0 + k)] + G[l0 + k]) for all r, k.
+// w_hi holds F[m .. m+R-1] and w_lo receives F[m-R .. m-1], m = t0 - l0.
+template <int R>
+__device__ __forceinline__ void chunk_step(const uint32_t (&w_hi)[R], uint32_t (&w_lo)[R], uint32_t (&acc)[R],
+                                           const uint32_t *f_chunk, const uint32_t *g_chunk)
+{
+#pragma unroll
+    for (int v = 0; v < R / 4; ++v) {
+        const uint4 x = *reinterpret_cast<const uint4 *>(f_chunk + 4 * v);
+        w_lo[4 * v + 0] = x.x; w_lo[4 * v + 1] = x.y; w_lo[4 * v + 2] = x.z; w_lo[4 * v + 3] = x.w;
+    }
+#pragma unroll
+    for (int v = 0; v < R / 4; ++v) {
+        const uint4 g4 = *reinterpret_cast<const uint4 *>(g_chunk + 4 * v);
+        const uint32_t g[4] = {g4.x, g4.y, g4.z, g4.w};
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+            const int k = 4 * v + kk;
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const int i = R + r - k;                       // 1 .. 2R-1
+                const uint32_t f = i >= R ? w_hi[i - R] : w_lo[i];
+                acc[r] = __viaddmin_u32(f, g[kk], acc[r]);
+            }
+        }
+    }
+}
+
+template <int R, int MAXT>
+__global__ void __launch_bounds__(MAXT)
+minplus_kernel(const Params p)
+{
+    extern __shared__ __align__(128) uint32_t smem[];
+    constexpr int CS = Tile<R>::kChunkStride;
+    const int n = blockIdx.x;
+    const int tid = threadIdx.x;
+    const int NT = blockDim.x;
+    const int T = p.T, pitch = p.pitch, S = p.prob.n_stages;
+    const int Tp = NT * R;                              // padded budget length, >= pitch
+
+    uint32_t *Fs = smem;                                // (NT + 1) chunks of CS words; chunk -1 first
+    uint32_t *Gbuf0 = Fs + (NT + 1) * CS;
+    uint32_t *Gbuf1 = Gbuf0 + Tp;
+    uint64_t *mbar = reinterpret_cast<uint64_t *>(Gbuf1 + Tp);
+    uint32_t *red = reinterpret_cast<uint32_t *>(mbar + 2);   // 32 words for the block reduction
+
+    const int t0 = tid * R;
+    uint32_t *my_chunk = Fs + (tid + 1) * CS;
+    const uint32_t row_bytes = (uint32_t)pitch * 4u;
+    const int32_t *G_inst = p.G + (size_t)n * S * pitch;
+
+    int32_t *h_o = p.out.h + (size_t)n * S, *c_o = p.out.c + (size_t)n * S, *b_o = p.out.b + (size_t)n * S;
+    // Writes the "no configuration" result with the given status (one thread).
+    auto write_unsolved = [&](int status) {
+        for (int s = 0; s < S; ++s) { h_o[s] = 0; c_o[s] = 0; b_o[s] = 0; }
+        p.out.total_cost[n] = -1;
+        p.out.latency_buckets[n] = -1;
+        p.out.status[n] = status;
+    };
+    if (p.inst_flag[n] != 0) {                          // bad input seen while scoring
+        if (tid == 0) write_unsolved(THEMIS_STATUS_BAD_INPUT);
+        return;
+    }
+
+    if (tid == 0) {
+        mbar_init(&mbar[0], 1);
+        mbar_init(&mbar[1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // "unreachable" in front of F[0], and behind the loaded part of each G buffer
+    if (tid < CS) Fs[tid] = kInfKey;
+    for (int l = pitch + tid; l < Tp; l += NT) {
+        Gbuf0[l] = kInfKey | (uint32_t)l;
+        Gbuf1[l] = kInfKey | (uint32_t)l;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_expect_tx(&mbar[0], row_bytes);
+        bulk_load(Gbuf0, G_inst, row_bytes, &mbar[0]);
+        if (S > 1) {
+            mbar_expect_tx(&mbar[1], row_bytes);
+            bulk_load(Gbuf1, G_inst + pitch, row_bytes, &mbar[1]);
+        }
+    }
+    int failed = 0;                                     // a bounded wait ran out
+    int pend0 = 0, pend1 = S > 1 ? 0 : -1;              // phase parity of a copy in flight, or -1
+
+    // stage 0: F_0 = G_0
+    if (!mbar_wait(&mbar[0], 0)) failed = 1; else pend0 = -1;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const uint32_t raw = Gbuf0[t0 + r];              // raw cost, or >= kInfCost when empty/padding
+        my_chunk[r] = min(raw, kInfCost) << kIdxBits;
+    }
+    failed = __syncthreads_or(failed);
+
+    for (int s = 1; s < S && !failed; ++s) {
+        const int cur = s & 1;
+        uint32_t *Gk = cur ? Gbuf1 : Gbuf0;
+        const int parity = (s >> 1) & 1;
+        if (!mbar_wait(&mbar[cur], (uint32_t)parity)) failed = 1;
+        else if (cur) pend1 = -1; else pend0 = -1;
+        // raw costs -> packed keys, in place (own R entries)
+        if (t0 < pitch) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const uint32_t raw = Gk[t0 + r];
+                Gk[t0 + r] = (min(raw, kInfCost) << kIdxBits) | (uint32_t)(t0 + r);
+            }
+        }
+        failed = __syncthreads_or(failed);               // keys and F_{s-1} visible to all
+        if (failed) break;
+        if (s + 1 < S) {                                 // the other buffer is free again
+            const int nxt = cur ^ 1;
+            if (tid == 0) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_expect_tx(&mbar[nxt], row_bytes);
+                bulk_load(nxt ? Gbuf1 : Gbuf0, G_inst + (size_t)(s + 1) * pitch, row_bytes, &mbar[nxt]);
+            }
+            if (nxt) pend1 = ((s + 1) >> 1) & 1; else pend0 = ((s + 1) >> 1) & 1;
+        }
+
+        uint32_t acc[R], wa[R], wb[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) { acc[r] = 0xFFFFFFFFu; wa[r] = my_chunk[r]; }
+        // All lanes of a warp walk the same l so that G is a broadcast; lanes
+        // that run past their own range read the "unreachable" chunk in front.
+        const int q_end = tid | 31;
+        int f_off = tid * CS;                            // word offset of chunk tid-1
+        const uint32_t *g = Gk;
+        for (int q = 0; q <= q_end; q += 2) {
+            chunk_step<R>(wa, wb, acc, Fs + max(f_off, 0), g);
+            chunk_step<R>(wb, wa, acc, Fs + max(f_off - CS, 0), g + R);
+            f_off -= 2 * CS;
+            g += 2 * R;
+        }
+        __syncthreads();                                 // every read of F_{s-1} is done
+
+        uint32_t a16[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const bool inf = acc[r] >= kInfKey;
+            my_chunk[r] = inf ? kInfKey : (acc[r] & ~kIdxMask);
+            a16[r] = inf ? 0u : (acc[r] & kIdxMask);
+        }
+        if (t0 + R <= pitch) {
+            uint16_t *A_row = p.A + ((size_t)n * S + s) * pitch + t0;
+#pragma unroll
+            for (int v = 0; v < R / 8; ++v) {
+                uint4 o;
+                o.x = a16[8 * v + 0] | (a16[8 * v + 1] << 16);
+                o.y = a16[8 * v + 2] | (a16[8 * v + 3] << 16);
+                o.z = a16[8 * v + 4] | (a16[8 * v + 5] << 16);
+                o.w = a16[8 * v + 6] | (a16[8 * v + 7] << 16);
+                *reinterpret_cast<uint4 *>(A_row + 8 * v) = o;
+            }
+        }
+    }
+    failed = __syncthreads_or(failed);
+
+    if (failed) {
+        // Let our own copies land (bounded) before the block's shared memory goes away.
+        if (pend0 >= 0) mbar_wait(&mbar[0], (uint32_t)pend0);
+        if (pend1 >= 0) mbar_wait(&mbar[1], (uint32_t)pend1);
+        if (tid == 0) write_unsolved(THEMIS_STATUS_TIMEOUT);
+        return;
+    }
+
+    // last prefix table to the workspace, and the final scan: cheapest total,
+    // lowest total latency among equals
+    uint32_t best = 0xFFFFFFFFu;
+    int32_t *F_row = p.F + (size_t)n * pitch;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int t = t0 + r;
+        const uint32_t fk = my_chunk[r];
+        if (t <= T) best = min(best, fk | (uint32_t)t);
+        if (t < pitch) F_row[t] = fk >= kInfKey ? THEMIS_G_INF : (int32_t)(fk >> kIdxBits);
+    }
+    best = __reduce_min_sync(0xFFFFFFFFu, best);
+    if ((tid & 31) == 0) red[tid >> 5] = best;
+    __syncthreads();                                     // also orders this block's A stores
+    if (tid == 0) {
+        for (int w = 1; w < (NT >> 5); ++w) best = min(best, red[w]);
+        if (best >= kInfKey) {
+            write_unsolved(THEMIS_STATUS_INFEASIBLE);
+        } else {
+            const int tstar = (int)(best & kIdxMask);
+            int t = tstar;
+            const int C = p.prob.c_max, NB = p.prob.n_batch;
+            for (int s = S - 1; s >= 0; --s) {
+                const size_t row = ((size_t)n * S + s) * pitch;
+                const int ell = s > 0 ? (int)p.A[row + t] : t;
+                const int idx = (int)p.Garg[row + ell];
+                const int bi = idx % NB, rest = idx / NB;
+                b_o[s] = p.prob.batch_sizes[bi];
+                c_o[s] = rest % C + 1;
+                h_o[s] = p.vertical ? p.replicas[(size_t)n * S + s] : rest / C + 1;
+                t -= ell;
+            }
+            p.out.total_cost[n] = (int32_t)(best >> kIdxBits);
+            p.out.latency_buckets[n] = tstar;
+            p.out.status[n] = THEMIS_STATUS_OK;
+        }
+    }
+}
+
+template <int R, int MAXT>
+cudaError_t launch_variant(const Params &p, int threads, size_t smem, cudaStream_t stream)
+{
+    cudaError_t e = cudaFuncSetAttribute(minplus_kernel<R, MAXT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return e;
+    minplus_kernel<R, MAXT><<<p.prob.n_instances, threads, smem, stream>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_minplus(const Params &p, int tile, cudaStream_t stream)
+{
+    const int cells = p.T + 1;
+    int R = tile;
+    if (R != 8 && R != 16) R = cells <= 2048 ? 8 : 16;
+    if (R == 8 && (cells + 7) / 8 > 1024) R = 16;
+    const int chunks = (cells + R - 1) / R;
+    const int threads = (chunks + 31) / 32 * 32;
+    const size_t words = (size_t)(threads + 1) * (R + 4) + 2u * (size_t)threads * R + 4 + 32;
+    const size_t smem = words * sizeof(uint32_t);
+    if (R == 8)
+        return threads <= 512 ? launch_variant<8, 512>(p, threads, smem, stream)
+                              : launch_variant<8, 1024>(p, threads, smem, stream);
+    return threads <= 512 ? launch_variant<16, 512>(p, threads, smem, stream)
+                          : launch_variant<16, 1024>(p, threads, smem, stream);
+}
+
+}  // namespace themis

@@ -1,0 +1,86 @@
+// Integer-ALU throughput probe: 16 independent add-then-min chains held in
+// registers, the operation pair of the min-plus recurrence, in several
+// instruction forms.  Every update reads two values produced one round earlier,
+// so nothing can be hoisted and no memory is touched.  It measures what the
+// arithmetic pipes sustain; it is not part of the method.
+#include "themis_internal.h"
+
+namespace themis {
+namespace {
+
+constexpr int kChains = 16;
+constexpr int kRoundsPerIter = 4;
+
+template <int MODE>
+__global__ void alu_probe_kernel(int iters, uint32_t *sink)
+{
+    const uint32_t seed = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t g0 = (seed & 7u) + 1u, g1 = ((seed >> 3) & 7u) + 2u;
+    uint32_t r = 0;
+    if (MODE == 4) {
+        float acc[kChains];
+#pragma unroll
+        for (int i = 0; i < kChains; ++i) acc[i] = 1.0e9f - (float)(seed * (i + 1) & 0xFFFF);
+        const float fg0 = (float)g0, fg1 = (float)g1;
+        for (int it = 0; it < iters; ++it) {
+#pragma unroll
+            for (int j = 0; j < kRoundsPerIter; ++j)
+#pragma unroll
+                for (int i = 0; i < kChains; ++i)
+                    acc[i] = fminf(acc[i], acc[(i + 1) % kChains] + ((i & 1) ? fg1 : fg0));
+        }
+#pragma unroll
+        for (int i = 0; i < kChains; ++i) r ^= __float_as_uint(acc[i]);
+    } else {
+        uint32_t acc[kChains];
+#pragma unroll
+        for (int i = 0; i < kChains; ++i) acc[i] = 0xF0000000u - seed * (i + 1);
+        for (int it = 0; it < iters; ++it) {
+#pragma unroll
+            for (int j = 0; j < kRoundsPerIter; ++j) {
+                if (MODE == 0) {            // add, then min: two instructions per update
+#pragma unroll
+                    for (int i = 0; i < kChains; ++i)
+                        acc[i] = min(acc[i], acc[(i + 1) % kChains] + ((i & 1) ? g1 : g0));
+                } else if (MODE == 1) {     // fused add-min: one instruction per update
+#pragma unroll
+                    for (int i = 0; i < kChains; ++i)
+                        acc[i] = __viaddmin_u32(acc[(i + 1) % kChains], (i & 1) ? g1 : g0, acc[i]);
+                } else if (MODE == 2) {     // two adds and one three-input min per two updates
+#pragma unroll
+                    for (int i = 0; i < kChains; i += 2) {
+                        const uint32_t s0 = acc[(i + 1) % kChains] + g0;
+                        const uint32_t s1 = acc[(i + 2) % kChains] + g1;
+                        acc[i] = __vimin3_u32(acc[i], s0, s1);
+                        const uint32_t s2 = acc[(i + 2) % kChains] + g0;
+                        const uint32_t s3 = acc[(i + 3) % kChains] + g1;
+                        acc[i + 1] = __vimin3_u32(acc[i + 1], s2, s3);
+                    }
+                } else {                    // MODE 3: packed 2 x 16-bit fused add-min
+#pragma unroll
+                    for (int i = 0; i < kChains; ++i)
+                        acc[i] = __viaddmin_u16x2(acc[(i + 1) % kChains], (i & 1) ? g1 : g0, acc[i]);
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < kChains; ++i) r ^= acc[i];
+    }
+    sink[blockIdx.x * blockDim.x + threadIdx.x] = r;
+}
+
+}  // namespace
+
+cudaError_t launch_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *sink, cudaStream_t stream)
+{
+    switch (mode) {
+        case 0: alu_probe_kernel<0><<<blocks, threads, 0, stream>>>(iters, sink); break;
+        case 1: alu_probe_kernel<1><<<blocks, threads, 0, stream>>>(iters, sink); break;
+        case 2: alu_probe_kernel<2><<<blocks, threads, 0, stream>>>(iters, sink); break;
+        case 3: alu_probe_kernel<3><<<blocks, threads, 0, stream>>>(iters, sink); break;
+        default: alu_probe_kernel<4><<<blocks, threads, 0, stream>>>(iters, sink); break;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace themis

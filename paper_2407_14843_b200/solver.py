@@ -1,0 +1,268 @@
+"""Python binding of ``libthemis.so``: argument marshalling only.
+
+Every function here has the name of the C entry point it forwards to
+(``include/themis.h``); tensors are passed as raw device (or host) pointers
+and the current torch CUDA stream as the stream handle.  PyTorch is used for
+device memory and streams, nothing else: every step of the solver runs in the
+library's CUDA kernels.  There is no CPU fallback: if the library has not been
+built, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libthemis.so")
+
+QUEUE_PER_REPLICA = 1
+OK, E_INVALID_ARG, E_UNSUPPORTED_SIZE, E_WORKSPACE_TOO_SMALL, E_CUDA = 0, -1, -2, -3, -4
+STATUS_OK, STATUS_INFEASIBLE, STATUS_BAD_INPUT, STATUS_TIMEOUT = 0, 1, -1, -2
+G_INF = 2 ** 31 - 1
+MAX_T = 16383
+
+EXPORTS = (
+    "themis_version", "themis_strerror", "themis_workspace_bytes", "themis_workspace_layout",
+    "themis_solve_batch", "themis_solve_vertical_batch", "themis_score_batch", "themis_minplus_batch",
+    "themis_host_workspace_bytes", "themis_solve_batch_host", "themis_alu_probe",
+    "themis_set_minplus_tile",
+)
+
+
+class ThemisError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {themis_strerror(code)} ({code})")
+
+
+class Problem(ctypes.Structure):
+    """Mirror of ``themis_problem_t``."""
+    _fields_ = [("n_instances", ctypes.c_int32), ("n_stages", ctypes.c_int32),
+                ("n_profiles", ctypes.c_int32), ("c_max", ctypes.c_int32),
+                ("n_batch", ctypes.c_int32), ("batch_sizes", ctypes.c_int32 * 16),
+                ("h_max", ctypes.c_int32), ("slo_us", ctypes.c_int32),
+                ("bucket_us", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+    @classmethod
+    def make(cls, n_instances: int, n_stages: int, n_profiles: int, c_max: int,
+             batch_sizes: Sequence[int], h_max: int, slo_us: int, bucket_us: int, flags: int = 0) -> "Problem":
+        p = cls()
+        p.n_instances, p.n_stages, p.n_profiles = n_instances, n_stages, n_profiles
+        p.c_max, p.h_max, p.slo_us, p.bucket_us, p.flags = c_max, h_max, slo_us, bucket_us, flags
+        p.n_batch = len(batch_sizes)
+        for i, b in enumerate(list(batch_sizes)[:16]):
+            p.batch_sizes[i] = int(b)
+        return p
+
+    @classmethod
+    def of_workload(cls, wl) -> "Problem":
+        return cls.make(wl.n_instances, wl.n_stages, wl.n_profiles, wl.c_max, wl.batch_sizes,
+                        wl.h_max, wl.slo_us, wl.bucket_us, wl.flags)
+
+
+class Result(ctypes.Structure):
+    """Mirror of ``themis_result_t`` (raw pointers)."""
+    _fields_ = [(k, ctypes.c_void_p) for k in ("h", "c", "b", "total_cost", "latency_buckets", "status")]
+
+
+class WorkspaceLayout(ctypes.Structure):
+    """Mirror of ``themis_workspace_layout_t``."""
+    _fields_ = [("g_offset", ctypes.c_size_t), ("garg_offset", ctypes.c_size_t),
+                ("a_offset", ctypes.c_size_t), ("f_offset", ctypes.c_size_t),
+                ("flag_offset", ctypes.c_size_t), ("total_bytes", ctypes.c_size_t),
+                ("row_pitch", ctypes.c_int32), ("T", ctypes.c_int32)]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2407_14843_b200.build` "
+            "(there is no fallback implementation)")
+    lib = ctypes.CDLL(LIB_PATH)
+    PP, vp, sz = ctypes.POINTER(Problem), ctypes.c_void_p, ctypes.c_size_t
+    lib.themis_version.restype = ctypes.c_int
+    lib.themis_version.argtypes = []
+    lib.themis_strerror.restype = ctypes.c_char_p
+    lib.themis_strerror.argtypes = [ctypes.c_int]
+    lib.themis_workspace_bytes.argtypes = [PP, ctypes.c_int, ctypes.POINTER(sz)]
+    lib.themis_host_workspace_bytes.argtypes = [PP, ctypes.c_int, ctypes.POINTER(sz)]
+    lib.themis_workspace_layout.argtypes = [PP, ctypes.c_int, ctypes.POINTER(WorkspaceLayout)]
+    lib.themis_solve_batch.argtypes = [PP, vp, vp, vp, Result, vp, sz, vp]
+    lib.themis_solve_vertical_batch.argtypes = [PP, vp, vp, vp, vp, Result, vp, sz, vp]
+    lib.themis_score_batch.argtypes = [PP, vp, vp, vp, vp, vp, sz, vp]
+    lib.themis_minplus_batch.argtypes = [PP, vp, Result, vp, sz, vp]
+    lib.themis_solve_batch_host.argtypes = [PP, vp, vp, vp, vp, Result, vp, sz, vp]
+    lib.themis_alu_probe.argtypes = [ctypes.c_int] * 4 + [vp, vp]
+    lib.themis_set_minplus_tile.argtypes = [ctypes.c_int]
+    for name in EXPORTS:
+        if name != "themis_strerror":
+            getattr(lib, name).restype = ctypes.c_int
+    return lib
+
+
+_lib = _load()
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != OK:
+        raise ThemisError(rc, where)
+
+
+def _dptr(t: Optional[torch.Tensor], dtype: torch.dtype, what: str, cuda: bool = True):
+    if t is None:
+        return None
+    if t.dtype != dtype or not t.is_contiguous() or t.is_cuda != cuda:
+        raise TypeError(f"{what}: expected a contiguous {'cuda' if cuda else 'cpu'} tensor of {dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _result(out: dict, cuda: bool = True) -> Result:
+    r = Result()
+    for k in ("h", "c", "b", "total_cost", "latency_buckets", "status"):
+        setattr(r, k, _dptr(out[k], torch.int32, f"out[{k!r}]", cuda).value)
+    return r
+
+
+def themis_version() -> int:
+    return _lib.themis_version()
+
+
+def themis_strerror(code: int) -> str:
+    return _lib.themis_strerror(code).decode()
+
+
+def themis_workspace_bytes(problem: Problem, vertical: bool) -> int:
+    n = ctypes.c_size_t()
+    _check(_lib.themis_workspace_bytes(ctypes.byref(problem), int(vertical), ctypes.byref(n)),
+           "themis_workspace_bytes")
+    return n.value
+
+
+def themis_host_workspace_bytes(problem: Problem, vertical: bool) -> int:
+    n = ctypes.c_size_t()
+    _check(_lib.themis_host_workspace_bytes(ctypes.byref(problem), int(vertical), ctypes.byref(n)),
+           "themis_host_workspace_bytes")
+    return n.value
+
+
+def themis_workspace_layout(problem: Problem, vertical: bool) -> WorkspaceLayout:
+    lay = WorkspaceLayout()
+    _check(_lib.themis_workspace_layout(ctypes.byref(problem), int(vertical), ctypes.byref(lay)),
+           "themis_workspace_layout")
+    return lay
+
+
+def themis_solve_batch(problem: Problem, lat_us, profile_id, lambda_mrps, out: dict, workspace) -> None:
+    _check(_lib.themis_solve_batch(
+        ctypes.byref(problem), _dptr(lat_us, torch.int32, "lat_us"), _dptr(profile_id, torch.int32, "profile_id"),
+        _dptr(lambda_mrps, torch.uint32, "lambda_mrps"), _result(out),
+        _dptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()), "themis_solve_batch")
+
+
+def themis_solve_vertical_batch(problem: Problem, lat_us, profile_id, lambda_mrps, replicas, out: dict,
+                                workspace) -> None:
+    _check(_lib.themis_solve_vertical_batch(
+        ctypes.byref(problem), _dptr(lat_us, torch.int32, "lat_us"), _dptr(profile_id, torch.int32, "profile_id"),
+        _dptr(lambda_mrps, torch.uint32, "lambda_mrps"), _dptr(replicas, torch.int32, "replicas"), _result(out),
+        _dptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()), "themis_solve_vertical_batch")
+
+
+def themis_score_batch(problem: Problem, lat_us, profile_id, lambda_mrps, replicas, workspace) -> None:
+    _check(_lib.themis_score_batch(
+        ctypes.byref(problem), _dptr(lat_us, torch.int32, "lat_us"), _dptr(profile_id, torch.int32, "profile_id"),
+        _dptr(lambda_mrps, torch.uint32, "lambda_mrps"), _dptr(replicas, torch.int32, "replicas"),
+        _dptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()), "themis_score_batch")
+
+
+def themis_minplus_batch(problem: Problem, replicas, out: dict, workspace) -> None:
+    _check(_lib.themis_minplus_batch(
+        ctypes.byref(problem), _dptr(replicas, torch.int32, "replicas"), _result(out),
+        _dptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()), "themis_minplus_batch")
+
+
+def themis_solve_batch_host(problem: Problem, lat_us, profile_id, lambda_mrps, replicas, out: dict,
+                            workspace) -> None:
+    """Inputs and ``out`` are CPU tensors (pinned for asynchronous copies)."""
+    _check(_lib.themis_solve_batch_host(
+        ctypes.byref(problem), _dptr(lat_us, torch.int32, "lat_us", False),
+        _dptr(profile_id, torch.int32, "profile_id", False),
+        _dptr(lambda_mrps, torch.uint32, "lambda_mrps", False), _dptr(replicas, torch.int32, "replicas", False),
+        _result(out, cuda=False), _dptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()),
+        "themis_solve_batch_host")
+
+
+def themis_alu_probe(mode: int, blocks: int, threads: int, iters: int, sink) -> None:
+    if sink.numel() < blocks * threads:
+        raise ValueError("sink too small")
+    _check(_lib.themis_alu_probe(mode, blocks, threads, iters, _dptr(sink, torch.uint32, "sink"), _stream()),
+           "themis_alu_probe")
+
+
+def themis_set_minplus_tile(cells_per_thread: int) -> None:
+    _check(_lib.themis_set_minplus_tile(cells_per_thread), "themis_set_minplus_tile")
+
+
+# --- plumbing helpers (allocation and copies only) ---------------------------
+
+def alloc_result(n_instances: int, n_stages: int, device="cuda", pin: bool = False) -> dict:
+    """Result tensors of the shapes ``themis_result_t`` expects."""
+    kw = dict(dtype=torch.int32, device=device)
+    if pin and device == "cpu":
+        kw["pin_memory"] = True
+    out = {k: torch.empty((n_instances, n_stages), **kw) for k in ("h", "c", "b")}
+    out.update({k: torch.empty(n_instances, **kw) for k in ("total_cost", "latency_buckets", "status")})
+    return out
+
+
+def alloc_workspace(problem: Problem, vertical: bool, host_variant: bool = False) -> torch.Tensor:
+    n = themis_host_workspace_bytes(problem, vertical) if host_variant else themis_workspace_bytes(problem, vertical)
+    return torch.empty(n, dtype=torch.uint8, device="cuda")
+
+
+def workload_to_device(wl, device="cuda") -> dict:
+    """Copies a ``workloads.Workload``'s arrays to the device."""
+    d = {"lat_us": torch.from_numpy(wl.lat_us).to(device),
+         "profile_id": torch.from_numpy(wl.profile_id).to(device),
+         "lambda_mrps": torch.from_numpy(wl.lambda_mrps).to(device),
+         "replicas": torch.from_numpy(wl.replicas).to(device) if wl.vertical else None}
+    return d
+
+
+def workspace_tables(problem: Problem, vertical: bool, workspace: torch.Tensor) -> dict:
+    """Views of the intermediate tables G, Garg, A, F inside a workspace."""
+    lay = themis_workspace_layout(problem, vertical)
+    N, S, P = problem.n_instances, problem.n_stages, lay.row_pitch
+    def view(off, dtype, shape):
+        n = 1
+        for s in shape:
+            n *= s
+        nbytes = n * torch.empty((), dtype=dtype).element_size()
+        return workspace[off:off + nbytes].view(dtype).view(*shape)
+    return {"G": view(lay.g_offset, torch.int32, (N, S, P)),
+            "Garg": view(lay.garg_offset, torch.uint16, (N, S, P)),
+            "A": view(lay.a_offset, torch.uint16, (N, S, P)),
+            "F": view(lay.f_offset, torch.int32, (N, P)),
+            "T": lay.T, "row_pitch": P}
+
+
+def solve(wl, dev: Optional[dict] = None, workspace: Optional[torch.Tensor] = None,
+          out: Optional[dict] = None):
+    """Solve a workload on the current device: allocates what is not given,
+    then calls ``themis_solve_batch`` / ``themis_solve_vertical_batch``."""
+    problem = Problem.of_workload(wl)
+    dev = dev if dev is not None else workload_to_device(wl)
+    workspace = workspace if workspace is not None else alloc_workspace(problem, wl.vertical)
+    out = out if out is not None else alloc_result(wl.n_instances, wl.n_stages)
+    if wl.vertical:
+        themis_solve_vertical_batch(problem, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"],
+                                    dev["replicas"], out, workspace)
+    else:
+        themis_solve_batch(problem, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"], out, workspace)
+    return out, workspace

@@ -1,0 +1,323 @@
+"""Parity of the CUDA path (called through the C ABI) with the CPU oracle,
+element by element and bit-exact, on the same seeded inputs."""
+import dataclasses
+import json
+import os
+
+import numpy as np
+import pytest
+
+from paper_2407_14843_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def S():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("the gpu tests need a CUDA device")
+    from paper_2407_14843_b200 import solver
+    return solver
+
+
+def _gpu_solve(S, wl, tables=False):
+    import torch
+    out, ws = S.solve(wl)
+    torch.cuda.synchronize()
+    res = {k: v.cpu().numpy() for k, v in out.items()}
+    if tables:
+        tb = S.workspace_tables(S.Problem.of_workload(wl), wl.vertical, ws)
+        W1 = wl.T + 1
+        res["G"] = tb["G"][:, :, :W1].cpu().numpy()
+        res["Garg"] = tb["Garg"][:, :, :W1].cpu().numpy()
+        res["A"] = tb["A"][:, :, :W1].cpu().numpy()
+        res["F"] = tb["F"][:, :W1].cpu().numpy()
+        res["G_pad"] = tb["G"][:, :, W1:].cpu().numpy()
+    return res
+
+
+RESULT_KEYS = ("status", "total_cost", "latency_buckets", "h", "c", "b")
+
+
+def _assert_results_equal(gpu, ref, idx=None):
+    for k in RESULT_KEYS:
+        a = gpu[k] if idx is None else gpu[k][idx]
+        assert np.array_equal(a, ref[k]), f"{k} differs at instances {np.argwhere(a != ref[k])[:5].tolist()}"
+
+
+def _assert_tables_equal(S, gpu, ref):
+    """G, Garg everywhere; F (last prefix) everywhere; A where F_s[t] is reachable."""
+    assert np.array_equal(gpu["G"], ref["G"])
+    assert np.array_equal(gpu["Garg"], ref["Garg"])
+    assert (gpu["G_pad"] == S.G_INF).all()
+    assert np.array_equal(gpu["F"], ref["F"][:, -1, :])
+    reach = ref["F"] != S.G_INF
+    reach[:, 0, :] = False                     # A has no row for the first stage
+    assert np.array_equal(gpu["A"][reach], ref["A"][reach])
+    unreach = ~reach
+    unreach[:, 0, :] = False
+    assert not gpu["A"][unreach].any()
+
+
+# ---------------------------------------------------------------- small, full tables
+
+@pytest.mark.parametrize("tile", [8, 16])
+def test_config1_every_table(S, oracle_mod, tile):
+    """Smallest benchmark configuration: every intermediate table and result."""
+    S.themis_set_minplus_tile(tile)
+    try:
+        wl = W.make_workload(1)
+        ref = oracle_mod.solve_batch(wl, dumps=True)
+        gpu = _gpu_solve(S, wl, tables=True)
+        _assert_tables_equal(S, gpu, ref)
+        _assert_results_equal(gpu, ref)
+    finally:
+        S.themis_set_minplus_tile(0)
+
+
+@pytest.mark.parametrize("cfg,n", [(2, 96), (3, 160), (4, 12), (5, 3)])
+@pytest.mark.parametrize("tile", [8, 16])
+def test_config_subsets_every_table(S, oracle_mod, cfg, n, tile):
+    """Subsets of the larger configurations (several tiles, ragged tail: T+1 is
+    never a multiple of the tile): every table and result."""
+    if tile == 8 and cfg == 5:
+        pytest.skip("8 cells per thread would need more than 1024 threads at T = 8192")
+    S.themis_set_minplus_tile(tile)
+    try:
+        wl = W.make_workload(cfg, n)
+        if cfg == 3:   # seconds spread over the day so that spikes are included
+            full = W.make_workload(3)
+            pick = np.linspace(0, full.n_instances - 1, n).astype(int)
+            wl = dataclasses.replace(full, n_instances=n, profile_id=full.profile_id[pick].copy(),
+                                     lambda_mrps=full.lambda_mrps[pick].copy(), replicas=full.replicas[pick].copy())
+        ref = oracle_mod.solve_batch(wl, dumps=True)
+        gpu = _gpu_solve(S, wl, tables=True)
+        _assert_tables_equal(S, gpu, ref)
+        _assert_results_equal(gpu, ref)
+    finally:
+        S.themis_set_minplus_tile(0)
+
+
+@pytest.mark.parametrize("flags", [0, W.QUEUE_PER_REPLICA])
+@pytest.mark.parametrize("vertical", [False, True])
+def test_random_tiny_against_enumeration(S, oracle_mod, flags, vertical):
+    """Random tiny instances near the feasibility edge, against the exhaustive
+    Eq. 6 enumeration (not only the DP oracle)."""
+    for seed in range(5):
+        T = 50 + 31 * seed
+        wl = W.random_tiny_workload(4000 + seed, 40, 1 + seed % 3, 6, (1, 2, 4, 8), 4, T,
+                                    flags=flags, vertical=vertical, rate_lo=20.0, rate_hi=200.0)
+        gpu = _gpu_solve(S, wl)
+        for n in range(wl.n_instances):
+            bf = oracle_mod.brute_force(wl, n)
+            assert gpu["status"][n] == bf["status"]
+            assert gpu["total_cost"][n] == bf["total_cost"] and gpu["latency_buckets"][n] == bf["latency_buckets"]
+            for k in ("h", "c", "b"):
+                assert np.array_equal(gpu[k][n], bf[k])
+
+
+def test_hand_worked_cases(S):
+    """The hand-derived fixtures, straight against the CUDA path."""
+    from tests.test_oracle_pins import _hand_workload, hand_cases
+    for case in hand_cases():
+        wl = _hand_workload(case)
+        gpu = _gpu_solve(S, wl)
+        exp = case["expect"]
+        assert int(gpu["status"][0]) == exp["status"], case["name"]
+        assert gpu["h"][0].tolist() == exp["h"] and gpu["c"][0].tolist() == exp["c"], case["name"]
+        assert gpu["b"][0].tolist() == exp["b"], case["name"]
+        assert int(gpu["total_cost"][0]) == exp["total_cost"], case["name"]
+        assert int(gpu["latency_buckets"][0]) == exp["latency_buckets"], case["name"]
+
+
+def test_paper_scale_vertical(S, oracle_mod):
+    """A pipeline of the paper's own size: 3 stages, b and c in 1..16, one
+    replica per stage, SLO 2550 ms, queue delay exactly as Eq. 4."""
+    wl = W.paper_scale_workload(40)
+    ref = oracle_mod.solve_batch(wl, dumps=True)
+    gpu = _gpu_solve(S, wl, tables=True)
+    _assert_tables_equal(S, gpu, ref)
+    _assert_results_equal(gpu, ref)
+    assert (ref["status"] == 0).any()
+
+
+# ---------------------------------------------------------------- edge cases
+
+@pytest.mark.parametrize("T", [1, 2, 31, 32, 33, 255, 256, 257, 511, 2047, 2048, 2049])
+def test_budget_lengths_around_tile_boundaries(S, oracle_mod, T):
+    wl = W.random_tiny_workload(5000 + T, 6, 3, 8, (1, 2, 4), 4, T, bucket_us=max(1, 400_000 // T) if T < 400 else 1000,
+                                rate_lo=20.0, rate_hi=120.0)
+    ref = oracle_mod.solve_batch(wl, dumps=True)
+    gpu = _gpu_solve(S, wl, tables=True)
+    _assert_tables_equal(S, gpu, ref)
+    _assert_results_equal(gpu, ref)
+
+
+def test_maximum_budget_length(S, oracle_mod):
+    """T = 16383, the largest supported budget (1024 threads x 16 cells)."""
+    wl = W.random_tiny_workload(5100, 2, 3, 16, (1, 2, 4, 8, 16), 8, 16383, bucket_us=100,
+                                rate_lo=50.0, rate_hi=400.0)
+    ref = oracle_mod.solve_batch(wl, dumps=True)
+    gpu = _gpu_solve(S, wl, tables=True)
+    _assert_tables_equal(S, gpu, ref)
+    _assert_results_equal(gpu, ref)
+    assert (ref["status"] == 0).all()
+
+
+@pytest.mark.parametrize("n_stages", [1, 2, 64])
+def test_stage_counts(S, oracle_mod, n_stages):
+    wl = W.random_tiny_workload(5200 + n_stages, 5, n_stages, 4, (1, 2, 4), 3, 40 * n_stages + 60,
+                                rate_lo=10.0, rate_hi=60.0)
+    ref = oracle_mod.solve_batch(wl, dumps=True)
+    gpu = _gpu_solve(S, wl, tables=True)
+    _assert_tables_equal(S, gpu, ref)
+    _assert_results_equal(gpu, ref)
+
+
+def test_single_instance_single_candidate(S, oracle_mod):
+    wl = W.random_tiny_workload(5300, 1, 2, 1, (1,), 1, 100, rate_lo=5.0, rate_hi=6.0)
+    ref = oracle_mod.solve_batch(wl)
+    _assert_results_equal(_gpu_solve(S, wl), ref)
+
+
+def test_all_infeasible_and_all_slack(S, oracle_mod):
+    tight = W.random_tiny_workload(5400, 16, 4, 4, (1, 2), 2, 20, rate_lo=300.0, rate_hi=900.0)
+    ref = oracle_mod.solve_batch(tight)
+    assert (ref["status"] == 1).all()
+    _assert_results_equal(_gpu_solve(S, tight), ref)
+    slack = W.random_tiny_workload(5401, 16, 4, 4, (1, 2), 2, 9000, rate_lo=5.0, rate_hi=20.0)
+    ref = oracle_mod.solve_batch(slack)
+    assert (ref["status"] == 0).all()
+    _assert_results_equal(_gpu_solve(S, slack), ref)
+
+
+def test_null_profile_id_means_profile_zero(S, oracle_mod):
+    import torch
+    wl = W.make_workload(2, 32)
+    wl0 = dataclasses.replace(wl, profile_id=np.zeros(32, np.int32))
+    ref = oracle_mod.solve_batch(wl0)
+    dev = S.workload_to_device(wl0)
+    dev["profile_id"] = None
+    out, _ = S.solve(wl0, dev=dev)
+    torch.cuda.synchronize()
+    _assert_results_equal({k: v.cpu().numpy() for k, v in out.items()}, ref)
+
+
+def test_bad_device_inputs_are_reported_per_instance(S, oracle_mod):
+    """lambda = 0, a non-positive latency and replicas < 1 do not fault: the
+    instance gets THEMIS_STATUS_BAD_INPUT, its neighbours are solved."""
+    wl = W.make_workload(2, 8)
+    lam = wl.lambda_mrps.copy()
+    lam[3] = 0
+    bad = dataclasses.replace(wl, lambda_mrps=lam)
+    gpu = _gpu_solve(S, bad)
+    ref = oracle_mod.solve_batch(wl)
+    assert gpu["status"][3] == S.STATUS_BAD_INPUT and gpu["total_cost"][3] == -1 and not gpu["h"][3].any()
+    keep = np.arange(8) != 3
+    for k in RESULT_KEYS:
+        assert np.array_equal(gpu[k][keep], ref[k][keep])
+    lat = wl.lat_us.copy()
+    lat[int(wl.profile_id[5]), 1, 0, 0] = 0
+    gpu = _gpu_solve(S, dataclasses.replace(wl, lat_us=lat))
+    assert gpu["status"][5] == S.STATUS_BAD_INPUT
+    v = W.make_workload(3, 8)
+    rep = v.replicas.copy()
+    rep[2, 4] = 0
+    gpu = _gpu_solve(S, dataclasses.replace(v, replicas=rep))
+    assert gpu["status"][2] == S.STATUS_BAD_INPUT and (gpu["status"][[0, 1, 3]] != S.STATUS_BAD_INPUT).all()
+
+
+def test_repeatable_and_tile_independent(S):
+    """Same inputs, two runs and both tile sizes: identical words everywhere
+    (every cross-thread hand-off is a barrier, so nothing may depend on timing)."""
+    wl = W.make_workload(4, 24)
+    runs = []
+    for tile in (16, 16, 8):
+        S.themis_set_minplus_tile(tile)
+        runs.append(_gpu_solve(S, wl, tables=True))
+    S.themis_set_minplus_tile(0)
+    for r in runs[1:]:
+        for k in RESULT_KEYS + ("G", "Garg", "A", "F"):
+            assert np.array_equal(runs[0][k], r[k]), k
+
+
+def test_two_step_entry_points_equal_the_solver(S, oracle_mod):
+    import torch
+    wl = W.make_workload(3, 64)
+    prob = S.Problem.of_workload(wl)
+    dev = S.workload_to_device(wl)
+    ws = S.alloc_workspace(prob, True)
+    out = S.alloc_result(wl.n_instances, wl.n_stages)
+    S.themis_score_batch(prob, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"], dev["replicas"], ws)
+    S.themis_minplus_batch(prob, dev["replicas"], out, ws)
+    torch.cuda.synchronize()
+    ref = oracle_mod.solve_batch(wl)
+    _assert_results_equal({k: v.cpu().numpy() for k, v in out.items()}, ref)
+
+
+@pytest.mark.parametrize("cfg,n", [(2, 64), (3, 64)])
+def test_host_buffer_entry_point(S, oracle_mod, cfg, n):
+    """themis_solve_batch_host: host arrays in, host arrays out."""
+    import torch
+    wl = W.make_workload(cfg, n)
+    prob = S.Problem.of_workload(wl)
+    ws = S.alloc_workspace(prob, wl.vertical, host_variant=True)
+    out = S.alloc_result(n, wl.n_stages, device="cpu", pin=True)
+    pin = lambda a: None if a is None else torch.from_numpy(a).pin_memory()
+    S.themis_solve_batch_host(prob, pin(wl.lat_us), pin(wl.profile_id), pin(wl.lambda_mrps),
+                              pin(wl.replicas) if wl.vertical else None, out, ws)
+    ref = oracle_mod.solve_batch(wl)
+    _assert_results_equal({k: v.numpy() for k, v in out.items()}, ref)
+
+
+# ---------------------------------------------------------------- full sizes
+
+def _check_properties(wl, gpu):
+    """Properties that hold at any size: totals are consistent, values in range."""
+    ok = gpu["status"] == 0
+    assert set(np.unique(gpu["status"])) <= {0, 1}
+    assert np.array_equal((gpu["h"] * gpu["c"]).sum(1)[ok], gpu["total_cost"][ok])
+    assert (gpu["latency_buckets"][ok] <= wl.T).all() and (gpu["latency_buckets"][ok] >= wl.n_stages).all()
+    assert (gpu["c"][ok] >= 1).all() and (gpu["c"][ok] <= wl.c_max).all()
+    assert np.isin(gpu["b"][ok], wl.batch_sizes).all()
+    if wl.vertical:
+        assert np.array_equal(gpu["h"][ok], wl.replicas[ok])
+    else:
+        assert (gpu["h"][ok] >= 1).all() and (gpu["h"][ok] <= wl.h_max).all()
+    assert (gpu["total_cost"][~ok] == -1).all() and not gpu["h"][~ok].any()
+    # every returned stage configuration sustains the arrival rate (Eq. 6)
+    bi = np.searchsorted(np.asarray(wl.batch_sizes), gpu["b"].clip(min=1))
+    n_i, s_i = np.meshgrid(np.arange(wl.n_instances), np.arange(wl.n_stages), indexing="ij")
+    l_us = wl.lat_us[wl.profile_id[n_i], s_i, (gpu["c"] - 1).clip(min=0), bi].astype(np.int64)
+    supply = gpu["h"].astype(np.int64) * gpu["b"].astype(np.int64) * 10 ** 9
+    demand = wl.lambda_mrps.astype(np.int64)[:, None] * l_us
+    assert (supply >= demand)[ok].all()
+
+
+def test_config2_full(S, oracle_mod):
+    wl = W.make_workload(2)
+    gpu = _gpu_solve(S, wl)
+    _check_properties(wl, gpu)
+    _assert_results_equal(gpu, oracle_mod.solve_batch(wl))
+
+
+@pytest.mark.parametrize("cfg,n_sample", [(3, 1024), (4, 40), (5, 8)])
+def test_full_size_configs_sampled(S, oracle_mod, cfg, n_sample):
+    """The full batch in the launch configuration the benchmark times; sampled
+    instances are compared with the oracle one by one, every instance is checked
+    against the size-independent properties."""
+    wl = W.make_workload(cfg)
+    gpu = _gpu_solve(S, wl)
+    _check_properties(wl, gpu)
+    pick = np.unique(np.concatenate([
+        W.rand_int(77, cfg, np.arange(n_sample, dtype=np.uint64), 0, wl.n_instances - 1),
+        [0, wl.n_instances - 1]]))
+    if cfg == 3:   # make sure spike seconds (possibly infeasible) are sampled
+        hot = np.argsort(wl.lambda_mrps)[-16:]
+        pick = np.unique(np.concatenate([pick, hot, np.flatnonzero(gpu["status"] == 1)[:64]]))
+    sub = dataclasses.replace(wl, n_instances=len(pick), profile_id=wl.profile_id[pick].copy(),
+                              lambda_mrps=wl.lambda_mrps[pick].copy(),
+                              replicas=None if wl.replicas is None else wl.replicas[pick].copy())
+    ref = oracle_mod.solve_batch(sub)
+    _assert_results_equal(gpu, ref, idx=pick)
