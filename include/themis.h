@@ -64,6 +64,7 @@ extern "C" {
 #define THEMIS_E_UNSUPPORTED_SIZE (-2)
 #define THEMIS_E_WORKSPACE_TOO_SMALL (-3)
 #define THEMIS_E_CUDA (-4)
+#define THEMIS_E_STATIC_SCRATCH_EXCEEDED (-5)
 
 /* per-instance status */
 #define THEMIS_STATUS_OK 0
@@ -173,6 +174,38 @@ int themis_solve_batch_host(const themis_problem_t *problem, const int32_t *h_la
                             const int32_t *h_profile_id, const uint32_t *h_lambda_mrps,
                             const int32_t *h_replicas, themis_result_t h_out,
                             void *d_workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Solver variant for callers that cannot allocate device memory.  (The paper has
+ * no counterpart; this is a convenience of the library.)
+ *
+ * Some callers have no way to obtain a workspace: code running under a memory
+ * pool that hands out no scratch, a plug-in that is only given its input and
+ * output buffers, a service that must not call cudaMalloc on its request path
+ * because that call synchronises the device.  For them this entry point runs
+ * the same two kernels as themis_solve_batch / themis_solve_vertical_batch
+ * (d_replicas = NULL selects the joint problem) with the intermediate tables in
+ * a fixed buffer of THEMIS_STATIC_SCRATCH_BYTES that is part of the library
+ * image: every GPU that loads the library holds that much memory until the
+ * process exits.  It calls no allocation or free routine of any kind.
+ *
+ *  - Limit: themis_workspace_bytes(problem) must not exceed
+ *    THEMIS_STATIC_SCRATCH_BYTES; larger problems are refused with
+ *    THEMIS_E_STATIC_SCRATCH_EXCEEDED before anything is launched (split the
+ *    batch, or use the workspace entry points).
+ *  - The first call on each device looks up the buffer's device address (with
+ *    that device current).  Make that first call outside any stream capture.
+ *  - All calls share the one buffer, which keeps whatever the last call left in
+ *    it.  Nothing in it has to start at zero: every word a call reads it has
+ *    written itself first, so no clearing is done.  Two calls whose kernels
+ *    overlap on the GPU (different streams, or different host threads on
+ *    different streams) race on the buffer and give wrong results: keep calls on
+ *    one stream, or order them with events.
+ */
+#define THEMIS_STATIC_SCRATCH_BYTES (32u << 20)
+int themis_solve_batch_static(const themis_problem_t *problem, const int32_t *d_lat_us,
+                              const int32_t *d_profile_id, const uint32_t *d_lambda_mrps,
+                              const int32_t *d_replicas, themis_result_t out, void *cuda_stream);
 
 /*
  * Integer-ALU throughput probe (not part of the method): every thread runs

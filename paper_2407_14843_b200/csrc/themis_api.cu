@@ -2,6 +2,8 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "themis_internal.h"
 
 namespace themis {
@@ -158,6 +160,34 @@ int host_stage_of(const themis_problem_t *pr, int vertical, size_t base, HostSta
     return THEMIS_OK;
 }
 
+// Scratch of themis_solve_batch_static: lives in the library image, one copy per
+// device that loads it.  In host code this name is only a handle for
+// cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[THEMIS_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_ptr[kMaxDevices];   // device address of g_static_scratch, per device ordinal
+
+// Device address of the static scratch on the current device; looked up on the
+// first call per device.
+int static_scratch_ptr(void **out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail_cuda(e);
+    if (dev < 0 || dev >= kMaxDevices) return THEMIS_E_UNSUPPORTED_SIZE;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return fail_cuda(e);
+        g_static_ptr[dev] = p;
+    }
+    *out = g_static_ptr[dev];
+    return THEMIS_OK;
+}
+
 }  // namespace
 }  // namespace themis
 
@@ -174,6 +204,9 @@ const char *themis_strerror(int code)
         case THEMIS_E_INVALID_ARG: return "invalid argument";
         case THEMIS_E_UNSUPPORTED_SIZE: return "problem size outside the supported limits";
         case THEMIS_E_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case THEMIS_E_STATIC_SCRATCH_EXCEEDED:
+            return "problem needs more scratch than the library's built-in 32 MiB buffer; "
+                   "split the batch or use the workspace entry points";
         case THEMIS_E_CUDA:
             snprintf(t_msg, sizeof(t_msg), "CUDA error: %s", cudaGetErrorString(t_last_cuda));
             return t_msg;
@@ -290,6 +323,22 @@ int themis_solve_batch_host(const themis_problem_t *problem, const int32_t *h_la
 #undef THEMIS_COPY
     e = cudaStreamSynchronize(st);
     return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
+}
+
+int themis_solve_batch_static(const themis_problem_t *problem, const int32_t *d_lat_us,
+                              const int32_t *d_profile_id, const uint32_t *d_lambda_mrps,
+                              const int32_t *d_replicas, themis_result_t out, void *cuda_stream)
+{
+    const int vertical = d_replicas != nullptr;
+    themis_workspace_layout_t L;
+    int rc = layout_of(problem, vertical, &L);
+    if (rc != THEMIS_OK) return rc;
+    if (L.total_bytes > (size_t)THEMIS_STATIC_SCRATCH_BYTES) return THEMIS_E_STATIC_SCRATCH_EXCEEDED;
+    void *scratch = nullptr;
+    rc = static_scratch_ptr(&scratch);
+    if (rc != THEMIS_OK) return rc;
+    return solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, d_replicas, vertical, out, scratch,
+                      (size_t)THEMIS_STATIC_SCRATCH_BYTES, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_sink, void *cuda_stream)

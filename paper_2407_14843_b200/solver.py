@@ -20,6 +20,8 @@ LIB_PATH = os.path.join(_PKG, "libthemis.so")
 
 QUEUE_PER_REPLICA = 1
 OK, E_INVALID_ARG, E_UNSUPPORTED_SIZE, E_WORKSPACE_TOO_SMALL, E_CUDA = 0, -1, -2, -3, -4
+E_STATIC_SCRATCH_EXCEEDED = -5
+STATIC_SCRATCH_BYTES = 32 << 20
 STATUS_OK, STATUS_INFEASIBLE, STATUS_BAD_INPUT, STATUS_TIMEOUT = 0, 1, -1, -2
 G_INF = 2 ** 31 - 1
 MAX_T = 16383
@@ -28,7 +30,7 @@ EXPORTS = (
     "themis_version", "themis_strerror", "themis_workspace_bytes", "themis_workspace_layout",
     "themis_solve_batch", "themis_solve_vertical_batch", "themis_score_batch", "themis_minplus_batch",
     "themis_host_workspace_bytes", "themis_solve_batch_host", "themis_alu_probe",
-    "themis_set_minplus_tile",
+    "themis_set_minplus_tile", "themis_solve_batch_static",
 )
 
 
@@ -95,6 +97,7 @@ def _load() -> ctypes.CDLL:
     lib.themis_score_batch.argtypes = [PP, vp, vp, vp, vp, vp, sz, vp]
     lib.themis_minplus_batch.argtypes = [PP, vp, Result, vp, sz, vp]
     lib.themis_solve_batch_host.argtypes = [PP, vp, vp, vp, vp, Result, vp, sz, vp]
+    lib.themis_solve_batch_static.argtypes = [PP, vp, vp, vp, vp, Result, vp]
     lib.themis_alu_probe.argtypes = [ctypes.c_int] * 4 + [vp, vp]
     lib.themis_set_minplus_tile.argtypes = [ctypes.c_int]
     for name in EXPORTS:
@@ -196,6 +199,19 @@ def themis_solve_batch_host(problem: Problem, lat_us, profile_id, lambda_mrps, r
         _dptr(lambda_mrps, torch.uint32, "lambda_mrps", False), _dptr(replicas, torch.int32, "replicas", False),
         _result(out, cuda=False), _dptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()),
         "themis_solve_batch_host")
+
+
+def themis_solve_batch_static(problem: Problem, lat_us, profile_id, lambda_mrps, replicas, out: dict) -> None:
+    """Solver variant that needs no workspace from the caller: the tables live
+    in a 32 MiB buffer inside the library (for callers that cannot allocate
+    device memory).  Problems whose ``themis_workspace_bytes`` exceeds
+    ``STATIC_SCRATCH_BYTES`` raise ``ThemisError`` with
+    ``E_STATIC_SCRATCH_EXCEEDED``.  All calls share that buffer, so keep them
+    on one stream; make the first call on a device outside stream capture."""
+    _check(_lib.themis_solve_batch_static(
+        ctypes.byref(problem), _dptr(lat_us, torch.int32, "lat_us"), _dptr(profile_id, torch.int32, "profile_id"),
+        _dptr(lambda_mrps, torch.uint32, "lambda_mrps"), _dptr(replicas, torch.int32, "replicas"), _result(out),
+        _stream()), "themis_solve_batch_static")
 
 
 def themis_alu_probe(mode: int, blocks: int, threads: int, iters: int, sink) -> None:
