@@ -103,8 +103,9 @@ typedef struct {
  * start; rows are row_pitch entries long, entries beyond T are padding).
  *   G    int32  [N][S][row_pitch]  per-bucket minimum cost, THEMIS_G_INF if empty
  *   Garg uint16 [N][S][row_pitch]  lowest candidate index attaining G (0 if empty)
- *   A    uint16 [N][S][row_pitch]  A[s][t] = lowest l attaining F_s[t] (row 0 unused,
- *                                  0 where F_s[t] is unreachable)
+ *   A    uint16 [N][S][row_pitch]  mode 1: A[s][t] = lowest l attaining F_s[t] (row 0
+ *                                  unused, 0 where F_s[t] is unreachable); mode 0: the
+ *                                  prefix tables F_s[t] (see themis_set_minplus_mode)
  *   F    int32  [N][row_pitch]     last prefix table F_{S-1}, THEMIS_G_INF if unreachable
  * Candidate index: idx = ((h-1)*c_max + (c-1))*n_batch + bi (joint),
  *                  idx = (c-1)*n_batch + bi (vertical). */
@@ -219,6 +220,16 @@ int themis_solve_batch_static(const themis_problem_t *problem, const int32_t *d_
  */
 int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_sink,
                      void *cuda_stream);
+
+/* Which min-plus kernel themis_minplus_batch and the solvers run.  Results do not
+ * depend on it; the layout of the A rows of the workspace does.
+ *   0 (default): packed 16-bit kernel (two budget cells per register).  The A
+ *      rows then hold the prefix tables themselves, uint16 F_s[t] with
+ *      0x7FFF = unreachable or >= 32767, and the backtrack recovers the argmin
+ *      along the optimal path only.  Instances whose optimum does not fit 16
+ *      bits are redone by the 32-bit kernel in a second launch.
+ *   1: 32-bit kernel only; the A rows hold the argmin tables described above. */
+int themis_set_minplus_mode(int mode);
 
 /* Tuning knob of the min-plus kernel: consecutive budget cells per thread
  * (8 or 16); 0 restores the built-in choice.  Results do not depend on it. */

@@ -12,6 +12,7 @@ namespace {
 thread_local cudaError_t t_last_cuda = cudaSuccess;
 thread_local char t_msg[256];
 int g_tile = 0;   // min-plus cells per thread; 0 = built-in choice
+int g_mode = 0;   // 0: packed 16-bit min-plus kernel with 32-bit second pass; 1: 32-bit kernel only
 
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
@@ -121,7 +122,20 @@ int minplus_impl(const themis_problem_t *pr, const int32_t *rep, int vertical, t
     if (rc != THEMIS_OK) return rc;
     if (!result_ok(out) || (vertical && !rep)) return THEMIS_E_INVALID_ARG;
     P.replicas = rep; P.out = out;
-    cudaError_t e = launch_minplus(P, g_tile, st);
+    cudaError_t e;
+    if (g_mode == 1) {
+        e = launch_minplus(P, g_tile, st);
+    } else {
+        e = launch_minplus16(P, g_tile, st);
+        // A total can only reach the 16-bit saturation value if the static bound allows it
+        // (vertical: the bound depends on replicas[], which lives on the device).
+        const bool may_saturate =
+            vertical || (int64_t)pr->n_stages * pr->h_max * pr->c_max >= (int64_t)kInf16;
+        if (e == cudaSuccess && may_saturate) {
+            P.only_flagged = 1;
+            e = launch_minplus(P, g_tile, st);
+        }
+    }
     return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
 }
 
@@ -347,6 +361,13 @@ int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_s
         return THEMIS_E_INVALID_ARG;
     cudaError_t e = launch_alu_probe(mode, blocks, threads, iters, d_sink, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
+}
+
+int themis_set_minplus_mode(int mode)
+{
+    if (mode != 0 && mode != 1) return THEMIS_E_INVALID_ARG;
+    g_mode = mode;
+    return THEMIS_OK;
 }
 
 int themis_set_minplus_tile(int cells_per_thread)

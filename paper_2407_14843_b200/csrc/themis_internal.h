@@ -16,6 +16,16 @@ constexpr uint32_t kIdxMask = (1u << kIdxBits) - 1u;
 constexpr uint32_t kInfCost = (1u << 17) - 1u;
 constexpr uint32_t kInfKey = kInfCost << kIdxBits;
 
+// inst_flag values: 0 clean, 1 bad input seen while scoring, 2 set by the packed
+// 16-bit min-plus kernel when a total reached its saturation value and the
+// instance has to be redone by the 32-bit kernel.
+constexpr int32_t kFlagBadInput = 1;
+constexpr int32_t kFlagNeedsWide = 2;
+
+// Packed 16-bit path: costs are exact below kInf16 and saturate there; two of
+// them add without carrying into the neighbouring half-word.
+constexpr uint32_t kInf16 = 0x7FFFu;
+
 // Rows of the workspace tables are padded to a multiple of this many entries,
 // so every row starts 64-byte aligned (uint16) / 128-byte aligned (int32) and
 // bulk copies of whole rows meet the 16-byte rule.
@@ -27,6 +37,7 @@ struct Params {
     int32_t pitch;      // row pitch of G / Garg / A / F in entries
     int32_t vertical;   // 1: h fixed per stage from replicas[]
     int32_t K;          // candidates per stage
+    int32_t only_flagged;  // wide min-plus kernel: solve only instances flagged kFlagNeedsWide
     const int32_t *lat_us;
     const int32_t *profile_id;
     const uint32_t *lambda_mrps;
@@ -41,6 +52,7 @@ struct Params {
 
 cudaError_t launch_score(const Params &p, cudaStream_t stream);
 cudaError_t launch_minplus(const Params &p, int tile, cudaStream_t stream);
+cudaError_t launch_minplus16(const Params &p, int tile, cudaStream_t stream);
 cudaError_t launch_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *sink,
                              cudaStream_t stream);
 

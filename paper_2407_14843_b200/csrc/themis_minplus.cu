@@ -23,57 +23,11 @@
 // half of a double buffer, completion signalled on an mbarrier, while stage s
 // computes.  Every wait on an mbarrier is bounded; on expiry the block reports
 // THEMIS_STATUS_TIMEOUT for its instance and leaves.
+#include "themis_async.cuh"
 #include "themis_internal.h"
 
 namespace themis {
 namespace {
-
-constexpr uint32_t kWaitLimit = 1u << 20;   // try_wait attempts before giving up
-
-__device__ __forceinline__ uint32_t smem_addr(const void *p)
-{
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
-}
-
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
-                 : "memory");
-}
-
-// One-dimensional bulk asynchronous copy global -> this block's shared memory.
-// Both addresses 16-byte aligned, bytes a multiple of 16.
-__device__ __forceinline__ void bulk_load(void *dst_smem, const void *src_gmem, uint32_t bytes, uint64_t *bar)
-{
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-            smem_addr(dst_smem)),
-        "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar))
-        : "memory");
-}
-
-// Bounded wait for the given phase parity; false if the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
-{
-    const uint32_t a = smem_addr(bar);
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done)
-            : "r"(a), "r"(parity)
-            : "memory");
-        if (done) return true;
-    }
-    return false;
-}
 
 template <int R>
 struct Tile {
@@ -140,7 +94,9 @@ minplus_kernel(const Params p)
         p.out.latency_buckets[n] = -1;
         p.out.status[n] = status;
     };
-    if (p.inst_flag[n] != 0) {                          // bad input seen while scoring
+    if (p.only_flagged) {                               // second pass: only what the packed kernel left over
+        if (p.inst_flag[n] != kFlagNeedsWide) return;
+    } else if (p.inst_flag[n] != 0) {                   // bad input seen while scoring
         if (tid == 0) write_unsolved(THEMIS_STATUS_BAD_INPUT);
         return;
     }

@@ -25,12 +25,13 @@ STATIC_SCRATCH_BYTES = 32 << 20
 STATUS_OK, STATUS_INFEASIBLE, STATUS_BAD_INPUT, STATUS_TIMEOUT = 0, 1, -1, -2
 G_INF = 2 ** 31 - 1
 MAX_T = 16383
+INF16 = 0x7FFF
 
 EXPORTS = (
     "themis_version", "themis_strerror", "themis_workspace_bytes", "themis_workspace_layout",
     "themis_solve_batch", "themis_solve_vertical_batch", "themis_score_batch", "themis_minplus_batch",
     "themis_host_workspace_bytes", "themis_solve_batch_host", "themis_alu_probe",
-    "themis_set_minplus_tile", "themis_solve_batch_static",
+    "themis_set_minplus_tile", "themis_solve_batch_static", "themis_set_minplus_mode",
 )
 
 
@@ -100,6 +101,7 @@ def _load() -> ctypes.CDLL:
     lib.themis_solve_batch_static.argtypes = [PP, vp, vp, vp, vp, Result, vp]
     lib.themis_alu_probe.argtypes = [ctypes.c_int] * 4 + [vp, vp]
     lib.themis_set_minplus_tile.argtypes = [ctypes.c_int]
+    lib.themis_set_minplus_mode.argtypes = [ctypes.c_int]
     for name in EXPORTS:
         if name != "themis_strerror":
             getattr(lib, name).restype = ctypes.c_int
@@ -219,6 +221,10 @@ def themis_alu_probe(mode: int, blocks: int, threads: int, iters: int, sink) -> 
         raise ValueError("sink too small")
     _check(_lib.themis_alu_probe(mode, blocks, threads, iters, _dptr(sink, torch.uint32, "sink"), _stream()),
            "themis_alu_probe")
+
+
+def themis_set_minplus_mode(mode: int) -> None:
+    _check(_lib.themis_set_minplus_mode(mode), "themis_set_minplus_mode")
 
 
 def themis_set_minplus_tile(cells_per_thread: int) -> None:

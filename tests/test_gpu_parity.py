@@ -46,11 +46,31 @@ def _assert_results_equal(gpu, ref, idx=None):
         assert np.array_equal(a, ref[k]), f"{k} differs at instances {np.argwhere(a != ref[k])[:5].tolist()}"
 
 
+MODE = {"mode": 0}   # min-plus kernel under test: 0 packed 16-bit (default), 1 32-bit
+
+
+@pytest.fixture(params=[0, 1], ids=["packed16", "wide32"])
+def mode(request, S):
+    S.themis_set_minplus_mode(request.param)
+    MODE["mode"] = request.param
+    yield request.param
+    S.themis_set_minplus_mode(0)
+    MODE["mode"] = 0
+
+
 def _assert_tables_equal(S, gpu, ref):
-    """G, Garg everywhere; F (last prefix) everywhere; A where F_s[t] is reachable."""
+    """G, Garg everywhere; F (last prefix) where the instance is solved; then
+    32-bit kernel: A where F_s[t] is reachable (0 elsewhere);
+    packed kernel: every prefix table F_s[t], saturated at 0x7FFF."""
     assert np.array_equal(gpu["G"], ref["G"])
     assert np.array_equal(gpu["Garg"], ref["Garg"])
     assert (gpu["G_pad"] == S.G_INF).all()
+    if MODE["mode"] == 0:
+        solved = ref["status"] == 0
+        assert np.array_equal(gpu["F"][solved], ref["F"][solved, -1, :])
+        assert (ref["F"][ref["F"] != S.G_INF] < S.INF16).all(), "use the saturation test for such inputs"
+        assert np.array_equal(gpu["A"], np.minimum(ref["F"], S.INF16).astype(np.uint16))
+        return
     assert np.array_equal(gpu["F"], ref["F"][:, -1, :])
     reach = ref["F"] != S.G_INF
     reach[:, 0, :] = False                     # A has no row for the first stage
@@ -63,7 +83,7 @@ def _assert_tables_equal(S, gpu, ref):
 # ---------------------------------------------------------------- small, full tables
 
 @pytest.mark.parametrize("tile", [8, 16])
-def test_config1_every_table(S, oracle_mod, tile):
+def test_config1_every_table(S, oracle_mod, tile, mode):
     """Smallest benchmark configuration: every intermediate table and result."""
     S.themis_set_minplus_tile(tile)
     try:
@@ -78,7 +98,7 @@ def test_config1_every_table(S, oracle_mod, tile):
 
 @pytest.mark.parametrize("cfg,n", [(2, 96), (3, 160), (4, 12), (5, 3)])
 @pytest.mark.parametrize("tile", [8, 16])
-def test_config_subsets_every_table(S, oracle_mod, cfg, n, tile):
+def test_config_subsets_every_table(S, oracle_mod, cfg, n, tile, mode):
     """Subsets of the larger configurations (several tiles, ragged tail: T+1 is
     never a multiple of the tile): every table and result."""
     if tile == 8 and cfg == 5:
@@ -101,7 +121,7 @@ def test_config_subsets_every_table(S, oracle_mod, cfg, n, tile):
 
 @pytest.mark.parametrize("flags", [0, W.QUEUE_PER_REPLICA])
 @pytest.mark.parametrize("vertical", [False, True])
-def test_random_tiny_against_enumeration(S, oracle_mod, flags, vertical):
+def test_random_tiny_against_enumeration(S, oracle_mod, flags, vertical, mode):
     """Random tiny instances near the feasibility edge, against the exhaustive
     Eq. 6 enumeration (not only the DP oracle)."""
     for seed in range(5):
@@ -117,7 +137,7 @@ def test_random_tiny_against_enumeration(S, oracle_mod, flags, vertical):
                 assert np.array_equal(gpu[k][n], bf[k])
 
 
-def test_hand_worked_cases(S):
+def test_hand_worked_cases(S, mode):
     """The hand-derived fixtures, straight against the CUDA path."""
     from tests.test_oracle_pins import _hand_workload, hand_cases
     for case in hand_cases():
@@ -131,7 +151,7 @@ def test_hand_worked_cases(S):
         assert int(gpu["latency_buckets"][0]) == exp["latency_buckets"], case["name"]
 
 
-def test_paper_scale_vertical(S, oracle_mod):
+def test_paper_scale_vertical(S, oracle_mod, mode):
     """A pipeline of the paper's own size: 3 stages, b and c in 1..16, one
     replica per stage, SLO 2550 ms, queue delay exactly as Eq. 4."""
     wl = W.paper_scale_workload(40)
@@ -145,7 +165,7 @@ def test_paper_scale_vertical(S, oracle_mod):
 # ---------------------------------------------------------------- edge cases
 
 @pytest.mark.parametrize("T", [1, 2, 31, 32, 33, 255, 256, 257, 511, 2047, 2048, 2049])
-def test_budget_lengths_around_tile_boundaries(S, oracle_mod, T):
+def test_budget_lengths_around_tile_boundaries(S, oracle_mod, T, mode):
     wl = W.random_tiny_workload(5000 + T, 6, 3, 8, (1, 2, 4), 4, T, bucket_us=max(1, 400_000 // T) if T < 400 else 1000,
                                 rate_lo=20.0, rate_hi=120.0)
     ref = oracle_mod.solve_batch(wl, dumps=True)
@@ -154,7 +174,7 @@ def test_budget_lengths_around_tile_boundaries(S, oracle_mod, T):
     _assert_results_equal(gpu, ref)
 
 
-def test_maximum_budget_length(S, oracle_mod):
+def test_maximum_budget_length(S, oracle_mod, mode):
     """T = 16383, the largest supported budget (1024 threads x 16 cells)."""
     wl = W.random_tiny_workload(5100, 2, 3, 16, (1, 2, 4, 8, 16), 8, 16383, bucket_us=100,
                                 rate_lo=50.0, rate_hi=400.0)
@@ -166,7 +186,7 @@ def test_maximum_budget_length(S, oracle_mod):
 
 
 @pytest.mark.parametrize("n_stages", [1, 2, 64])
-def test_stage_counts(S, oracle_mod, n_stages):
+def test_stage_counts(S, oracle_mod, n_stages, mode):
     wl = W.random_tiny_workload(5200 + n_stages, 5, n_stages, 4, (1, 2, 4), 3, 40 * n_stages + 60,
                                 rate_lo=10.0, rate_hi=60.0)
     ref = oracle_mod.solve_batch(wl, dumps=True)
@@ -181,7 +201,7 @@ def test_single_instance_single_candidate(S, oracle_mod):
     _assert_results_equal(_gpu_solve(S, wl), ref)
 
 
-def test_all_infeasible_and_all_slack(S, oracle_mod):
+def test_all_infeasible_and_all_slack(S, oracle_mod, mode):
     tight = W.random_tiny_workload(5400, 16, 4, 4, (1, 2), 2, 20, rate_lo=300.0, rate_hi=900.0)
     ref = oracle_mod.solve_batch(tight)
     assert (ref["status"] == 1).all()
@@ -204,7 +224,7 @@ def test_null_profile_id_means_profile_zero(S, oracle_mod):
     _assert_results_equal({k: v.cpu().numpy() for k, v in out.items()}, ref)
 
 
-def test_bad_device_inputs_are_reported_per_instance(S, oracle_mod):
+def test_bad_device_inputs_are_reported_per_instance(S, oracle_mod, mode):
     """lambda = 0, a non-positive latency and replicas < 1 do not fault: the
     instance gets THEMIS_STATUS_BAD_INPUT, its neighbours are solved."""
     wl = W.make_workload(2, 8)
@@ -228,7 +248,7 @@ def test_bad_device_inputs_are_reported_per_instance(S, oracle_mod):
     assert gpu["status"][2] == S.STATUS_BAD_INPUT and (gpu["status"][[0, 1, 3]] != S.STATUS_BAD_INPUT).all()
 
 
-def test_repeatable_and_tile_independent(S):
+def test_repeatable_and_tile_independent(S, mode):
     """Same inputs, two runs and both tile sizes: identical words everywhere
     (every cross-thread hand-off is a barrier, so nothing may depend on timing)."""
     wl = W.make_workload(4, 24)
@@ -240,6 +260,36 @@ def test_repeatable_and_tile_independent(S):
     for r in runs[1:]:
         for k in RESULT_KEYS + ("G", "Garg", "A", "F"):
             assert np.array_equal(runs[0][k], r[k]), k
+
+
+def test_both_kernels_agree(S):
+    """Packed 16-bit and 32-bit min-plus kernels: the same results, word for word."""
+    wl = W.make_workload(3, 300)
+    S.themis_set_minplus_mode(1)
+    wide = _gpu_solve(S, wl)
+    S.themis_set_minplus_mode(0)
+    packed = _gpu_solve(S, wl)
+    for k in RESULT_KEYS:
+        assert np.array_equal(wide[k], packed[k]), k
+
+
+def test_totals_beyond_16_bits_fall_back_to_the_wide_kernel(S, oracle_mod):
+    """Vertical problem with thousands of replicas per stage: optimal totals of
+    40000 and more do not fit the packed kernel's 15-bit costs; those instances
+    are redone by the 32-bit kernel.  Mixed with cheap instances and with
+    infeasible ones in the same batch."""
+    base = W.random_tiny_workload(5600, 24, 6, 2, (1, 2, 4), 4, 420, vertical=True, rate_lo=10.0, rate_hi=60.0)
+    rep = base.replicas.copy()
+    rep[0::3] = 6000                        # 6 stages x 6000 x c: totals of 36000 .. 72000
+    rep[1::3] = np.maximum(rep[1::3], 1)
+    lam = base.lambda_mrps.copy()
+    lam[2::3] = 4_000_000                   # 4000 rps on a handful of replicas: infeasible
+    wl = dataclasses.replace(base, replicas=rep, lambda_mrps=lam)
+    ref = oracle_mod.solve_batch(wl)
+    assert (ref["total_cost"] >= S.INF16).any() and (ref["status"] == 1).any()
+    assert ((ref["total_cost"] > 0) & (ref["total_cost"] < S.INF16)).any()
+    S.themis_set_minplus_mode(0)
+    _assert_results_equal(_gpu_solve(S, wl), ref)
 
 
 def test_two_step_entry_points_equal_the_solver(S, oracle_mod):
@@ -295,7 +345,7 @@ def _check_properties(wl, gpu):
     assert (supply >= demand)[ok].all()
 
 
-def test_config2_full(S, oracle_mod):
+def test_config2_full(S, oracle_mod, mode):
     wl = W.make_workload(2)
     gpu = _gpu_solve(S, wl)
     _check_properties(wl, gpu)
@@ -303,7 +353,7 @@ def test_config2_full(S, oracle_mod):
 
 
 @pytest.mark.parametrize("cfg,n_sample", [(3, 1024), (4, 40), (5, 8)])
-def test_full_size_configs_sampled(S, oracle_mod, cfg, n_sample):
+def test_full_size_configs_sampled(S, oracle_mod, cfg, n_sample, mode):
     """The full batch in the launch configuration the benchmark times; sampled
     instances are compared with the oracle one by one, every instance is checked
     against the size-independent properties."""
