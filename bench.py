@@ -30,11 +30,13 @@ if ROOT not in sys.path:
 METRIC = "dp_instances_per_s"
 UNIT = "instances/s"
 
-# INT32 ALU peak of one B200 for the recurrence's operation pair: 148 SMs x 64
-# integer lanes per SM per clock x 1.965 GHz boost clock, one fused add-min
-# (two integer operations) per lane per clock.
+# Integer ALU peak of one B200 for the recurrence's operation pair: 148 SMs x 64
+# integer lanes per SM per clock x 1.965 GHz boost clock, one fused add-min (two
+# integer operations) per lane per clock on 32-bit words; the packed 16-bit form
+# of the same instruction does two half-word cells per lane per clock.
 N_SMS, INT_LANES_PER_SM, SM_GHZ = 148, 64, 1.965
-ALU_PEAK_TOPS = N_SMS * INT_LANES_PER_SM * 2 * SM_GHZ / 1e3
+ALU_PEAK_TOPS_INT32 = N_SMS * INT_LANES_PER_SM * 2 * SM_GHZ / 1e3
+ALU_PEAK_TOPS_INT16X2 = 2 * ALU_PEAK_TOPS_INT32
 HBM_FALLBACK_GBS = 6650.0
 
 # DRAM bytes (read + write) of one min-plus launch from the ncu capture summarised
@@ -42,8 +44,8 @@ HBM_FALLBACK_GBS = 6650.0
 # to the instance count (one block per instance, no reuse across blocks).  The
 # figure is only reported while the kernel source still has the recorded hash.
 NCU_TRAFFIC = {
-    "config": 4, "bytes_per_instance": (267.730176e6 + 110.708992e6) / 2048,
-    "source": "paper_2407_14843_b200/csrc/themis_minplus.cu", "sha256_16": "454ebb1401351c38",
+    "config": 4, "bytes_per_instance": (285.001728e6 + 131.188736e6) / 2048,
+    "source": "paper_2407_14843_b200/csrc/themis_minplus16.cu", "sha256_16": "18c2d4846bde6818",
 }
 
 
@@ -57,6 +59,8 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--minplus-mode", type=int, default=0, choices=[0, 1],
+                    help="0: packed 16-bit min-plus kernel (default); 1: 32-bit kernel")
     return ap.parse_args()
 
 
@@ -205,17 +209,19 @@ class ClockSampler:
                 "samples": len(sm), "power_w_max": max(power)}
 
 
-def probe_alu_peak(solver, torch):
-    """Fused add-min updates per second sustained by themis_alu_probe (TOP/s, two ops per update)."""
+def probe_alu_peak(solver, torch, mode):
+    """Add-min throughput sustained by themis_alu_probe in TOP/s (two operations
+    per cell update): mode 1 = fused 32-bit add-min, mode 3 = packed 2 x 16-bit."""
     blocks, threads, iters = N_SMS * 8, 256, 4000
+    cells_per_update = 2 if mode == 3 else 1
     sink = torch.empty(blocks * threads, dtype=torch.uint32, device="cuda")
-    solver.themis_alu_probe(1, blocks, threads, 50, sink)
+    solver.themis_alu_probe(mode, blocks, threads, 50, sink)
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record()
-    solver.themis_alu_probe(1, blocks, threads, iters, sink)
+    solver.themis_alu_probe(mode, blocks, threads, iters, sink)
     b.record()
     torch.cuda.synchronize()
-    return 2.0 * blocks * threads * iters * 64 / (a.elapsed_time(b) * 1e-3) / 1e12
+    return 2.0 * cells_per_update * blocks * threads * iters * 64 / (a.elapsed_time(b) * 1e-3) / 1e12
 
 
 # --------------------------------------------------------------------------- the CUDA arm
@@ -249,6 +255,8 @@ def run_ours(args):
         dist.barrier()
     from paper_2407_14843_b200 import solver
 
+    solver.themis_set_minplus_mode(args.minplus_mode)
+    packed = args.minplus_mode == 0
     prob = solver.Problem.of_workload(wl)
     dev = solver.workload_to_device(wl)
     ws = solver.alloc_workspace(prob, wl.vertical, host_variant=True)
@@ -272,7 +280,8 @@ def run_ours(args):
 
     for _ in range(max(args.warmup, 1)):
         step()
-    alu_probe_tops = probe_alu_peak(solver, torch) if rank == 0 else None
+    alu_probe_tops = {"int32": probe_alu_peak(solver, torch, 1), "int16x2": probe_alu_peak(solver, torch, 3)} \
+        if rank == 0 else None
     barrier()
 
     uuid = str(getattr(torch.cuda.get_device_properties(local_rank), "uuid", ""))
@@ -330,8 +339,12 @@ def run_ours(args):
         return
 
     N_total = wl.n_instances * world
+    # score + min-plus, plus the 32-bit second pass where a total may exceed 15 bits
+    second_pass = packed and (wl.vertical or wl.n_stages * wl.h_max * wl.c_max >= 0x7FFF)
+    launches_per_step = 3 if second_pass else 2
     cells_per_launch = wl.n_instances * wl.minplus_cells
     achieved_tops = 2.0 * cells_per_launch / (minplus_ms * 1e-3) / 1e12
+    alu_peak = ALU_PEAK_TOPS_INT16X2 if packed else ALU_PEAK_TOPS_INT32
     lay = solver.themis_workspace_layout(prob, wl.vertical)
     score_bytes = 6.0 * lay.row_pitch * wl.n_instances * wl.n_stages
     hbm_peak, hbm_kind = measured_hbm_peak()
@@ -343,15 +356,18 @@ def run_ours(args):
         "data": "synthetic", "config": workload_config(wl, args, world),
         "cell_updates_per_s": world * cells_per_launch * args.steps / (total_ms * 1e-3),
         "minplus_cell_updates_per_s_kernel": cells_per_launch / (minplus_ms * 1e-3),
-        "kernels_ms": {"score_kernel": score_ms, "minplus_kernel": minplus_ms},
+        "kernels_ms": {"score_kernel": score_ms, ("minplus16_kernel" if packed else "minplus_kernel"): minplus_ms},
         "infeasible_instances": n_infeasible, "device_error_instances": n_error,
         "input_checksums": wl.checksums(),
         "roofline": {
-            "kernel": "minplus_kernel", "bound": "alu", "achieved": achieved_tops, "peak": ALU_PEAK_TOPS,
-            "unit": "TOP/s (int32 add+min, 2 per cell update)", "frac": achieved_tops / ALU_PEAK_TOPS,
-            "traffic": ncu_traffic_bytes(args.config, wl.n_instances), "peak_kind": "derived: 148 SMs x 64 int lanes x 2 ops x 1.965 GHz",
-            "peak_probe": alu_probe_tops, "algorithmic_cells_per_launch": cells_per_launch,
-            "avg_launch_ms": minplus_ms,
+            "kernel": "minplus16_kernel" if packed else "minplus_kernel", "bound": "alu",
+            "achieved": achieved_tops, "peak": alu_peak,
+            "unit": "TOP/s (integer add+min, 2 per cell update)", "frac": achieved_tops / alu_peak,
+            "traffic": ncu_traffic_bytes(args.config, wl.n_instances) if packed else None,
+            "peak_kind": ("derived: 148 SMs x 64 int lanes x 2 ops x 1.965 GHz"
+                          + (" x 2 half-word cells per lane (packed 16-bit add-min)" if packed else "")),
+            "peak_probe": alu_probe_tops, "frac_of_int32_peak": achieved_tops / ALU_PEAK_TOPS_INT32,
+            "algorithmic_cells_per_launch": cells_per_launch, "avg_launch_ms": minplus_ms,
         },
         "roofline_score_kernel": {
             "kernel": "score_kernel", "bound": "hbm", "achieved": score_gbs, "peak": hbm_peak, "unit": "GB/s",
@@ -360,7 +376,7 @@ def run_ours(args):
         },
         "e2e": {"value": N_total * args.e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": args.e2e_steps, "matches_device_path": same},
-        "gpu_launches": 2 * args.steps,
+        "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks,
     }
     if cpu is not None:
