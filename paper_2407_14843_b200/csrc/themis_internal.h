@@ -38,6 +38,7 @@ struct Params {
     int32_t vertical;   // 1: h fixed per stage from replicas[]
     int32_t K;          // candidates per stage
     int32_t only_flagged;  // wide min-plus kernel: solve only instances flagged kFlagNeedsWide
+    uint8_t warp_group[32];  // min-plus kernels: tile group (32 tiles) owned by each warp
     const int32_t *lat_us;
     const int32_t *profile_id;
     const uint32_t *lambda_mrps;
@@ -49,6 +50,24 @@ struct Params {
     int32_t *inst_flag;  // [N] nonzero = bad input seen by the scoring kernel
     themis_result_t out;
 };
+
+// Deals the tile groups of a min-plus block (group g costs g + 1 units: its columns
+// are that much longer) to the block's warps so that the SM's four warp schedulers,
+// which take a block's warps round-robin, end up with equal shares: longest group
+// first, always to the least loaded scheduler that still has a free warp.
+inline void assign_warp_groups(int n_warps, uint8_t *warp_group)
+{
+    int load[4] = {0, 0, 0, 0}, used[4] = {0, 0, 0, 0}, cap[4];
+    for (int c = 0; c < 4; ++c) cap[c] = (n_warps - c + 3) / 4;
+    for (int g = n_warps - 1; g >= 0; --g) {
+        int best = -1;
+        for (int c = 0; c < 4; ++c)
+            if (used[c] < cap[c] && (best < 0 || load[c] < load[best])) best = c;
+        warp_group[4 * used[best] + best] = (uint8_t)g;
+        load[best] += g + 1;
+        ++used[best];
+    }
+}
 
 cudaError_t launch_score(const Params &p, cudaStream_t stream);
 cudaError_t launch_minplus(const Params &p, int tile, cudaStream_t stream);

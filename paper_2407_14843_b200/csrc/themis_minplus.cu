@@ -81,8 +81,9 @@ minplus_kernel(const Params p)
     uint64_t *mbar = reinterpret_cast<uint64_t *>(Gbuf1 + Tp);
     uint32_t *red = reinterpret_cast<uint32_t *>(mbar + 2);   // 32 words for the block reduction
 
-    const int t0 = tid * R;
-    uint32_t *my_chunk = Fs + (tid + 1) * CS;
+    const int tile = ((int)p.warp_group[tid >> 5] << 5) | (tid & 31);                   // groups dealt by assign_warp_groups
+    const int t0 = tile * R;
+    uint32_t *my_chunk = Fs + (tile + 1) * CS;
     const uint32_t row_bytes = (uint32_t)pitch * 4u;
     const int32_t *G_inst = p.G + (size_t)n * S * pitch;
 
@@ -165,8 +166,8 @@ minplus_kernel(const Params p)
         for (int r = 0; r < R; ++r) { acc[r] = 0xFFFFFFFFu; wa[r] = my_chunk[r]; }
         // All lanes of a warp walk the same l so that G is a broadcast; lanes
         // that run past their own range read the "unreachable" chunk in front.
-        const int q_end = tid | 31;
-        int f_off = tid * CS;                            // word offset of chunk tid-1
+        const int q_end = tile | 31;
+        int f_off = tile * CS;                           // word offset of chunk tile-1
         const uint32_t *g = Gk;
         for (int q = 0; q <= q_end; q += 2) {
             chunk_step<R>(wa, wb, acc, Fs + max(f_off, 0), g);
@@ -246,8 +247,10 @@ minplus_kernel(const Params p)
 }
 
 template <int R, int MAXT>
-cudaError_t launch_variant(const Params &p, int threads, size_t smem, cudaStream_t stream)
+cudaError_t launch_variant(const Params &p_in, int threads, size_t smem, cudaStream_t stream)
 {
+    Params p = p_in;
+    assign_warp_groups(threads / 32, p.warp_group);
     cudaError_t e = cudaFuncSetAttribute(minplus_kernel<R, MAXT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)smem);
     if (e != cudaSuccess) return e;

@@ -93,6 +93,7 @@ minplus16_kernel(const Params p)
 {
     extern __shared__ __align__(128) uint32_t smem[];
     constexpr int H = Tile16<R>::H, CS = Tile16<R>::CS;
+    constexpr int U = R == 8 ? 4 : 2;                     // chunk steps per loop iteration
     const int n = blockIdx.x;
     const int tid = threadIdx.x;
     const int NT = blockDim.x;
@@ -106,9 +107,13 @@ minplus16_kernel(const Params p)
     uint64_t *mbar = reinterpret_cast<uint64_t *>(Gbuf1 + Tp);
     uint32_t *red = reinterpret_cast<uint32_t *>(mbar + 2);   // 32 words
     uint32_t *xchg = red + 32;                                // 32 words: last accp word of each warp
+    uint32_t *stage_lmin = xchg + 32;                         // 64 words: first reachable l of every G_s
 
-    const int t0 = tid * R;
-    uint32_t *my_chunk = Fw + (kPadChunks + tid) * CS;
+    // Which tile (R consecutive cells) this thread owns: lanes keep consecutive tiles,
+    // warps take the tile groups the host dealt them (see assign_warp_groups).
+    const int tile = ((int)p.warp_group[tid >> 5] << 5) | (tid & 31);
+    const int t0 = tile * R;
+    uint32_t *my_chunk = Fw + (kPadChunks + tile) * CS;
     const uint32_t row_bytes = (uint32_t)pitch * 4u;
     const int32_t *G_inst = p.G + (size_t)n * S * pitch;
     uint16_t *F16_inst = p.A + (size_t)n * S * pitch;     // prefix tables F_s as uint16 rows
@@ -131,6 +136,7 @@ minplus16_kernel(const Params p)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = tid; i < kPadChunks * CS; i += NT) Fw[i] = kInf16x2;
+    for (int i = tid; i < THEMIS_MAX_STAGES; i += NT) stage_lmin[i] = 0xFFFFFFFFu;
     for (int l = pitch + tid; l < Tp; l += NT) {
         Gbuf0[l] = kInf16x2;
         Gbuf1[l] = kInf16x2;
@@ -162,17 +168,28 @@ minplus16_kernel(const Params p)
 
     // stage 0: F_0 = G_0
     if (!mbar_wait(&mbar[0], 0)) failed = 1; else pend0 = -1;
+    // Records the lowest reachable index among this thread's R entries of row s.
+    auto note_first_reachable = [&](uint32_t first, int s) {
+        first = __reduce_min_sync(0xFFFFFFFFu, first);
+        if ((tid & 31) == 0 && first != 0xFFFFFFFFu) atomicMin(&stage_lmin[s], first);
+    };
     {
-        uint32_t w[H];
+        uint32_t w[H], first = 0xFFFFFFFFu;
 #pragma unroll
-        for (int r = 0; r < H; ++r) {
+        for (int r = H - 1; r >= 0; --r) {
             // raw costs; entries beyond the loaded row hold kInf16x2, far above kInf16
             const uint32_t lo = min(Gbuf0[t0 + 2 * r], kInf16), hi = min(Gbuf0[t0 + 2 * r + 1], kInf16);
             w[r] = lo | (hi << 16);
+            if (hi < kInf16) first = (uint32_t)(t0 + 2 * r + 1);
+            if (lo < kInf16) first = (uint32_t)(t0 + 2 * r);
         }
+        note_first_reachable(first, 0);
         store_chunk(w, 0);
     }
     failed = __syncthreads_or(failed);
+    // Lowest reachable budget of the prefix F_{s-1} (0xFFFFFFFF: nothing reachable).  Everything
+    // below it, and every G_s[l] below that row's first reachable l, can only give "unreachable".
+    uint32_t prefix_min = stage_lmin[0];
 
     for (int s = 1; s < S && !failed; ++s) {
         const int cur = s & 1;
@@ -181,12 +198,17 @@ minplus16_kernel(const Params p)
         if (!mbar_wait(&mbar[cur], (uint32_t)parity)) failed = 1;
         else if (cur) pend1 = -1; else pend0 = -1;
         // raw costs -> saturated cost duplicated into both half-words, in place
-        if (t0 < pitch) {
+        {
+            uint32_t first = 0xFFFFFFFFu;
+            if (t0 < pitch) {
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                const uint32_t v = min(Gk[t0 + r], kInf16);
-                Gk[t0 + r] = v | (v << 16);
+                for (int r = R - 1; r >= 0; --r) {
+                    const uint32_t v = min(Gk[t0 + r], kInf16);
+                    Gk[t0 + r] = v | (v << 16);
+                    if (v < kInf16) first = (uint32_t)(t0 + r);
+                }
             }
+            note_first_reachable(first, s);
         }
         failed = __syncthreads_or(failed);                // G_s and F_{s-1} visible to all
         if (failed) break;
@@ -202,24 +224,38 @@ minplus16_kernel(const Params p)
 
         uint32_t acc[H], accp[H], wa[H], wb[H];
 #pragma unroll
-        for (int r = 0; r < H; ++r) { acc[r] = 0xFFFFFFFFu; accp[r] = 0xFFFFFFFFu; wa[r] = my_chunk[r]; }
+        for (int r = 0; r < H; ++r) { acc[r] = 0xFFFFFFFFu; accp[r] = 0xFFFFFFFFu; }
         // All lanes of a warp walk the same l so that G is a broadcast; lanes that run
-        // past their own range read the "unreachable" chunks in front of F[0].
-        const int q_end = tid | 31;
-        const uint32_t *f_lo = my_chunk - CS;
-        const uint32_t *g = Gk;
-        for (int q = 0; q <= q_end; q += 2) {
-            chunk_step16<R>(wa, wb, acc, accp, f_lo, g);
-            chunk_step16<R>(wb, wa, acc, accp, f_lo - CS, g + R);
-            f_lo -= 2 * CS;
-            g += 2 * R;
+        // past their own range read the "unreachable" chunks in front of F[0].  Chunks of
+        // l below G_s's first reachable entry, and chunks that only meet F_{s-1} below its
+        // first reachable budget, are skipped (whole steps of U chunks, block-uniform).
+        const uint32_t g_min = stage_lmin[s];
+        const bool dead = g_min == 0xFFFFFFFFu || prefix_min == 0xFFFFFFFFu;
+        const int q_lo = dead ? 0 : (int)(g_min / R) & ~(U - 1);
+        const int q_hi = dead ? -1 : (tile | 31) - ((int)(prefix_min / R) & ~(U - 1));
+        if (q_lo <= q_hi) {
+            const uint32_t *f_hi = my_chunk - q_lo * CS;  // chunk tile - q_lo: at worst a pad chunk
+#pragma unroll
+            for (int r = 0; r < H; ++r) wa[r] = f_hi[r];
+            const uint32_t *f_lo = f_hi - CS;
+            const uint32_t *g = Gk + q_lo * R;
+            for (int q = q_lo; q <= q_hi; q += U) {
+#pragma unroll
+                for (int u = 0; u < U; u += 2) {
+                    chunk_step16<R>(wa, wb, acc, accp, f_lo - u * CS, g + u * R);
+                    chunk_step16<R>(wb, wa, acc, accp, f_lo - (u + 1) * CS, g + (u + 1) * R);
+                }
+                f_lo -= U * CS;
+                g += U * R;
+            }
         }
-        if ((tid & 31) == 31) xchg[tid >> 5] = accp[H - 1];
+        prefix_min = dead ? 0xFFFFFFFFu : prefix_min + g_min;
+        if ((tid & 31) == 31) xchg[tile >> 5] = accp[H - 1];
         __syncthreads();                                  // every read of F_{s-1} is done
 
         // merge: cell 2j comes from acc[j].lo and accp[j-1].hi, cell 2j+1 from acc[j].hi and accp[j].lo
         uint32_t left = __shfl_up_sync(0xFFFFFFFFu, accp[H - 1], 1);
-        if ((tid & 31) == 0) left = tid == 0 ? 0xFFFFFFFFu : xchg[(tid >> 5) - 1];
+        if ((tid & 31) == 0) left = tile == 0 ? 0xFFFFFFFFu : xchg[(tile >> 5) - 1];
         uint32_t w[H];
 #pragma unroll
         for (int r = 0; r < H; ++r) {
@@ -326,8 +362,10 @@ minplus16_kernel(const Params p)
 }
 
 template <int R, int MAXT>
-cudaError_t launch_variant16(const Params &p, int threads, size_t smem, cudaStream_t stream)
+cudaError_t launch_variant16(const Params &p_in, int threads, size_t smem, cudaStream_t stream)
 {
+    Params p = p_in;
+    assign_warp_groups(threads / 32, p.warp_group);
     cudaError_t e = cudaFuncSetAttribute(minplus16_kernel<R, MAXT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)smem);
     if (e != cudaSuccess) return e;
@@ -341,12 +379,12 @@ cudaError_t launch_minplus16(const Params &p, int tile, cudaStream_t stream)
 {
     const int cells = p.T + 1;
     int R = tile;
-    if (R != 8 && R != 16) R = cells <= 2048 ? 8 : 16;
+    if (R != 8 && R != 16) R = 8;                        // finer tiles waste fewer cells past the diagonal
     if (R == 8 && (cells + 7) / 8 > 1024) R = 16;
     const int chunks = (cells + R - 1) / R;
     const int threads = (chunks + 31) / 32 * 32;
     const int CS = R == 16 ? 12 : 4;
-    const size_t words = (size_t)(kPadChunks + threads) * CS + 2u * (size_t)threads * R + 4 + 32 + 32;
+    const size_t words = (size_t)(kPadChunks + threads) * CS + 2u * (size_t)threads * R + 4 + 32 + 32 + THEMIS_MAX_STAGES;
     const size_t smem = words * sizeof(uint32_t);
     if (R == 8)
         return threads <= 512 ? launch_variant16<8, 512>(p, threads, smem, stream)
