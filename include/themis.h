@@ -149,6 +149,25 @@ int themis_solve_vertical_batch(const themis_problem_t *problem, const int32_t *
                                 void *d_workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Horizontal-only variant (Algorithm 2): one-core replicas.  problem->c_max must
+ * be 1 and d_lat_us is [P][S][1][n_batch].  For every stage and batch size the
+ * replica count is not enumerated but computed, h = ceil(lambda / thr(b, 1)), the
+ * fewest replicas with thr * h >= lambda (Algorithm 2 prints a floor, which would
+ * break Eq. 6's throughput constraint); batch sizes that would need more than
+ * problem->h_max replicas are dropped.  Cost of a stage is h.  Results equal those
+ * of themis_solve_batch on the same problem (extra replicas only add cost and
+ * queuing delay), at n_batch instead of h_max * n_batch candidates per stage.
+ * In the workspace, Garg holds the batch index and G the replica count.
+ * Solving the same pipelines at the current and at the predicted arrival rate
+ * (two batches, or one batch of 2N instances) and comparing the returned
+ * configurations is the paper's test for a stable workload (Section "Transition").
+ */
+int themis_solve_horizontal_batch(const themis_problem_t *problem, const int32_t *d_lat_us,
+                                  const int32_t *d_profile_id, const uint32_t *d_lambda_mrps,
+                                  themis_result_t out, void *d_workspace, size_t workspace_bytes,
+                                  void *cuda_stream);
+
+/*
  * The two halves of the solvers, for checking and timing each step on its own.
  * themis_score_batch fills G and Garg of the workspace (candidate scoring: the
  * inner loops of Algorithm 1 with Eq. 4 and the throughput test of Eq. 6);

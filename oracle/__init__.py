@@ -60,7 +60,9 @@ def _load():
         lib.oracle_score_stage.argtypes = [P, vp, ctypes.c_uint32, ctypes.c_int32, ctypes.c_int32, vp, vp]
         lib.oracle_minplus.restype = None
         lib.oracle_minplus.argtypes = [ctypes.c_int32, vp, vp, vp, vp]
-        for fn in (lib.oracle_alg1_scatter, lib.brute_force_instance):
+        lib.oracle_solve_horizontal_batch.restype = ctypes.c_int
+        lib.oracle_solve_horizontal_batch.argtypes = [P] + [vp] * 13 + [ctypes.c_int]
+        for fn in (lib.oracle_alg1_scatter, lib.oracle_alg2_scatter, lib.brute_force_instance):
             fn.restype = ctypes.c_int
             fn.argtypes = [P, vp, ctypes.c_uint32, vp, vp, vp, vp, vp, vp]
         _lib = lib
@@ -90,9 +92,11 @@ def _c(a, dtype):
     return None if a is None else np.ascontiguousarray(a, dtype=dtype)
 
 
-def solve_batch(wl, dumps: bool = False, n_threads: int = 0) -> dict:
+def solve_batch(wl, dumps: bool = False, n_threads: int = 0, horizontal: bool = False) -> dict:
     """Solve every instance of a workload (any object with the attributes of
     ``workloads.Workload``) with the dynamic-programming oracle.
+    ``horizontal`` selects Algorithm 2 (one-core replicas, replica count
+    computed per batch size, at most ``h_max``); the workload must have c_max 1.
 
     Returns numpy arrays ``h, c, b`` [N][S], ``total_cost, latency_buckets,
     status`` [N] and ``threads``; with ``dumps`` also ``G, Garg, F, A``
@@ -112,14 +116,16 @@ def solve_batch(wl, dumps: bool = False, n_threads: int = 0) -> dict:
         out["Garg"] = np.empty((N, S, W), np.uint16)
         out["F"] = np.empty((N, S, W), np.int32)
         out["A"] = np.empty((N, S, W), np.uint16)
-    rc = lib.oracle_solve_batch(
-        ctypes.byref(p), _ptr(lat), _ptr(pid), _ptr(lam), _ptr(rep),
-        _ptr(out["h"]), _ptr(out["c"]), _ptr(out["b"]),
-        _ptr(out["total_cost"]), _ptr(out["latency_buckets"]), _ptr(out["status"]),
-        _ptr(out.get("G")), _ptr(out.get("Garg")), _ptr(out.get("F")), _ptr(out.get("A")),
-        int(n_threads))
+    tail = (_ptr(out["h"]), _ptr(out["c"]), _ptr(out["b"]),
+            _ptr(out["total_cost"]), _ptr(out["latency_buckets"]), _ptr(out["status"]),
+            _ptr(out.get("G")), _ptr(out.get("Garg")), _ptr(out.get("F")), _ptr(out.get("A")),
+            int(n_threads))
+    if horizontal:
+        rc = lib.oracle_solve_horizontal_batch(ctypes.byref(p), _ptr(lat), _ptr(pid), _ptr(lam), *tail)
+    else:
+        rc = lib.oracle_solve_batch(ctypes.byref(p), _ptr(lat), _ptr(pid), _ptr(lam), _ptr(rep), *tail)
     if rc < 0:
-        raise MemoryError("oracle_solve_batch: allocation failed")
+        raise MemoryError("oracle_solve_batch: allocation failed or unsupported problem")
     out["threads"] = rc
     return out
 
@@ -143,6 +149,11 @@ def _per_instance(fn, wl, n: int) -> dict:
 def alg1_scatter(wl, n: int) -> dict:
     """Instance ``n`` solved by Algorithm 1 in the paper's own loop order."""
     return _per_instance(_load().oracle_alg1_scatter, wl, n)
+
+
+def alg2_scatter(wl, n: int) -> dict:
+    """Instance ``n`` solved by Algorithm 2 in the paper's own loop order (c_max = 1)."""
+    return _per_instance(_load().oracle_alg2_scatter, wl, n)
 
 
 def brute_force(wl, n: int) -> dict:

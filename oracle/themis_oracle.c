@@ -27,7 +27,11 @@
  *   oracle_alg1_scatter     Algorithm 1 in the paper's own loop order
  *                           (stage, budget descending, cores, batch), scattering
  *                           into best[s][i + l];
- *   brute_force.c           Eq. 6 by exhaustive enumeration (separate file).
+ *   brute_force.c           Eq. 6 by exhaustive enumeration (separate file);
+ * and, for the horizontal-only solver of Algorithm 2 (one-core replicas, replica
+ * count computed as ceil(lambda / thr) per batch size):
+ *   oracle_solve_horizontal_batch   the same program over batch sizes only;
+ *   oracle_alg2_scatter             Algorithm 2 in the paper's loop order.
  *
  * Readings of the paper taken here (each is pinned by a test):
  *   - a candidate is skipped iff its replicas cannot sustain lambda or it does
@@ -126,6 +130,41 @@ void oracle_score_stage(const oracle_problem *p, const int32_t *lat_stage, uint3
 }
 
 /*
+ * Horizontal scaling (Algorithm 2): one-core replicas only.  For every batch
+ * size the replica count is computed, not enumerated: the fewest replicas whose
+ * combined throughput sustains lambda, h = ceil(lambda / thr(b, 1)) (Algorithm 2
+ * prints a floor, which would leave thr * h below lambda; Eq. 6 requires
+ * thr * h >= lambda).  Candidates that would need more than h_max replicas are
+ * dropped.  Cost is h (one core each); candidate index = batch index.
+ * lat_stage is [1][n_batch].
+ */
+static int horizontal_candidate(const oracle_problem *p, int32_t l_us, int32_t b, uint32_t lambda_m,
+                                int64_t *ell, int32_t *h_out)
+{
+    uint64_t per_replica = (uint64_t)b * 1000000000ull;              /* b / l, scaled */
+    uint64_t demand = (uint64_t)lambda_m * (uint64_t)l_us;
+    uint64_t h = ceil_div_u64(demand, per_replica);
+    if (h < 1) h = 1;
+    if (h > (uint64_t)p->h_max) return 0;
+    int32_t cost;
+    if (!score_candidate(l_us, (int32_t)h, 1, b, lambda_m, p->bucket_us, p->flags, ell, &cost)) return 0;
+    *h_out = (int32_t)h;
+    return 1;
+}
+
+void oracle_score_stage_horizontal(const oracle_problem *p, const int32_t *lat_stage, uint32_t lambda_m,
+                                   int32_t T, int32_t *G, uint16_t *Garg)
+{
+    for (int32_t l = 0; l <= T; ++l) { G[l] = ORACLE_INF; Garg[l] = 0; }
+    for (int32_t bi = 0; bi < p->n_batch; ++bi) {
+        int64_t ell; int32_t h;
+        if (!horizontal_candidate(p, lat_stage[bi], p->batch_sizes[bi], lambda_m, &ell, &h)) continue;
+        if (ell > T) continue;
+        if (h < G[ell]) { G[ell] = h; Garg[ell] = (uint16_t)bi; }
+    }
+}
+
+/*
  * Min-plus combine of the prefix with one more stage:
  *   F[t] = min_{0 <= l <= t} Fprev[t - l] + G[l],  A[t] = lowest l attaining it
  * (A[t] = 0 where F[t] is INF).
@@ -159,16 +198,21 @@ static void decode_idx(const oracle_problem *p, int32_t idx, int32_t h_fixed,
  * Returns 0 (solved) or 1 (infeasible).
  */
 static int solve_instance(const oracle_problem *p, const int32_t *lat_pipeline /* [S][C][B] */,
-                          uint32_t lambda_m, const int32_t *replicas /* [S] or NULL */,
+                          uint32_t lambda_m, const int32_t *replicas /* [S] or NULL */, int horizontal,
                           int32_t *h_out, int32_t *c_out, int32_t *b_out,
                           int32_t *cost_out, int32_t *lat_out,
                           int32_t *Gs, uint16_t *Gargs, int32_t *Fs, uint16_t *As)
 {
     const int32_t S = p->n_stages, T = p->slo_us / p->bucket_us, W = T + 1;
     const int32_t stage_words = p->c_max * p->n_batch;
-    for (int32_t s = 0; s < S; ++s)
-        oracle_score_stage(p, lat_pipeline + (size_t)s * stage_words, lambda_m,
-                           replicas ? replicas[s] : 0, T, Gs + (size_t)s * W, Gargs + (size_t)s * W);
+    for (int32_t s = 0; s < S; ++s) {
+        if (horizontal)
+            oracle_score_stage_horizontal(p, lat_pipeline + (size_t)s * stage_words, lambda_m, T,
+                                          Gs + (size_t)s * W, Gargs + (size_t)s * W);
+        else
+            oracle_score_stage(p, lat_pipeline + (size_t)s * stage_words, lambda_m,
+                               replicas ? replicas[s] : 0, T, Gs + (size_t)s * W, Gargs + (size_t)s * W);
+    }
     /* first stage: the whole budget spent so far belongs to it */
     memcpy(Fs, Gs, sizeof(int32_t) * (size_t)W);
     memset(As, 0, sizeof(uint16_t) * (size_t)W);
@@ -190,7 +234,11 @@ static int solve_instance(const oracle_problem *p, const int32_t *lat_pipeline /
     for (int32_t s = S - 1; s >= 0; --s) {
         int32_t ell = s > 0 ? (int32_t)As[(size_t)s * W + t] : t;
         int32_t idx = Gargs[(size_t)s * W + ell];
-        decode_idx(p, idx, replicas ? replicas[s] : 0, &h_out[s], &c_out[s], &b_out[s]);
+        if (horizontal) {      /* the stage's cost is its replica count */
+            h_out[s] = Gs[(size_t)s * W + ell]; c_out[s] = 1; b_out[s] = p->batch_sizes[idx];
+        } else {
+            decode_idx(p, idx, replicas ? replicas[s] : 0, &h_out[s], &c_out[s], &b_out[s]);
+        }
         t -= ell;
     }
     *cost_out = best; *lat_out = tstar;
@@ -210,12 +258,12 @@ static int solve_instance(const oracle_problem *p, const int32_t *lat_pipeline /
  * n_threads <= 0 uses every core OpenMP sees.  Returns the thread count used,
  * or -1 on allocation failure.
  */
-int oracle_solve_batch(const oracle_problem *p, const int32_t *lat_us, const int32_t *profile_id,
-                       const uint32_t *lambda_mrps, const int32_t *replicas,
-                       int32_t *h, int32_t *c, int32_t *b,
-                       int32_t *total_cost, int32_t *latency_buckets, int32_t *status,
-                       int32_t *dump_G, uint16_t *dump_Garg, int32_t *dump_F, uint16_t *dump_A,
-                       int n_threads)
+static int solve_batch_mode(const oracle_problem *p, const int32_t *lat_us, const int32_t *profile_id,
+                            const uint32_t *lambda_mrps, const int32_t *replicas, int horizontal,
+                            int32_t *h, int32_t *c, int32_t *b,
+                            int32_t *total_cost, int32_t *latency_buckets, int32_t *status,
+                            int32_t *dump_G, uint16_t *dump_Garg, int32_t *dump_F, uint16_t *dump_A,
+                            int n_threads)
 {
     const int32_t N = p->n_instances, S = p->n_stages;
     const size_t W = (size_t)(p->slo_us / p->bucket_us) + 1;
@@ -244,7 +292,7 @@ int oracle_solve_batch(const oracle_problem *p, const int32_t *lat_us, const int
             for (int32_t n = 0; n < N; ++n) {
                 int32_t pid = profile_id ? profile_id[n] : 0;
                 status[n] = solve_instance(p, lat_us + (size_t)pid * pipeline_words, lambda_mrps[n],
-                                           replicas ? replicas + (size_t)n * S : NULL,
+                                           replicas ? replicas + (size_t)n * S : NULL, horizontal,
                                            h + (size_t)n * S, c + (size_t)n * S, b + (size_t)n * S,
                                            &total_cost[n], &latency_buckets[n], Gs, Gargs, Fs, As);
                 if (dump_G) memcpy(dump_G + (size_t)n * rows, Gs, sizeof(int32_t) * rows);
@@ -256,6 +304,92 @@ int oracle_solve_batch(const oracle_problem *p, const int32_t *lat_us, const int
         free(Gs); free(Fs); free(Gargs); free(As);
     }
     return failed ? -1 : used;
+}
+
+int oracle_solve_batch(const oracle_problem *p, const int32_t *lat_us, const int32_t *profile_id,
+                       const uint32_t *lambda_mrps, const int32_t *replicas,
+                       int32_t *h, int32_t *c, int32_t *b,
+                       int32_t *total_cost, int32_t *latency_buckets, int32_t *status,
+                       int32_t *dump_G, uint16_t *dump_Garg, int32_t *dump_F, uint16_t *dump_A,
+                       int n_threads)
+{
+    return solve_batch_mode(p, lat_us, profile_id, lambda_mrps, replicas, 0, h, c, b, total_cost,
+                            latency_buckets, status, dump_G, dump_Garg, dump_F, dump_A, n_threads);
+}
+
+/* Horizontal-only variant (Algorithm 2): c_max must be 1, lat_us is [P][S][1][n_batch]. */
+int oracle_solve_horizontal_batch(const oracle_problem *p, const int32_t *lat_us, const int32_t *profile_id,
+                                  const uint32_t *lambda_mrps,
+                                  int32_t *h, int32_t *c, int32_t *b,
+                                  int32_t *total_cost, int32_t *latency_buckets, int32_t *status,
+                                  int32_t *dump_G, uint16_t *dump_Garg, int32_t *dump_F, uint16_t *dump_A,
+                                  int n_threads)
+{
+    if (p->c_max != 1) return -1;
+    return solve_batch_mode(p, lat_us, profile_id, lambda_mrps, NULL, 1, h, c, b, total_cost,
+                            latency_buckets, status, dump_G, dump_Garg, dump_F, dump_A, n_threads);
+}
+
+/*
+ * Algorithm 2 in the paper's loop order, one instance: as oracle_alg1_scatter, with
+ * the candidate loop over batch sizes only and the replica count computed per
+ * candidate.  lat_pipeline is [S][1][n_batch].
+ */
+int oracle_alg2_scatter(const oracle_problem *p, const int32_t *lat_pipeline, uint32_t lambda_m,
+                        const int32_t *unused, int32_t *h_out, int32_t *c_out, int32_t *b_out,
+                        int32_t *cost_out, int32_t *lat_out)
+{
+    (void)unused;
+    const int32_t S = p->n_stages, T = p->slo_us / p->bucket_us, W = T + 1;
+    const size_t cells = (size_t)S * W;
+    uint8_t *dp = (uint8_t *)calloc(cells, 1);
+    int32_t *best_total = (int32_t *)malloc(sizeof(int32_t) * cells);
+    int32_t *best_ell = (int32_t *)malloc(sizeof(int32_t) * cells);
+    int32_t *best_ins = (int32_t *)malloc(sizeof(int32_t) * cells);
+    int32_t *best_bi = (int32_t *)malloc(sizeof(int32_t) * cells);
+    if (!dp || !best_total || !best_ell || !best_ins || !best_bi) {
+        free(dp); free(best_total); free(best_ell); free(best_ins); free(best_bi);
+        return -1;
+    }
+    for (int32_t s = 0; s < S; ++s) {
+        const int32_t *lat_stage = lat_pipeline + (size_t)s * p->n_batch;
+        for (int32_t i = T; i >= 0; --i) {
+            int reachable = (s == 0) ? (i == 0) : dp[(size_t)(s - 1) * W + i];
+            if (!reachable) continue;
+            for (int32_t bi = 0; bi < p->n_batch; ++bi) {
+                int64_t ell; int32_t ins;
+                if (!horizontal_candidate(p, lat_stage[bi], p->batch_sizes[bi], lambda_m, &ell, &ins)) continue;
+                if ((int64_t)i + ell > T) continue;
+                int32_t total = ins + (s == 0 ? 0 : best_total[(size_t)(s - 1) * W + i]);
+                size_t dst = (size_t)s * W + (size_t)(i + ell);
+                if (!dp[dst] || total < best_total[dst]) {
+                    dp[dst] = 1; best_total[dst] = total; best_ell[dst] = (int32_t)ell;
+                    best_ins[dst] = ins; best_bi[dst] = bi;
+                }
+            }
+        }
+    }
+    int32_t least = ORACLE_INF, ind = -1;
+    for (int32_t i = 0; i <= T; ++i) {
+        size_t k = (size_t)(S - 1) * W + i;
+        if (dp[k] && best_total[k] < least) { least = best_total[k]; ind = i; }
+    }
+    int rc = 1;
+    if (ind < 0) {
+        for (int32_t s = 0; s < S; ++s) { h_out[s] = 0; c_out[s] = 0; b_out[s] = 0; }
+        *cost_out = -1; *lat_out = -1;
+    } else {
+        int32_t t = ind;
+        for (int32_t s = S - 1; s >= 0; --s) {
+            size_t k = (size_t)s * W + t;
+            h_out[s] = best_ins[k]; c_out[s] = 1; b_out[s] = p->batch_sizes[best_bi[k]];
+            t -= best_ell[k];
+        }
+        *cost_out = least; *lat_out = ind;
+        rc = 0;
+    }
+    free(dp); free(best_total); free(best_ell); free(best_ins); free(best_bi);
+    return rc;
 }
 
 /*

@@ -12,6 +12,7 @@ namespace {
 thread_local cudaError_t t_last_cuda = cudaSuccess;
 thread_local char t_msg[256];
 int g_tile = 0;   // min-plus cells per thread; 0 = built-in choice
+thread_local bool g_horizontal = false;   // set by solve_impl for the launches it makes
 int g_mode = 0;   // 0: packed 16-bit min-plus kernel with 32-bit second pass; 1: 32-bit kernel only
 
 constexpr size_t kAlign = 256;
@@ -88,6 +89,7 @@ int make_params(const themis_problem_t *pr, int vertical, void *ws, size_t ws_by
     P->pitch = L.row_pitch;
     P->vertical = vertical ? 1 : 0;
     P->K = (vertical ? 1 : pr->h_max) * pr->c_max * pr->n_batch;
+    P->horizontal = (!vertical && g_horizontal) ? 1 : 0;
     char *base = static_cast<char *>(ws);
     P->G = reinterpret_cast<int32_t *>(base + L.g_offset);
     P->Garg = reinterpret_cast<uint16_t *>(base + L.garg_offset);
@@ -139,16 +141,20 @@ int minplus_impl(const themis_problem_t *pr, const int32_t *rep, int vertical, t
     return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
 }
 
+// mode: 0 joint, 1 vertical (h fixed), 2 horizontal (Algorithm 2)
 int solve_impl(const themis_problem_t *pr, const int32_t *lat, const int32_t *pid, const uint32_t *lam,
-               const int32_t *rep, int vertical, themis_result_t out, void *ws, size_t ws_bytes, cudaStream_t st)
+               const int32_t *rep, int mode, themis_result_t out, void *ws, size_t ws_bytes, cudaStream_t st)
 {
+    const int vertical = mode == 1;
+    g_horizontal = mode == 2;
     int32_t T, K;
     int rc = validate(pr, vertical, &T, &K);
     if (rc != THEMIS_OK) return rc;
     if (!result_ok(out)) return THEMIS_E_INVALID_ARG;
     rc = score_impl(pr, lat, pid, lam, rep, vertical, ws, ws_bytes, st);
-    if (rc != THEMIS_OK) return rc;
-    return minplus_impl(pr, rep, vertical, out, ws, ws_bytes, st);
+    if (rc == THEMIS_OK) rc = minplus_impl(pr, rep, vertical, out, ws, ws_bytes, st);
+    g_horizontal = false;
+    return rc;
 }
 
 // Staging area appended to the solver workspace by the host-buffer variant.
@@ -258,6 +264,16 @@ int themis_solve_vertical_batch(const themis_problem_t *problem, const int32_t *
 {
     if (!d_replicas) return THEMIS_E_INVALID_ARG;
     return solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, d_replicas, 1, out, d_workspace,
+                      workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int themis_solve_horizontal_batch(const themis_problem_t *problem, const int32_t *d_lat_us,
+                                  const int32_t *d_profile_id, const uint32_t *d_lambda_mrps,
+                                  themis_result_t out, void *d_workspace, size_t workspace_bytes,
+                                  void *cuda_stream)
+{
+    if (problem && problem->c_max != 1) return THEMIS_E_INVALID_ARG;
+    return solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, nullptr, 2, out, d_workspace,
                       workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 

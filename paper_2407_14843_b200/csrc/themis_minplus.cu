@@ -236,7 +236,8 @@ minplus_kernel(const Params p)
                 const int bi = idx % NB, rest = idx / NB;
                 b_o[s] = p.prob.batch_sizes[bi];
                 c_o[s] = rest % C + 1;
-                h_o[s] = p.vertical ? p.replicas[(size_t)n * S + s] : rest / C + 1;
+                h_o[s] = p.vertical ? p.replicas[(size_t)n * S + s]
+                       : p.horizontal ? G_inst[(size_t)s * pitch + ell] : rest / C + 1;
                 t -= ell;
             }
             p.out.total_cost[n] = (int32_t)(best >> kIdxBits);

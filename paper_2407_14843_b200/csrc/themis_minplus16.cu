@@ -341,7 +341,8 @@ minplus16_kernel(const Params p)
             const int bi = idx % NB, rest = idx / NB;
             b_o[s] = p.prob.batch_sizes[bi];
             c_o[s] = rest % C + 1;
-            h_o[s] = p.vertical ? p.replicas[(size_t)n * S + s] : rest / C + 1;
+            h_o[s] = p.vertical ? p.replicas[(size_t)n * S + s]
+                       : p.horizontal ? G_inst[(size_t)s * pitch + ell] : rest / C + 1;
         }
     }
     if (tid == 0) {
@@ -353,7 +354,7 @@ minplus16_kernel(const Params p)
             const int bi = idx % NB, rest = idx / NB;
             b_o[0] = p.prob.batch_sizes[bi];
             c_o[0] = rest % C + 1;
-            h_o[0] = p.vertical ? p.replicas[(size_t)n * S] : rest / C + 1;
+            h_o[0] = p.vertical ? p.replicas[(size_t)n * S] : p.horizontal ? G_inst[t] : rest / C + 1;
             p.out.total_cost[n] = (int32_t)best_cost;
             p.out.latency_buckets[n] = tstar;
             p.out.status[n] = THEMIS_STATUS_OK;

@@ -115,7 +115,9 @@ score_kernel(const Params p)
                 const uint32_t l_b = l_q + (l_r != 0u);
                 if (l_b > (uint32_t)T) continue;
                 const int b = p.prob.batch_sizes[bi];
-                const bool q_const = !q_grows_with_h || b == 1;
+                // Stop at the fewest replicas when more of them cannot reach another bucket
+                // more cheaply (q does not depend on h), or when only that count is a candidate.
+                const bool q_const = !q_grows_with_h || b == 1 || p.horizontal;
                 const uint32_t *q_row = Q_s + bi * HN;
                 const uint32_t *lmax_row = Lmax_s + bi * HN;
                 // Fewest replicas that sustain lambda: feasibility is monotone in h.  Start
@@ -127,7 +129,7 @@ score_kernel(const Params p)
                 if (k > 0 && (uint32_t)l_us <= lmax_row[k - 1]) k = 0;     // estimate not below: scan from 0
                 while (k < HN && (uint32_t)l_us > lmax_row[k]) ++k;        // cannot sustain lambda
                 uint32_t cost = (uint32_t)(h_lo + k) * (uint32_t)c;
-                uint32_t idx = (uint32_t)(k * CB + pair);
+                uint32_t idx = (uint32_t)((p.horizontal ? 0 : k * CB) + pair);
                 for (; k < HN; ++k, cost += (uint32_t)c, idx += (uint32_t)CB) {
                     const uint32_t ell = l_b + q_row[k];
                     if (ell > (uint32_t)T) break;                  // q never shrinks with h

@@ -32,6 +32,7 @@ EXPORTS = (
     "themis_solve_batch", "themis_solve_vertical_batch", "themis_score_batch", "themis_minplus_batch",
     "themis_host_workspace_bytes", "themis_solve_batch_host", "themis_alu_probe",
     "themis_set_minplus_tile", "themis_solve_batch_static", "themis_set_minplus_mode",
+    "themis_solve_horizontal_batch",
 )
 
 
@@ -95,6 +96,7 @@ def _load() -> ctypes.CDLL:
     lib.themis_workspace_layout.argtypes = [PP, ctypes.c_int, ctypes.POINTER(WorkspaceLayout)]
     lib.themis_solve_batch.argtypes = [PP, vp, vp, vp, Result, vp, sz, vp]
     lib.themis_solve_vertical_batch.argtypes = [PP, vp, vp, vp, vp, Result, vp, sz, vp]
+    lib.themis_solve_horizontal_batch.argtypes = [PP, vp, vp, vp, Result, vp, sz, vp]
     lib.themis_score_batch.argtypes = [PP, vp, vp, vp, vp, vp, sz, vp]
     lib.themis_minplus_batch.argtypes = [PP, vp, Result, vp, sz, vp]
     lib.themis_solve_batch_host.argtypes = [PP, vp, vp, vp, vp, Result, vp, sz, vp]
@@ -177,6 +179,13 @@ def themis_solve_vertical_batch(problem: Problem, lat_us, profile_id, lambda_mrp
         ctypes.byref(problem), _dptr(lat_us, torch.int32, "lat_us"), _dptr(profile_id, torch.int32, "profile_id"),
         _dptr(lambda_mrps, torch.uint32, "lambda_mrps"), _dptr(replicas, torch.int32, "replicas"), _result(out),
         _dptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()), "themis_solve_vertical_batch")
+
+
+def themis_solve_horizontal_batch(problem: Problem, lat_us, profile_id, lambda_mrps, out: dict, workspace) -> None:
+    _check(_lib.themis_solve_horizontal_batch(
+        ctypes.byref(problem), _dptr(lat_us, torch.int32, "lat_us"), _dptr(profile_id, torch.int32, "profile_id"),
+        _dptr(lambda_mrps, torch.uint32, "lambda_mrps"), _result(out),
+        _dptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()), "themis_solve_horizontal_batch")
 
 
 def themis_score_batch(problem: Problem, lat_us, profile_id, lambda_mrps, replicas, workspace) -> None:
@@ -275,14 +284,17 @@ def workspace_tables(problem: Problem, vertical: bool, workspace: torch.Tensor) 
 
 
 def solve(wl, dev: Optional[dict] = None, workspace: Optional[torch.Tensor] = None,
-          out: Optional[dict] = None):
+          out: Optional[dict] = None, horizontal: bool = False):
     """Solve a workload on the current device: allocates what is not given,
-    then calls ``themis_solve_batch`` / ``themis_solve_vertical_batch``."""
+    then calls ``themis_solve_batch`` / ``themis_solve_vertical_batch`` (or
+    ``themis_solve_horizontal_batch`` when ``horizontal``)."""
     problem = Problem.of_workload(wl)
     dev = dev if dev is not None else workload_to_device(wl)
     workspace = workspace if workspace is not None else alloc_workspace(problem, wl.vertical)
     out = out if out is not None else alloc_result(wl.n_instances, wl.n_stages)
-    if wl.vertical:
+    if horizontal:
+        themis_solve_horizontal_batch(problem, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"], out, workspace)
+    elif wl.vertical:
         themis_solve_vertical_batch(problem, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"],
                                     dev["replicas"], out, workspace)
     else:

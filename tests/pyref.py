@@ -31,6 +31,30 @@ def stage_candidates(lat_us_stage, c_max, batch_sizes, h_values, lambda_mrps, bu
     return out
 
 
+def stage_candidates_horizontal(lat_us_stage, batch_sizes, h_max, lambda_mrps, bucket_us, flags):
+    """Algorithm 2's candidates: one-core replicas, h = ceil(lambda / thr(b, 1))
+    (the fewest replicas with thr * h >= lambda), dropped when h > h_max."""
+    lam = Fraction(int(lambda_mrps), 1000)
+    w = Fraction(int(bucket_us), 1_000_000)
+    out = []
+    for bi, b in enumerate(batch_sizes):
+        l = Fraction(int(lat_us_stage[0][bi]), 1_000_000)
+        h = max(1, math.ceil(lam / (Fraction(b) / l)))
+        if h > h_max:
+            continue
+        q = Fraction(b - 1) / lam * (h if flags & 1 else 1)
+        out.append((bi, h, 1, b, math.ceil(l / w) + math.ceil(q / w), h))
+    return out
+
+
+def solve_instance_horizontal(wl, n):
+    pid = int(wl.profile_id[n])
+    stages = [stage_candidates_horizontal(wl.lat_us[pid][s], wl.batch_sizes, wl.h_max,
+                                          int(wl.lambda_mrps[n]), wl.bucket_us, wl.flags)
+              for s in range(wl.n_stages)]
+    return brute_force(stages, wl.T)
+
+
 def brute_force(stages, T):
     """Eq. 6 by enumeration with the lexicographic tie-break key
     (cost, total latency, ell_{S-1}, ..., ell_1, idx_0, ..., idx_{S-1})."""

@@ -21,9 +21,9 @@ def S():
     return solver
 
 
-def _gpu_solve(S, wl, tables=False):
+def _gpu_solve(S, wl, tables=False, horizontal=False):
     import torch
-    out, ws = S.solve(wl)
+    out, ws = S.solve(wl, horizontal=horizontal)
     torch.cuda.synchronize()
     res = {k: v.cpu().numpy() for k, v in out.items()}
     if tables:
@@ -160,6 +160,30 @@ def test_paper_scale_vertical(S, oracle_mod, mode):
     _assert_tables_equal(S, gpu, ref)
     _assert_results_equal(gpu, ref)
     assert (ref["status"] == 0).any()
+
+
+@pytest.mark.parametrize("flags", [0, W.QUEUE_PER_REPLICA])
+def test_horizontal_only_solver(S, oracle_mod, flags, mode):
+    """Algorithm 2 (one-core replicas, replica count computed): every table and
+    result against the oracle, and results against the joint entry point."""
+    for seed, (nb, h_max, T) in enumerate([((1, 2, 4, 8, 16), 12, 90), ((1, 2, 4, 8), 300, 700),
+                                           ((1, 2, 4, 8, 16, 32), 64, 2100)]):
+        wl = W.random_tiny_workload(7300 + seed, 48, 2 + seed, 1, nb, h_max, T, flags=flags,
+                                    rate_lo=20.0, rate_hi=900.0)
+        ref = oracle_mod.solve_batch(wl, dumps=True, horizontal=True)
+        gpu = _gpu_solve(S, wl, tables=True, horizontal=True)
+        _assert_tables_equal(S, gpu, ref)
+        _assert_results_equal(gpu, ref)
+        _assert_results_equal(_gpu_solve(S, wl), ref)          # joint solver, c_max = 1
+        assert (ref["status"] == 0).any()
+    import ctypes
+    bad = S.Problem.of_workload(W.make_workload(1))             # c_max = 8: refused
+    res = S.Result()
+    for k in ("h", "c", "b", "total_cost", "latency_buckets", "status"):
+        setattr(res, k, 256)
+    one = ctypes.c_void_p(256)
+    assert S._lib.themis_solve_horizontal_batch(ctypes.byref(bad), one, None, one, res, one, 1 << 40, None) \
+        == S.E_INVALID_ARG
 
 
 # ---------------------------------------------------------------- edge cases

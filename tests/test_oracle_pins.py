@@ -341,3 +341,50 @@ def test_pins_catch_planted_mistakes(oracle_mod):
     swapped = dataclasses.replace(wl, lat_us=np.ascontiguousarray(wl.lat_us.transpose(0, 1, 3, 2)))
     assert differs(oracle_mod.solve_batch(swapped)) > 0
     assert differs(oracle_mod.solve_batch(dataclasses.replace(wl, flags=0))) > 0
+
+
+# ---------------------------------------------------------------- horizontal-only solver (Algorithm 2)
+
+@pytest.mark.parametrize("flags", [0, W.QUEUE_PER_REPLICA])
+def test_horizontal_against_rational_brute_force_and_algorithm2(oracle_mod, flags):
+    """One-core replicas, replica count computed per batch size: the DP oracle
+    equals exhaustive search over batch-size tuples in exact rationals, and
+    Algorithm 2 run in the paper's loop order."""
+    n_inf = 0
+    for seed in range(8):
+        T = [60, 90, 140, 400][seed % 4]
+        wl = W.random_tiny_workload(7000 + seed, 24, 1 + seed % 4, 1, (1, 2, 4, 8, 16), 12, T, flags=flags,
+                                    rate_lo=20.0, rate_hi=400.0)
+        r = oracle_mod.solve_batch(wl, horizontal=True)
+        for n in range(wl.n_instances):
+            _assert_same(r, n, pyref.solve_instance_horizontal(wl, n), f"seed {seed} instance {n}")
+            _assert_same(r, n, oracle_mod.alg2_scatter(wl, n), f"scatter, seed {seed} instance {n}")
+        n_inf += int(r["status"].sum())
+        assert (r["c"][r["status"] == 0] == 1).all()
+    assert n_inf > 0
+
+
+def test_horizontal_equals_joint_restricted_to_one_core(oracle_mod):
+    """Extra replicas beyond the fewest that sustain lambda only add cost and
+    queuing delay, so enumerating h (joint solver, c_max = 1) changes nothing."""
+    wl = W.random_tiny_workload(7100, 48, 3, 1, (1, 2, 4, 8), 20, 110, rate_lo=20.0, rate_hi=300.0)
+    a = oracle_mod.solve_batch(wl, horizontal=True)
+    b = oracle_mod.solve_batch(wl)
+    for k in ("status", "total_cost", "latency_buckets", "h", "c", "b"):
+        assert np.array_equal(a[k], b[k]), k
+    assert (a["status"] == 0).any() and (a["status"] == 1).any()
+
+
+def test_horizontal_replica_counts_are_tight(oracle_mod):
+    """Every returned replica count sustains lambda and one replica fewer would not (Eq. 6)."""
+    wl = W.random_tiny_workload(7200, 32, 3, 1, (1, 2, 4, 8), 64, 3000, rate_lo=50.0, rate_hi=900.0)
+    r = oracle_mod.solve_batch(wl, horizontal=True)
+    for n in range(wl.n_instances):
+        if r["status"][n]:
+            continue
+        for s in range(wl.n_stages):
+            h, b = int(r["h"][n][s]), int(r["b"][n][s])
+            l_us = int(wl.lat_us[n][s][0][wl.batch_sizes.index(b)])
+            lam = int(wl.lambda_mrps[n])
+            assert h * b * 10 ** 9 >= lam * l_us
+            assert h == 1 or (h - 1) * b * 10 ** 9 < lam * l_us
