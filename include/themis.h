@@ -69,6 +69,8 @@ extern "C" {
 /* per-instance status */
 #define THEMIS_STATUS_OK 0
 #define THEMIS_STATUS_INFEASIBLE 1
+#define THEMIS_STATUS_SPLIT 2          /* themis_vertical_fallback_batch: part of the load is served
+                                          by the replicas in place, the rest needs extra replicas */
 #define THEMIS_STATUS_BAD_INPUT (-1)   /* lambda = 0, a latency <= 0 or replicas < 1 */
 #define THEMIS_STATUS_TIMEOUT (-2)     /* a bounded on-device wait expired */
 
@@ -147,6 +149,40 @@ int themis_solve_vertical_batch(const themis_problem_t *problem, const int32_t *
                                 const int32_t *d_profile_id, const uint32_t *d_lambda_mrps,
                                 const int32_t *d_replicas, themis_result_t out,
                                 void *d_workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Vertical solver with Algorithm 1's last branch.  Instances for which the
+ * replicas in place cannot serve lambda within the SLO at any core count are
+ * split: a bisection on the arrival rate finds a rate lambda_vertical that
+ * vertical scaling still serves, and the rest of the load is given to extra
+ * replicas with the cores and batch size just chosen,
+ *     extra[n][s] = ceil((lambda - lambda_vertical) / thr_s(b_s, c_s)).
+ * Search points are multiples k * resolution_mrps: lo = 0, hi = ceil(lambda /
+ * resolution); while hi - lo > 1: mid = (lo + hi) / 2, served at mid * resolution ?
+ * lo = mid : hi = mid (the printed loop's midpoint and branch are garbled; this is
+ * the reading taken).  Feasibility is not monotone in the rate in general, so, as
+ * in the paper, the result is a served rate whose next search point is not served,
+ * not necessarily the largest such rate.
+ *   lambda_max_mrps      host-side upper bound on every d_lambda_mrps[n]; fixes the
+ *                        number of bisection rounds, ceil(log2(ceil(max / resolution))),
+ *                        without reading the device.  An instance above the bound
+ *                        that needs the search gets THEMIS_STATUS_BAD_INPUT.
+ *   d_lambda_vertical    [N] uint32 out: lambda where the instance is feasible as it
+ *                        is, else the served rate found (0 if not even `resolution`
+ *                        is served: status stays THEMIS_STATUS_INFEASIBLE)
+ *   d_extra_replicas     [N][S] int32 out: 0 except for THEMIS_STATUS_SPLIT instances
+ *   out                  the vertical part's configuration (for split instances: the
+ *                        solve at lambda_vertical), status in {0, 1, 2, < 0}
+ * Every round re-solves only the instances still searching.  Workspace:
+ * themis_fallback_workspace_bytes.
+ */
+int themis_fallback_workspace_bytes(const themis_problem_t *problem, size_t *out_bytes);
+int themis_vertical_fallback_batch(const themis_problem_t *problem, const int32_t *d_lat_us,
+                                   const int32_t *d_profile_id, const uint32_t *d_lambda_mrps,
+                                   const int32_t *d_replicas, uint32_t resolution_mrps,
+                                   uint32_t lambda_max_mrps, themis_result_t out,
+                                   uint32_t *d_lambda_vertical, int32_t *d_extra_replicas,
+                                   void *d_workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * Horizontal-only variant (Algorithm 2): one-core replicas.  problem->c_max must

@@ -62,6 +62,8 @@ def _load():
         lib.oracle_minplus.argtypes = [ctypes.c_int32, vp, vp, vp, vp]
         lib.oracle_solve_horizontal_batch.restype = ctypes.c_int
         lib.oracle_solve_horizontal_batch.argtypes = [P] + [vp] * 13 + [ctypes.c_int]
+        lib.oracle_vertical_fallback_batch.restype = ctypes.c_int
+        lib.oracle_vertical_fallback_batch.argtypes = [P, vp, vp, vp, vp, ctypes.c_uint32] + [vp] * 8 + [ctypes.c_int]
         for fn in (lib.oracle_alg1_scatter, lib.oracle_alg2_scatter, lib.brute_force_instance):
             fn.restype = ctypes.c_int
             fn.argtypes = [P, vp, ctypes.c_uint32, vp, vp, vp, vp, vp, vp]
@@ -126,6 +128,31 @@ def solve_batch(wl, dumps: bool = False, n_threads: int = 0, horizontal: bool = 
         rc = lib.oracle_solve_batch(ctypes.byref(p), _ptr(lat), _ptr(pid), _ptr(lam), _ptr(rep), *tail)
     if rc < 0:
         raise MemoryError("oracle_solve_batch: allocation failed or unsupported problem")
+    out["threads"] = rc
+    return out
+
+
+def vertical_fallback_batch(wl, resolution_mrps: int = 1000, n_threads: int = 0) -> dict:
+    """Algorithm 1 with its last branch: instances the replicas in place cannot
+    serve are split into the largest rate found by bisection that vertical
+    scaling serves plus extra replicas for the rest.  Returns the arrays of
+    ``solve_batch`` (status 2 = split) plus ``lambda_vertical`` [N] and
+    ``extra_replicas`` [N][S]."""
+    lib = _load()
+    N, S = wl.n_instances, wl.n_stages
+    p = _problem_of(wl)
+    lat, pid = _c(wl.lat_us, np.int32), _c(wl.profile_id, np.int32)
+    lam, rep = _c(wl.lambda_mrps, np.uint32), _c(wl.replicas, np.int32)
+    out = {k: np.zeros((N, S), np.int32) for k in ("h", "c", "b", "extra_replicas")}
+    out.update({k: np.zeros(N, np.int32) for k in ("total_cost", "latency_buckets", "status")})
+    out["lambda_vertical"] = np.zeros(N, np.uint32)
+    rc = lib.oracle_vertical_fallback_batch(
+        ctypes.byref(p), _ptr(lat), _ptr(pid), _ptr(lam), _ptr(rep), int(resolution_mrps),
+        _ptr(out["h"]), _ptr(out["c"]), _ptr(out["b"]), _ptr(out["total_cost"]),
+        _ptr(out["latency_buckets"]), _ptr(out["status"]), _ptr(out["lambda_vertical"]),
+        _ptr(out["extra_replicas"]), int(n_threads))
+    if rc < 0:
+        raise RuntimeError("oracle_vertical_fallback_batch failed")
     out["threads"] = rc
     return out
 

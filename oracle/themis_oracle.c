@@ -331,6 +331,98 @@ int oracle_solve_horizontal_batch(const oracle_problem *p, const int32_t *lat_us
 }
 
 /*
+ * Algorithm 1's last branch, batch form.  When the replicas in place cannot serve
+ * lambda within the SLO at any core count, the paper bisects on the workload for
+ * the largest rate that vertical scaling still serves and brings up extra replicas,
+ * with the cores and batch size just chosen, for the rest.  Reading taken of the
+ * printed loop (whose midpoint and branch sense are garbled): search points are
+ * multiples k * resolution; lo = 0 (nothing served), hi = ceil(lambda / resolution)
+ * (known not to be served); while hi - lo > 1: mid = (lo + hi) / 2, served at
+ * mid * resolution ? lo = mid : hi = mid.  Feasibility is not monotone in the rate
+ * in general (queuing delay shrinks as the rate grows), so this is the paper's
+ * heuristic, not a maximum: the result is a rate that is served whose successor
+ * search point is not.
+ *   lambda_vertical[n] = lo * resolution (lambda itself if the instance is feasible;
+ *                        0 if no search point is served: status stays 1)
+ *   extra[n][s]        = ceil((lambda - lambda_vertical) / thr_s(b_s, c_s)) replicas
+ *   status             = 0 feasible as is, 2 split into vertical + extra replicas,
+ *                        1 not even the lowest search point is served
+ * h, c, b, total_cost, latency_buckets describe the vertical part.
+ */
+int oracle_vertical_fallback_batch(const oracle_problem *p, const int32_t *lat_us, const int32_t *profile_id,
+                                   const uint32_t *lambda_mrps, const int32_t *replicas, uint32_t resolution,
+                                   int32_t *h, int32_t *c, int32_t *b,
+                                   int32_t *total_cost, int32_t *latency_buckets, int32_t *status,
+                                   uint32_t *lambda_vertical, int32_t *extra, int n_threads)
+{
+    const int32_t N = p->n_instances, S = p->n_stages;
+    const size_t W = (size_t)(p->slo_us / p->bucket_us) + 1;
+    const size_t rows = (size_t)S * W;
+    const size_t pipeline_words = (size_t)S * p->c_max * p->n_batch;
+    int used = 1, failed = 0;
+    if (resolution < 1 || !replicas) return -1;
+#ifdef _OPENMP
+    if (n_threads <= 0) n_threads = omp_get_max_threads();
+    used = n_threads;
+#pragma omp parallel num_threads(n_threads)
+#endif
+    {
+        int32_t *Gs = (int32_t *)malloc(sizeof(int32_t) * rows);
+        int32_t *Fs = (int32_t *)malloc(sizeof(int32_t) * rows);
+        uint16_t *Gargs = (uint16_t *)malloc(sizeof(uint16_t) * rows);
+        uint16_t *As = (uint16_t *)malloc(sizeof(uint16_t) * rows);
+        if (!Gs || !Fs || !Gargs || !As) {
+#ifdef _OPENMP
+#pragma omp atomic write
+#endif
+            failed = 1;
+        } else {
+#ifdef _OPENMP
+#pragma omp for schedule(dynamic, 1)
+#endif
+            for (int32_t n = 0; n < N; ++n) {
+                const int32_t *lat = lat_us + (size_t)(profile_id ? profile_id[n] : 0) * pipeline_words;
+                const int32_t *rep = replicas + (size_t)n * S;
+                int32_t *hn = h + (size_t)n * S, *cn = c + (size_t)n * S, *bn = b + (size_t)n * S;
+                int32_t *en = extra + (size_t)n * S;
+                const uint32_t lam = lambda_mrps[n];
+                for (int32_t s = 0; s < S; ++s) en[s] = 0;
+                int st = solve_instance(p, lat, lam, rep, 0, hn, cn, bn, &total_cost[n], &latency_buckets[n],
+                                        Gs, Gargs, Fs, As);
+                lambda_vertical[n] = lam;
+                status[n] = st;
+                if (st == 0) continue;
+                uint64_t lo = 0, hi = ((uint64_t)lam + resolution - 1) / resolution;
+                while (hi - lo > 1) {
+                    uint64_t mid = (lo + hi) / 2;
+                    int served = solve_instance(p, lat, (uint32_t)(mid * resolution), rep, 0, hn, cn, bn,
+                                                &total_cost[n], &latency_buckets[n], Gs, Gargs, Fs, As) == 0;
+                    if (served) lo = mid; else hi = mid;
+                }
+                lambda_vertical[n] = (uint32_t)(lo * resolution);
+                if (lo == 0) {       /* leave the "no configuration" result of the last trial */
+                    solve_instance(p, lat, lam, rep, 0, hn, cn, bn, &total_cost[n], &latency_buckets[n],
+                                   Gs, Gargs, Fs, As);
+                    continue;
+                }
+                solve_instance(p, lat, lambda_vertical[n], rep, 0, hn, cn, bn, &total_cost[n],
+                               &latency_buckets[n], Gs, Gargs, Fs, As);
+                status[n] = 2;
+                const uint64_t rest = (uint64_t)lam - lambda_vertical[n];
+                for (int32_t s = 0; s < S; ++s) {
+                    int32_t bi = 0;
+                    while (p->batch_sizes[bi] != bn[s]) ++bi;
+                    uint64_t l_us = (uint64_t)lat[((size_t)s * p->c_max + (cn[s] - 1)) * p->n_batch + bi];
+                    en[s] = (int32_t)ceil_div_u64(rest * l_us, (uint64_t)bn[s] * 1000000000ull);
+                }
+            }
+        }
+        free(Gs); free(Fs); free(Gargs); free(As);
+    }
+    return failed ? -1 : used;
+}
+
+/*
  * Algorithm 2 in the paper's loop order, one instance: as oracle_alg1_scatter, with
  * the candidate loop over batch sizes only and the replica count computed per
  * candidate.  lat_pipeline is [S][1][n_batch].

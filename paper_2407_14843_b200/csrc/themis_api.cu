@@ -13,6 +13,7 @@ thread_local cudaError_t t_last_cuda = cudaSuccess;
 thread_local char t_msg[256];
 int g_tile = 0;   // min-plus cells per thread; 0 = built-in choice
 thread_local bool g_horizontal = false;   // set by solve_impl for the launches it makes
+thread_local const int32_t *g_active = nullptr;   // per-instance mask for the launches of one solve
 int g_mode = 0;   // 0: packed 16-bit min-plus kernel with 32-bit second pass; 1: 32-bit kernel only
 
 constexpr size_t kAlign = 256;
@@ -90,6 +91,7 @@ int make_params(const themis_problem_t *pr, int vertical, void *ws, size_t ws_by
     P->vertical = vertical ? 1 : 0;
     P->K = (vertical ? 1 : pr->h_max) * pr->c_max * pr->n_batch;
     P->horizontal = (!vertical && g_horizontal) ? 1 : 0;
+    P->active = g_active;
     char *base = static_cast<char *>(ws);
     P->G = reinterpret_cast<int32_t *>(base + L.g_offset);
     P->Garg = reinterpret_cast<uint16_t *>(base + L.garg_offset);
@@ -155,6 +157,29 @@ int solve_impl(const themis_problem_t *pr, const int32_t *lat, const int32_t *pi
     if (rc == THEMIS_OK) rc = minplus_impl(pr, rep, vertical, out, ws, ws_bytes, st);
     g_horizontal = false;
     return rc;
+}
+
+// Search state and trial results appended to the solver workspace by the fallback entry point.
+struct FallbackStage {
+    size_t lo, hi, active, iter_active, trial_lambda, h, c, b, cost, latb, status, total;
+};
+
+void fallback_stage_of(const themis_problem_t *pr, size_t base, FallbackStage *F)
+{
+    const size_t N = pr->n_instances, S = pr->n_stages;
+    size_t off = align_up(base);
+    F->lo = off; off = align_up(off + N * 4);
+    F->hi = off; off = align_up(off + N * 4);
+    F->active = off; off = align_up(off + N * 4);
+    F->iter_active = off; off = align_up(off + N * 4);
+    F->trial_lambda = off; off = align_up(off + N * 4);
+    F->h = off; off = align_up(off + N * S * 4);
+    F->c = off; off = align_up(off + N * S * 4);
+    F->b = off; off = align_up(off + N * S * 4);
+    F->cost = off; off = align_up(off + N * 4);
+    F->latb = off; off = align_up(off + N * 4);
+    F->status = off; off = align_up(off + N * 4);
+    F->total = off;
 }
 
 // Staging area appended to the solver workspace by the host-buffer variant.
@@ -265,6 +290,88 @@ int themis_solve_vertical_batch(const themis_problem_t *problem, const int32_t *
     if (!d_replicas) return THEMIS_E_INVALID_ARG;
     return solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, d_replicas, 1, out, d_workspace,
                       workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int themis_fallback_workspace_bytes(const themis_problem_t *problem, size_t *out_bytes)
+{
+    if (!out_bytes) return THEMIS_E_INVALID_ARG;
+    themis_workspace_layout_t L;
+    int rc = layout_of(problem, 1, &L);
+    if (rc != THEMIS_OK) return rc;
+    FallbackStage F;
+    fallback_stage_of(problem, L.total_bytes, &F);
+    *out_bytes = F.total;
+    return THEMIS_OK;
+}
+
+int themis_vertical_fallback_batch(const themis_problem_t *problem, const int32_t *d_lat_us,
+                                   const int32_t *d_profile_id, const uint32_t *d_lambda_mrps,
+                                   const int32_t *d_replicas, uint32_t resolution_mrps,
+                                   uint32_t lambda_max_mrps, themis_result_t out,
+                                   uint32_t *d_lambda_vertical, int32_t *d_extra_replicas,
+                                   void *d_workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    themis_workspace_layout_t L;
+    int rc = layout_of(problem, 1, &L);
+    if (rc != THEMIS_OK) return rc;
+    if (!d_replicas || !d_lambda_vertical || !d_extra_replicas || !result_ok(out) || !d_lat_us || !d_lambda_mrps ||
+        resolution_mrps < 1 || lambda_max_mrps < 1)
+        return THEMIS_E_INVALID_ARG;
+    if (!d_workspace || ((uintptr_t)d_workspace & (kAlign - 1))) return THEMIS_E_INVALID_ARG;
+    FallbackStage F;
+    fallback_stage_of(problem, L.total_bytes, &F);
+    if (workspace_bytes < F.total) return THEMIS_E_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char *base = static_cast<char *>(d_workspace);
+    const int N = problem->n_instances;
+    uint32_t *lo = reinterpret_cast<uint32_t *>(base + F.lo), *hi = reinterpret_cast<uint32_t *>(base + F.hi);
+    int32_t *active = reinterpret_cast<int32_t *>(base + F.active);
+    int32_t *iter_active = reinterpret_cast<int32_t *>(base + F.iter_active);
+    uint32_t *trial_lambda = reinterpret_cast<uint32_t *>(base + F.trial_lambda);
+    themis_result_t trial;
+    trial.h = reinterpret_cast<int32_t *>(base + F.h);
+    trial.c = reinterpret_cast<int32_t *>(base + F.c);
+    trial.b = reinterpret_cast<int32_t *>(base + F.b);
+    trial.total_cost = reinterpret_cast<int32_t *>(base + F.cost);
+    trial.latency_buckets = reinterpret_cast<int32_t *>(base + F.latb);
+    trial.status = reinterpret_cast<int32_t *>(base + F.status);
+
+    // 1. the whole load on the replicas in place
+    rc = solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, d_replicas, 1, out, d_workspace,
+                    L.total_bytes, st);
+    if (rc != THEMIS_OK) return rc;
+    cudaError_t e = launch_fb_init(N, resolution_mrps, out.status, d_lambda_mrps, lo, hi, active, st);
+    if (e != cudaSuccess) return fail_cuda(e);
+    // 2. bisection rounds: enough to close an interval of ceil(max / resolution) points
+    const unsigned long long points = ((unsigned long long)lambda_max_mrps + resolution_mrps - 1) / resolution_mrps;
+    int rounds = 0;
+    while ((1ull << rounds) < points) ++rounds;
+    for (int r = 0; r < rounds; ++r) {
+        e = launch_fb_trial(N, resolution_mrps, lo, hi, active, iter_active, trial_lambda, st);
+        if (e != cudaSuccess) return fail_cuda(e);
+        g_active = iter_active;
+        rc = solve_impl(problem, d_lat_us, d_profile_id, trial_lambda, d_replicas, 1, trial, d_workspace,
+                        L.total_bytes, st);
+        g_active = nullptr;
+        if (rc != THEMIS_OK) return rc;
+        e = launch_fb_update(N, lo, hi, iter_active, trial.status, st);
+        if (e != cudaSuccess) return fail_cuda(e);
+    }
+    // 3. the vertical part at the rate found, straight into the caller's arrays
+    e = launch_fb_final_trial(N, resolution_mrps, lo, active, iter_active, trial_lambda, st);
+    if (e != cudaSuccess) return fail_cuda(e);
+    g_active = iter_active;
+    rc = solve_impl(problem, d_lat_us, d_profile_id, trial_lambda, d_replicas, 1, out, d_workspace, L.total_bytes, st);
+    g_active = nullptr;
+    if (rc != THEMIS_OK) return rc;
+    // 4. the rest of the load on extra replicas
+    Params P;
+    rc = make_params(problem, 1, d_workspace, L.total_bytes, &P);
+    if (rc != THEMIS_OK) return rc;
+    P.lat_us = d_lat_us; P.profile_id = d_profile_id; P.lambda_mrps = d_lambda_mrps; P.replicas = d_replicas;
+    P.out = out;
+    e = launch_fb_finish(P, resolution_mrps, lo, hi, active, d_lambda_vertical, d_extra_replicas, st);
+    return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
 }
 
 int themis_solve_horizontal_batch(const themis_problem_t *problem, const int32_t *d_lat_us,

@@ -45,6 +45,7 @@ struct Params {
     const int32_t *profile_id;
     const uint32_t *lambda_mrps;
     const int32_t *replicas;
+    const int32_t *active;   // [N] or NULL: blocks of instances with active[n] == 0 leave at once
     int32_t *G;
     uint16_t *Garg;
     uint16_t *A;
@@ -74,6 +75,16 @@ inline void assign_warp_groups(int n_warps, uint8_t *warp_group)
 cudaError_t launch_score(const Params &p, cudaStream_t stream);
 cudaError_t launch_minplus(const Params &p, int tile, cudaStream_t stream);
 cudaError_t launch_minplus16(const Params &p, int tile, cudaStream_t stream);
+cudaError_t launch_fb_init(int N, uint32_t res, const int32_t *status, const uint32_t *lambda, uint32_t *lo,
+                           uint32_t *hi, int32_t *active, cudaStream_t st);
+cudaError_t launch_fb_trial(int N, uint32_t res, const uint32_t *lo, const uint32_t *hi, const int32_t *active,
+                            int32_t *iter_active, uint32_t *trial_lambda, cudaStream_t st);
+cudaError_t launch_fb_update(int N, uint32_t *lo, uint32_t *hi, const int32_t *iter_active,
+                             const int32_t *trial_status, cudaStream_t st);
+cudaError_t launch_fb_final_trial(int N, uint32_t res, const uint32_t *lo, const int32_t *active,
+                                  int32_t *iter_active, uint32_t *trial_lambda, cudaStream_t st);
+cudaError_t launch_fb_finish(const Params &p, uint32_t res, const uint32_t *lo, const uint32_t *hi,
+                             const int32_t *active, uint32_t *lambda_vertical, int32_t *extra, cudaStream_t st);
 cudaError_t launch_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *sink,
                              cudaStream_t stream);
 

@@ -70,6 +70,7 @@ minplus_kernel(const Params p)
     extern __shared__ __align__(128) uint32_t smem[];
     constexpr int CS = Tile<R>::kChunkStride;
     const int n = blockIdx.x;
+    if (p.active && !p.active[n]) return;
     const int tid = threadIdx.x;
     const int NT = blockDim.x;
     const int T = p.T, pitch = p.pitch, S = p.prob.n_stages;

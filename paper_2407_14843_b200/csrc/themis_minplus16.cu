@@ -95,6 +95,7 @@ minplus16_kernel(const Params p)
     constexpr int H = Tile16<R>::H, CS = Tile16<R>::CS;
     constexpr int U = R == 8 ? 4 : 2;                     // chunk steps per loop iteration
     const int n = blockIdx.x;
+    if (p.active && !p.active[n]) return;
     const int tid = threadIdx.x;
     const int NT = blockDim.x;
     const int n_warps = NT >> 5;

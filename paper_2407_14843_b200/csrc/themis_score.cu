@@ -36,6 +36,7 @@ score_kernel(const Params p)
 {
     extern __shared__ __align__(16) uint32_t smem[];
     const int n = blockIdx.x;
+    if (p.active && !p.active[n]) return;
     const int tid = threadIdx.x;
     const int T = p.T, pitch = p.pitch;
     const int S = p.prob.n_stages, C = p.prob.c_max, NB = p.prob.n_batch;

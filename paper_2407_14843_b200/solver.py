@@ -23,6 +23,7 @@ OK, E_INVALID_ARG, E_UNSUPPORTED_SIZE, E_WORKSPACE_TOO_SMALL, E_CUDA = 0, -1, -2
 E_STATIC_SCRATCH_EXCEEDED = -5
 STATIC_SCRATCH_BYTES = 32 << 20
 STATUS_OK, STATUS_INFEASIBLE, STATUS_BAD_INPUT, STATUS_TIMEOUT = 0, 1, -1, -2
+STATUS_SPLIT = 2
 G_INF = 2 ** 31 - 1
 MAX_T = 16383
 INF16 = 0x7FFF
@@ -32,7 +33,7 @@ EXPORTS = (
     "themis_solve_batch", "themis_solve_vertical_batch", "themis_score_batch", "themis_minplus_batch",
     "themis_host_workspace_bytes", "themis_solve_batch_host", "themis_alu_probe",
     "themis_set_minplus_tile", "themis_solve_batch_static", "themis_set_minplus_mode",
-    "themis_solve_horizontal_batch",
+    "themis_solve_horizontal_batch", "themis_fallback_workspace_bytes", "themis_vertical_fallback_batch",
 )
 
 
@@ -96,6 +97,9 @@ def _load() -> ctypes.CDLL:
     lib.themis_workspace_layout.argtypes = [PP, ctypes.c_int, ctypes.POINTER(WorkspaceLayout)]
     lib.themis_solve_batch.argtypes = [PP, vp, vp, vp, Result, vp, sz, vp]
     lib.themis_solve_vertical_batch.argtypes = [PP, vp, vp, vp, vp, Result, vp, sz, vp]
+    lib.themis_fallback_workspace_bytes.argtypes = [PP, ctypes.POINTER(sz)]
+    lib.themis_vertical_fallback_batch.argtypes = [PP, vp, vp, vp, vp, ctypes.c_uint32, ctypes.c_uint32, Result,
+                                                   vp, vp, vp, sz, vp]
     lib.themis_solve_horizontal_batch.argtypes = [PP, vp, vp, vp, Result, vp, sz, vp]
     lib.themis_score_batch.argtypes = [PP, vp, vp, vp, vp, vp, sz, vp]
     lib.themis_minplus_batch.argtypes = [PP, vp, Result, vp, sz, vp]
@@ -179,6 +183,24 @@ def themis_solve_vertical_batch(problem: Problem, lat_us, profile_id, lambda_mrp
         ctypes.byref(problem), _dptr(lat_us, torch.int32, "lat_us"), _dptr(profile_id, torch.int32, "profile_id"),
         _dptr(lambda_mrps, torch.uint32, "lambda_mrps"), _dptr(replicas, torch.int32, "replicas"), _result(out),
         _dptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()), "themis_solve_vertical_batch")
+
+
+def themis_fallback_workspace_bytes(problem: Problem) -> int:
+    n = ctypes.c_size_t()
+    _check(_lib.themis_fallback_workspace_bytes(ctypes.byref(problem), ctypes.byref(n)),
+           "themis_fallback_workspace_bytes")
+    return n.value
+
+
+def themis_vertical_fallback_batch(problem: Problem, lat_us, profile_id, lambda_mrps, replicas,
+                                   resolution_mrps: int, lambda_max_mrps: int, out: dict,
+                                   lambda_vertical, extra_replicas, workspace) -> None:
+    _check(_lib.themis_vertical_fallback_batch(
+        ctypes.byref(problem), _dptr(lat_us, torch.int32, "lat_us"), _dptr(profile_id, torch.int32, "profile_id"),
+        _dptr(lambda_mrps, torch.uint32, "lambda_mrps"), _dptr(replicas, torch.int32, "replicas"),
+        int(resolution_mrps), int(lambda_max_mrps), _result(out),
+        _dptr(lambda_vertical, torch.uint32, "lambda_vertical"), _dptr(extra_replicas, torch.int32, "extra_replicas"),
+        _dptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()), "themis_vertical_fallback_batch")
 
 
 def themis_solve_horizontal_batch(problem: Problem, lat_us, profile_id, lambda_mrps, out: dict, workspace) -> None:

@@ -186,6 +186,36 @@ def test_horizontal_only_solver(S, oracle_mod, flags, mode):
         == S.E_INVALID_ARG
 
 
+@pytest.mark.parametrize("res", [1000, 25000])
+def test_vertical_fallback(S, oracle_mod, res, mode):
+    """Algorithm 1 with its last branch (bisection on the rate + extra replicas):
+    every output against the oracle, on trace seconds around the largest spikes."""
+    import torch
+    from tests.test_oracle_pins import _spiky_vertical_workload
+    wl = _spiky_vertical_workload(40)
+    ref = oracle_mod.vertical_fallback_batch(wl, res)
+    assert (ref["status"] == 2).any() and (ref["status"] == 0).any()
+    prob = S.Problem.of_workload(wl)
+    dev = S.workload_to_device(wl)
+    ws = torch.empty(S.themis_fallback_workspace_bytes(prob), dtype=torch.uint8, device="cuda")
+    out = S.alloc_result(wl.n_instances, wl.n_stages)
+    lam_v = torch.empty(wl.n_instances, dtype=torch.uint32, device="cuda")
+    extra = torch.empty((wl.n_instances, wl.n_stages), dtype=torch.int32, device="cuda")
+    S.themis_vertical_fallback_batch(prob, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"], dev["replicas"],
+                                     res, int(wl.lambda_mrps.max()), out, lam_v, extra, ws)
+    torch.cuda.synchronize()
+    gpu = {k: v.cpu().numpy() for k, v in out.items()}
+    _assert_results_equal(gpu, ref)
+    assert np.array_equal(lam_v.cpu().numpy(), ref["lambda_vertical"])
+    assert np.array_equal(extra.cpu().numpy(), ref["extra_replicas"])
+    # a bound on lambda that is too low is reported, not silently wrong
+    S.themis_vertical_fallback_batch(prob, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"], dev["replicas"],
+                                     res, 4 * res, out, lam_v, extra, ws)
+    torch.cuda.synchronize()
+    st = out["status"].cpu().numpy()
+    assert (st[ref["status"] == 2] == S.STATUS_BAD_INPUT).all() and (st[ref["status"] == 0] == 0).all()
+
+
 # ---------------------------------------------------------------- edge cases
 
 @pytest.mark.parametrize("T", [1, 2, 31, 32, 33, 255, 256, 257, 511, 2047, 2048, 2049])

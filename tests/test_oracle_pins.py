@@ -388,3 +388,61 @@ def test_horizontal_replica_counts_are_tight(oracle_mod):
             lam = int(wl.lambda_mrps[n])
             assert h * b * 10 ** 9 >= lam * l_us
             assert h == 1 or (h - 1) * b * 10 ** 9 < lam * l_us
+
+
+# ---------------------------------------------------------------- Algorithm 1's last branch
+
+def _spiky_vertical_workload(n_hot=24):
+    """Seconds of the day-long trace around its largest spikes plus quiet ones."""
+    full = W.make_workload(3)
+    hot = np.argsort(full.lambda_mrps)[-n_hot:]
+    pick = np.unique(np.concatenate([hot, np.arange(0, full.n_instances, 7200)]))
+    return dataclasses.replace(full, n_instances=len(pick), profile_id=full.profile_id[pick].copy(),
+                               lambda_mrps=full.lambda_mrps[pick].copy(), replicas=full.replicas[pick].copy())
+
+
+def test_vertical_fallback_invariants(oracle_mod):
+    """Where the replicas in place cannot serve the load: the rate found is
+    served, the next search point is not, the extra replicas carry exactly the
+    rest (one fewer would not), and feasible instances are left alone."""
+    wl = _spiky_vertical_workload()
+    res = 1000
+    r = oracle_mod.vertical_fallback_batch(wl, res)
+    plain = oracle_mod.solve_batch(wl)
+    split = r["status"] == 2
+    assert split.any() and (r["status"] == 0).any()
+    assert np.array_equal(r["status"] == 0, plain["status"] == 0)
+    keep = plain["status"] == 0
+    for k in ("h", "c", "b", "total_cost", "latency_buckets"):
+        assert np.array_equal(r[k][keep], plain[k][keep])
+    assert np.array_equal(r["lambda_vertical"][keep], wl.lambda_mrps[keep]) and not r["extra_replicas"][keep].any()
+    lv = r["lambda_vertical"]
+    assert (lv[split] % res == 0).all() and (lv[split] > 0).all() and (lv[split] < wl.lambda_mrps[split]).all()
+    at = oracle_mod.solve_batch(dataclasses.replace(wl, lambda_mrps=np.where(split, lv, wl.lambda_mrps).astype(np.uint32)))
+    above = oracle_mod.solve_batch(dataclasses.replace(
+        wl, lambda_mrps=np.where(split, np.minimum(lv + res, wl.lambda_mrps), wl.lambda_mrps).astype(np.uint32)))
+    assert (at["status"][split] == 0).all() and (above["status"][split] == 1).all()
+    for k in ("h", "c", "b", "total_cost", "latency_buckets"):
+        assert np.array_equal(r[k][split], at[k][split])
+    for n in np.flatnonzero(split):
+        rest = int(wl.lambda_mrps[n]) - int(lv[n])
+        for s in range(wl.n_stages):
+            c, b, e = int(r["c"][n][s]), int(r["b"][n][s]), int(r["extra_replicas"][n][s])
+            l_us = int(wl.lat_us[0][s][c - 1][wl.batch_sizes.index(b)])
+            assert e * b * 10 ** 9 >= rest * l_us and (e - 1) * b * 10 ** 9 < rest * l_us
+
+
+def test_vertical_fallback_finds_the_maximum_when_feasibility_is_monotone(oracle_mod):
+    """Batch size 1 only (no queuing term): feasibility is monotone in the rate, so
+    the bisection result is the largest served multiple of the resolution, which a
+    linear scan over every search point confirms."""
+    base = W.random_tiny_workload(7400, 10, 2, 4, (1,), 3, 60, vertical=True, rate_lo=150.0, rate_hi=400.0)
+    res = 5000
+    r = oracle_mod.vertical_fallback_batch(base, res)
+    assert (r["status"] == 2).any()
+    for n in np.flatnonzero(r["status"] != 0):
+        one = base.take(1, int(n))
+        served = [k for k in range(1, int(base.lambda_mrps[n]) // res + 1)
+                  if oracle_mod.solve_batch(dataclasses.replace(one, lambda_mrps=np.asarray([k * res], np.uint32)))["status"][0] == 0]
+        assert int(r["lambda_vertical"][n]) == (max(served) * res if served else 0)
+        assert (r["status"][n] == 2) == bool(served)
