@@ -109,6 +109,10 @@ score_kernel(const Params p)
                 const int pair = (c - 1) * NB + bi;
                 const int32_t l_us = lat_s[pair];
                 if (l_us <= 0) { saw_bad_latency = 1; continue; }
+                // Same latency with one core fewer: that candidate reaches the same buckets with
+                // the same replica counts at a lower cost, so this one can never be a minimum
+                // (latency tables are flat over long runs of core counts).
+                if (c > 1 && lat_s[pair - NB] == l_us) continue;
                 // l_b = ceil(l_us / w): quotient estimate by the precomputed reciprocal, then fix up
                 uint32_t l_q = __umulhi((uint32_t)l_us, w_magic);
                 uint32_t l_r = (uint32_t)l_us - l_q * w_us;

@@ -446,3 +446,25 @@ def test_vertical_fallback_finds_the_maximum_when_feasibility_is_monotone(oracle
                   if oracle_mod.solve_batch(dataclasses.replace(one, lambda_mrps=np.asarray([k * res], np.uint32)))["status"][0] == 0]
         assert int(r["lambda_vertical"][n]) == (max(served) * res if served else 0)
         assert (r["status"][n] == 2) == bool(served)
+
+
+def test_full_queue_model_reduces_to_the_simplified_one():
+    """Eq. 3, q = max((b-1)/lambda, l(b,c) - (n*b+1)/lambda): for every candidate
+    that satisfies the throughput constraint of Eq. 6 the second term is negative,
+    so the solver's queue model (Eq. 4) is Eq. 3 on the feasible set."""
+    from fractions import Fraction
+    wl = W.make_workload(2, 16)
+    checked = 0
+    for n in range(0, 16, 5):
+        lam = Fraction(int(wl.lambda_mrps[n]), 1000)
+        for s in range(wl.n_stages):
+            for h in range(1, wl.h_max + 1, 3):
+                for c in range(1, wl.c_max + 1, 5):
+                    for bi, b in enumerate(wl.batch_sizes):
+                        l = Fraction(int(wl.lat_us[wl.profile_id[n]][s][c - 1][bi]), 1_000_000)
+                        if h * Fraction(b) / l >= lam:
+                            second = l - Fraction(h * b + 1) / lam
+                            assert second < 0
+                            assert max(Fraction(b - 1) / lam, second) == Fraction(b - 1) / lam
+                            checked += 1
+    assert checked > 500
