@@ -283,7 +283,13 @@ int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_s
  *      0x7FFF = unreachable or >= 32767, and the backtrack recovers the argmin
  *      along the optimal path only.  Instances whose optimum does not fit 16
  *      bits are redone by the 32-bit kernel in a second launch.
- *   1: 32-bit kernel only; the A rows hold the argmin tables described above. */
+ *   1: 32-bit kernel only; the A rows hold the argmin tables described above.
+ *   2: recurrence restricted to the undominated entries of every G_s (an entry is
+ *      dominated when a smaller l has a cost at most as high; such entries never
+ *      occur in the returned solution).  Returned configurations, costs, latencies
+ *      and statuses are identical to modes 0 and 1 at a small fraction of the work;
+ *      the A and F tables are those of the restricted problem.  Budgets above about
+ *      11000 buckets run mode 0 instead. */
 int themis_set_minplus_mode(int mode);
 
 /* Tuning knob of the min-plus kernel: consecutive budget cells per thread

@@ -14,7 +14,8 @@ thread_local char t_msg[256];
 int g_tile = 0;   // min-plus cells per thread; 0 = built-in choice
 thread_local bool g_horizontal = false;   // set by solve_impl for the launches it makes
 thread_local const int32_t *g_active = nullptr;   // per-instance mask for the launches of one solve
-int g_mode = 0;   // 0: packed 16-bit min-plus kernel with 32-bit second pass; 1: 32-bit kernel only
+int g_mode = 0;   // 0: packed 16-bit dense kernel with 32-bit second pass; 1: 32-bit dense kernel;
+                  // 2: recurrence over undominated entries only (dense packed kernel above 11000 buckets)
 
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
@@ -129,6 +130,8 @@ int minplus_impl(const themis_problem_t *pr, const int32_t *rep, int vertical, t
     cudaError_t e;
     if (g_mode == 1) {
         e = launch_minplus(P, g_tile, st);
+    } else if (g_mode == 2 && pruned_smem_bytes(P.pitch) <= 227u * 1024u) {
+        e = launch_minplus_pruned(P, st);
     } else {
         e = launch_minplus16(P, g_tile, st);
         // A total can only reach the 16-bit saturation value if the static bound allows it
@@ -488,7 +491,7 @@ int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_s
 
 int themis_set_minplus_mode(int mode)
 {
-    if (mode != 0 && mode != 1) return THEMIS_E_INVALID_ARG;
+    if (mode < 0 || mode > 2) return THEMIS_E_INVALID_ARG;
     g_mode = mode;
     return THEMIS_OK;
 }

@@ -75,6 +75,9 @@ inline void assign_warp_groups(int n_warps, uint8_t *warp_group)
 cudaError_t launch_score(const Params &p, cudaStream_t stream);
 cudaError_t launch_minplus(const Params &p, int tile, cudaStream_t stream);
 cudaError_t launch_minplus16(const Params &p, int tile, cudaStream_t stream);
+cudaError_t launch_minplus_pruned(const Params &p, cudaStream_t stream);
+// Dynamic shared memory of the pruned kernel for a row pitch; it cannot run above 227 KB.
+inline size_t pruned_smem_bytes(int pitch) { return sizeof(uint32_t) * (5u * (size_t)pitch + 4 + 32); }
 cudaError_t launch_fb_init(int N, uint32_t res, const int32_t *status, const uint32_t *lambda, uint32_t *lo,
                            uint32_t *hi, int32_t *active, cudaStream_t st);
 cudaError_t launch_fb_trial(int N, uint32_t res, const uint32_t *lo, const uint32_t *hi, const int32_t *active,

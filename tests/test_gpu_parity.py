@@ -46,10 +46,10 @@ def _assert_results_equal(gpu, ref, idx=None):
         assert np.array_equal(a, ref[k]), f"{k} differs at instances {np.argwhere(a != ref[k])[:5].tolist()}"
 
 
-MODE = {"mode": 0}   # min-plus kernel under test: 0 packed 16-bit (default), 1 32-bit
+MODE = {"mode": 0}   # min-plus kernel under test: 0 packed 16-bit (default), 1 32-bit, 2 pruned
 
 
-@pytest.fixture(params=[0, 1], ids=["packed16", "wide32"])
+@pytest.fixture(params=[0, 1, 2], ids=["packed16", "wide32", "pruned"])
 def mode(request, S):
     S.themis_set_minplus_mode(request.param)
     MODE["mode"] = request.param
@@ -65,6 +65,8 @@ def _assert_tables_equal(S, gpu, ref):
     assert np.array_equal(gpu["G"], ref["G"])
     assert np.array_equal(gpu["Garg"], ref["Garg"])
     assert (gpu["G_pad"] == S.G_INF).all()
+    if MODE["mode"] == 2:      # tables of the restricted problem: only the results are comparable
+        return
     if MODE["mode"] == 0:
         solved = ref["status"] == 0
         assert np.array_equal(gpu["F"][solved], ref["F"][solved, -1, :])
@@ -316,15 +318,17 @@ def test_repeatable_and_tile_independent(S, mode):
             assert np.array_equal(runs[0][k], r[k]), k
 
 
-def test_both_kernels_agree(S):
-    """Packed 16-bit and 32-bit min-plus kernels: the same results, word for word."""
-    wl = W.make_workload(3, 300)
-    S.themis_set_minplus_mode(1)
-    wide = _gpu_solve(S, wl)
-    S.themis_set_minplus_mode(0)
-    packed = _gpu_solve(S, wl)
-    for k in RESULT_KEYS:
-        assert np.array_equal(wide[k], packed[k]), k
+def test_all_kernels_agree(S):
+    """Packed 16-bit, 32-bit and pruned min-plus kernels: the same results, word for word."""
+    for wl in (W.make_workload(3, 300), W.make_workload(4, 96), W.make_workload(2, 512)):
+        runs = []
+        for m in (1, 0, 2):
+            S.themis_set_minplus_mode(m)
+            runs.append(_gpu_solve(S, wl))
+        S.themis_set_minplus_mode(0)
+        for r in runs[1:]:
+            for k in RESULT_KEYS:
+                assert np.array_equal(runs[0][k], r[k]), k
 
 
 def test_totals_beyond_16_bits_fall_back_to_the_wide_kernel(S, oracle_mod):
