@@ -292,8 +292,9 @@ int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_s
  *      11000 buckets run mode 0 instead. */
 int themis_set_minplus_mode(int mode);
 
-/* Tuning knob of the min-plus kernel: consecutive budget cells per thread
- * (8 or 16); 0 restores the built-in choice.  Results do not depend on it. */
+/* Tuning knob of the dense min-plus kernels: consecutive budget cells per thread
+ * (4, 8 or 16; the 32-bit kernel treats 4 as its default); 0 restores the built-in
+ * choice.  Results do not depend on it. */
 int themis_set_minplus_tile(int cells_per_thread);
 
 /* Text for a return code; for THEMIS_E_CUDA includes the last CUDA error seen by

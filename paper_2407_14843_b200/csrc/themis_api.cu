@@ -498,7 +498,8 @@ int themis_set_minplus_mode(int mode)
 
 int themis_set_minplus_tile(int cells_per_thread)
 {
-    if (cells_per_thread != 0 && cells_per_thread != 8 && cells_per_thread != 16) return THEMIS_E_INVALID_ARG;
+    if (cells_per_thread != 0 && cells_per_thread != 4 && cells_per_thread != 8 && cells_per_thread != 16)
+        return THEMIS_E_INVALID_ARG;
     g_tile = cells_per_thread;
     return THEMIS_OK;
 }

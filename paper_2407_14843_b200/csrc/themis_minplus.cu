@@ -266,7 +266,7 @@ cudaError_t launch_minplus(const Params &p, int tile, cudaStream_t stream)
 {
     const int cells = p.T + 1;
     int R = tile;
-    if (R != 8 && R != 16) R = cells <= 2048 ? 8 : 16;
+    if (R != 8 && R != 16) R = 8;                       // (4 is a packed-kernel tile only)
     if (R == 8 && (cells + 7) / 8 > 1024) R = 16;
     const int chunks = (cells + R - 1) / R;
     const int threads = (chunks + 31) / 32 * 32;

@@ -43,6 +43,34 @@ struct Tile16 {
                                                           // consecutive lanes in distinct bank groups
 };
 
+// H consecutive words (H = 2, 4 or 8) from / to 8- or 16-byte aligned memory.
+template <int H>
+__device__ __forceinline__ void load_words(uint32_t (&w)[H], const uint32_t *src)
+{
+    if constexpr (H == 2) {
+        const uint2 x = *reinterpret_cast<const uint2 *>(src);
+        w[0] = x.x; w[1] = x.y;
+    } else {
+#pragma unroll
+        for (int v = 0; v < H / 4; ++v) {
+            const uint4 x = *reinterpret_cast<const uint4 *>(src + 4 * v);
+            w[4 * v + 0] = x.x; w[4 * v + 1] = x.y; w[4 * v + 2] = x.z; w[4 * v + 3] = x.w;
+        }
+    }
+}
+
+template <int H>
+__device__ __forceinline__ void store_words(const uint32_t (&w)[H], uint32_t *dst)
+{
+    if constexpr (H == 2) {
+        *reinterpret_cast<uint2 *>(dst) = make_uint2(w[0], w[1]);
+    } else {
+#pragma unroll
+        for (int v = 0; v < H / 4; ++v)
+            *reinterpret_cast<uint4 *>(dst + 4 * v) = make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
+    }
+}
+
 // One chunk step: R values of l (H even/odd pairs) against the thread's R cells.
 // w_hi holds words m .. m+H-1 of F, w_lo receives words m-H .. m-1 (m = J - q*H).
 template <int R>
@@ -51,11 +79,7 @@ __device__ __forceinline__ void chunk_step16(const uint32_t (&w_hi)[R / 2], uint
                                              const uint32_t *f_chunk, const uint32_t *g_chunk)
 {
     constexpr int H = R / 2;
-#pragma unroll
-    for (int v = 0; v < H / 4; ++v) {
-        const uint4 x = *reinterpret_cast<const uint4 *>(f_chunk + 4 * v);
-        w_lo[4 * v + 0] = x.x; w_lo[4 * v + 1] = x.y; w_lo[4 * v + 2] = x.z; w_lo[4 * v + 3] = x.w;
-    }
+    load_words<H>(w_lo, f_chunk);
 #pragma unroll
     for (int v = 0; v < R / 4; ++v) {
         const uint4 g4 = *reinterpret_cast<const uint4 *>(g_chunk + 4 * v);   // l = l0+4v .. l0+4v+3
@@ -93,7 +117,7 @@ minplus16_kernel(const Params p)
 {
     extern __shared__ __align__(128) uint32_t smem[];
     constexpr int H = Tile16<R>::H, CS = Tile16<R>::CS;
-    constexpr int U = R == 8 ? 4 : 2;                     // chunk steps per loop iteration
+    constexpr int U = 32 / R;                             // chunk steps per loop iteration (2, 4 or 8)
     const int n = blockIdx.x;
     if (p.active && !p.active[n]) return;
     const int tid = threadIdx.x;
@@ -157,14 +181,9 @@ minplus16_kernel(const Params p)
 
     // Stores the thread's H words of F_s to shared memory and to the uint16 table.
     auto store_chunk = [&](const uint32_t (&w)[H], int s) {
-#pragma unroll
-        for (int v = 0; v < H / 4; ++v)
-            *reinterpret_cast<uint4 *>(my_chunk + 4 * v) = make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
-        if (t0 + R <= pitch) {
-            uint4 *dst = reinterpret_cast<uint4 *>(F16_inst + (size_t)s * pitch + t0);
-#pragma unroll
-            for (int v = 0; v < H / 4; ++v) dst[v] = make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
-        }
+        store_words<H>(w, my_chunk);
+        if (t0 + R <= pitch)
+            store_words<H>(w, reinterpret_cast<uint32_t *>(F16_inst + (size_t)s * pitch + t0));
     };
 
     // stage 0: F_0 = G_0
@@ -381,13 +400,20 @@ cudaError_t launch_minplus16(const Params &p, int tile, cudaStream_t stream)
 {
     const int cells = p.T + 1;
     int R = tile;
-    if (R != 8 && R != 16) R = 8;                        // finer tiles waste fewer cells past the diagonal
+    // Finer tiles waste fewer cells past the diagonal (a warp spans 32 tiles and all its lanes
+    // run to its longest column) but pay more loads per update: 4 cells per thread up to 1024
+    // budget cells, 8 up to 8192, else 16.
+    if (R != 4 && R != 8 && R != 16) R = cells <= 1024 ? 4 : 8;
+    if (R == 4 && (cells + 3) / 4 > 1024) R = 8;
     if (R == 8 && (cells + 7) / 8 > 1024) R = 16;
     const int chunks = (cells + R - 1) / R;
     const int threads = (chunks + 31) / 32 * 32;
-    const int CS = R == 16 ? 12 : 4;
+    const int CS = R == 16 ? 12 : R / 2;
     const size_t words = (size_t)(kPadChunks + threads) * CS + 2u * (size_t)threads * R + 4 + 32 + 32 + THEMIS_MAX_STAGES;
     const size_t smem = words * sizeof(uint32_t);
+    if (R == 4)
+        return threads <= 512 ? launch_variant16<4, 512>(p, threads, smem, stream)
+                              : launch_variant16<4, 1024>(p, threads, smem, stream);
     if (R == 8)
         return threads <= 512 ? launch_variant16<8, 512>(p, threads, smem, stream)
                               : launch_variant16<8, 1024>(p, threads, smem, stream);

@@ -84,7 +84,7 @@ def _assert_tables_equal(S, gpu, ref):
 
 # ---------------------------------------------------------------- small, full tables
 
-@pytest.mark.parametrize("tile", [8, 16])
+@pytest.mark.parametrize("tile", [4, 8, 16])
 def test_config1_every_table(S, oracle_mod, tile, mode):
     """Smallest benchmark configuration: every intermediate table and result."""
     S.themis_set_minplus_tile(tile)
@@ -99,7 +99,7 @@ def test_config1_every_table(S, oracle_mod, tile, mode):
 
 
 @pytest.mark.parametrize("cfg,n", [(2, 96), (3, 160), (4, 12), (5, 3)])
-@pytest.mark.parametrize("tile", [8, 16])
+@pytest.mark.parametrize("tile", [4, 8, 16])
 def test_config_subsets_every_table(S, oracle_mod, cfg, n, tile, mode):
     """Subsets of the larger configurations (several tiles, ragged tail: T+1 is
     never a multiple of the tile): every table and result."""
@@ -309,7 +309,7 @@ def test_repeatable_and_tile_independent(S, mode):
     (every cross-thread hand-off is a barrier, so nothing may depend on timing)."""
     wl = W.make_workload(4, 24)
     runs = []
-    for tile in (16, 16, 8):
+    for tile in (16, 16, 8, 4):
         S.themis_set_minplus_tile(tile)
         runs.append(_gpu_solve(S, wl, tables=True))
     S.themis_set_minplus_tile(0)
