@@ -289,7 +289,15 @@ int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_s
  *      occur in the returned solution).  Returned configurations, costs, latencies
  *      and statuses are identical to modes 0 and 1 at a small fraction of the work;
  *      the A and F tables are those of the restricted problem.  Budgets above about
- *      11000 buckets run mode 0 instead. */
+ *      11000 buckets run mode 0 instead.
+ *   3: the solvers (themis_solve_*batch, host and static variants, the fallback) run
+ *      ONE kernel that scores only the candidates that can matter (per cores and
+ *      batch size the fewest replicas that sustain lambda), keeps only undominated
+ *      stage entries and undominated prefix states (budget, total), and never writes
+ *      a dense table: the G, Garg and A rows of the workspace then hold the stage
+ *      fronts and the argmin of the front cells only.  Same results again.  The
+ *      two-step entry points behave as in mode 2.  Falls back to mode 2 when its
+ *      shared memory (about 12 * row_pitch bytes plus tables) does not fit. */
 int themis_set_minplus_mode(int mode);
 
 /* Tuning knob of the dense min-plus kernels: consecutive budget cells per thread

@@ -12,10 +12,15 @@ namespace {
 thread_local cudaError_t t_last_cuda = cudaSuccess;
 thread_local char t_msg[256];
 int g_tile = 0;   // min-plus cells per thread; 0 = built-in choice
-thread_local bool g_horizontal = false;   // set by solve_impl for the launches it makes
-thread_local const int32_t *g_active = nullptr;   // per-instance mask for the launches of one solve
+// Which problem a launch solves and for which instances.
+enum Mode { kJoint = 0, kVertical = 1, kHorizontal = 2 };
+struct SolveOpts {
+    Mode mode = kJoint;
+    const int32_t *active = nullptr;   // [N] device mask, or nullptr: every instance
+};
 int g_mode = 0;   // 0: packed 16-bit dense kernel with 32-bit second pass; 1: 32-bit dense kernel;
-                  // 2: recurrence over undominated entries only (dense packed kernel above 11000 buckets)
+                  // 2: recurrence over undominated entries only (dense packed kernel above 11000 buckets);
+                  // 3: scoring and recurrence on undominated entries in one kernel
 
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
@@ -78,8 +83,9 @@ int layout_of(const themis_problem_t *pr, int vertical, themis_workspace_layout_
     return THEMIS_OK;
 }
 
-int make_params(const themis_problem_t *pr, int vertical, void *ws, size_t ws_bytes, Params *P)
+int make_params(const themis_problem_t *pr, const SolveOpts &opts, void *ws, size_t ws_bytes, Params *P)
 {
+    const int vertical = opts.mode == kVertical;
     themis_workspace_layout_t L;
     int rc = layout_of(pr, vertical, &L);
     if (rc != THEMIS_OK) return rc;
@@ -91,8 +97,8 @@ int make_params(const themis_problem_t *pr, int vertical, void *ws, size_t ws_by
     P->pitch = L.row_pitch;
     P->vertical = vertical ? 1 : 0;
     P->K = (vertical ? 1 : pr->h_max) * pr->c_max * pr->n_batch;
-    P->horizontal = (!vertical && g_horizontal) ? 1 : 0;
-    P->active = g_active;
+    P->horizontal = opts.mode == kHorizontal ? 1 : 0;
+    P->active = opts.active;
     char *base = static_cast<char *>(ws);
     P->G = reinterpret_cast<int32_t *>(base + L.g_offset);
     P->Garg = reinterpret_cast<uint16_t *>(base + L.garg_offset);
@@ -108,10 +114,11 @@ bool result_ok(const themis_result_t &o)
 }
 
 int score_impl(const themis_problem_t *pr, const int32_t *lat, const int32_t *pid, const uint32_t *lam,
-               const int32_t *rep, int vertical, void *ws, size_t ws_bytes, cudaStream_t st)
+               const int32_t *rep, const SolveOpts &opts, void *ws, size_t ws_bytes, cudaStream_t st)
 {
+    const int vertical = opts.mode == kVertical;
     Params P;
-    int rc = make_params(pr, vertical, ws, ws_bytes, &P);
+    int rc = make_params(pr, opts, ws, ws_bytes, &P);
     if (rc != THEMIS_OK) return rc;
     if (!lat || !lam || (vertical && !rep)) return THEMIS_E_INVALID_ARG;
     P.lat_us = lat; P.profile_id = pid; P.lambda_mrps = lam; P.replicas = rep;
@@ -119,18 +126,19 @@ int score_impl(const themis_problem_t *pr, const int32_t *lat, const int32_t *pi
     return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
 }
 
-int minplus_impl(const themis_problem_t *pr, const int32_t *rep, int vertical, themis_result_t out, void *ws,
-                 size_t ws_bytes, cudaStream_t st)
+int minplus_impl(const themis_problem_t *pr, const int32_t *rep, const SolveOpts &opts, themis_result_t out,
+                 void *ws, size_t ws_bytes, cudaStream_t st)
 {
+    const int vertical = opts.mode == kVertical;
     Params P;
-    int rc = make_params(pr, vertical, ws, ws_bytes, &P);
+    int rc = make_params(pr, opts, ws, ws_bytes, &P);
     if (rc != THEMIS_OK) return rc;
     if (!result_ok(out) || (vertical && !rep)) return THEMIS_E_INVALID_ARG;
     P.replicas = rep; P.out = out;
     cudaError_t e;
     if (g_mode == 1) {
         e = launch_minplus(P, g_tile, st);
-    } else if (g_mode == 2 && pruned_smem_bytes(P.pitch) <= 227u * 1024u) {
+    } else if (g_mode >= 2 && pruned_smem_bytes(P.pitch) <= kMaxDynamicSmem) {
         e = launch_minplus_pruned(P, st);
     } else {
         e = launch_minplus16(P, g_tile, st);
@@ -146,19 +154,28 @@ int minplus_impl(const themis_problem_t *pr, const int32_t *rep, int vertical, t
     return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
 }
 
-// mode: 0 joint, 1 vertical (h fixed), 2 horizontal (Algorithm 2)
 int solve_impl(const themis_problem_t *pr, const int32_t *lat, const int32_t *pid, const uint32_t *lam,
-               const int32_t *rep, int mode, themis_result_t out, void *ws, size_t ws_bytes, cudaStream_t st)
+               const int32_t *rep, const SolveOpts &opts, themis_result_t out, void *ws, size_t ws_bytes,
+               cudaStream_t st)
 {
-    const int vertical = mode == 1;
-    g_horizontal = mode == 2;
+    const int vertical = opts.mode == kVertical;
     int32_t T, K;
     int rc = validate(pr, vertical, &T, &K);
     if (rc != THEMIS_OK) return rc;
     if (!result_ok(out)) return THEMIS_E_INVALID_ARG;
-    rc = score_impl(pr, lat, pid, lam, rep, vertical, ws, ws_bytes, st);
-    if (rc == THEMIS_OK) rc = minplus_impl(pr, rep, vertical, out, ws, ws_bytes, st);
-    g_horizontal = false;
+    if (g_mode == 3) {          // one kernel on undominated entries, when its shared memory fits
+        Params P;
+        rc = make_params(pr, opts, ws, ws_bytes, &P);
+        if (rc != THEMIS_OK) return rc;
+        if (!lat || !lam || (vertical && !rep)) return THEMIS_E_INVALID_ARG;
+        P.lat_us = lat; P.profile_id = pid; P.lambda_mrps = lam; P.replicas = rep; P.out = out;
+        if (sparse_smem_bytes(P) <= kMaxDynamicSmem) {
+            cudaError_t e = launch_solve_sparse(P, st);
+            return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
+        }
+    }
+    rc = score_impl(pr, lat, pid, lam, rep, opts, ws, ws_bytes, st);
+    if (rc == THEMIS_OK) rc = minplus_impl(pr, rep, opts, out, ws, ws_bytes, st);
     return rc;
 }
 
@@ -281,7 +298,7 @@ int themis_solve_batch(const themis_problem_t *problem, const int32_t *d_lat_us,
                        const uint32_t *d_lambda_mrps, themis_result_t out, void *d_workspace,
                        size_t workspace_bytes, void *cuda_stream)
 {
-    return solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, nullptr, 0, out, d_workspace,
+    return solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, nullptr, SolveOpts{kJoint}, out, d_workspace,
                       workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -291,7 +308,7 @@ int themis_solve_vertical_batch(const themis_problem_t *problem, const int32_t *
                                 size_t workspace_bytes, void *cuda_stream)
 {
     if (!d_replicas) return THEMIS_E_INVALID_ARG;
-    return solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, d_replicas, 1, out, d_workspace,
+    return solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, d_replicas, SolveOpts{kVertical}, out, d_workspace,
                       workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -340,7 +357,7 @@ int themis_vertical_fallback_batch(const themis_problem_t *problem, const int32_
     trial.status = reinterpret_cast<int32_t *>(base + F.status);
 
     // 1. the whole load on the replicas in place
-    rc = solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, d_replicas, 1, out, d_workspace,
+    rc = solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, d_replicas, SolveOpts{kVertical}, out, d_workspace,
                     L.total_bytes, st);
     if (rc != THEMIS_OK) return rc;
     cudaError_t e = launch_fb_init(N, resolution_mrps, out.status, d_lambda_mrps, lo, hi, active, st);
@@ -352,10 +369,8 @@ int themis_vertical_fallback_batch(const themis_problem_t *problem, const int32_
     for (int r = 0; r < rounds; ++r) {
         e = launch_fb_trial(N, resolution_mrps, lo, hi, active, iter_active, trial_lambda, st);
         if (e != cudaSuccess) return fail_cuda(e);
-        g_active = iter_active;
-        rc = solve_impl(problem, d_lat_us, d_profile_id, trial_lambda, d_replicas, 1, trial, d_workspace,
-                        L.total_bytes, st);
-        g_active = nullptr;
+        rc = solve_impl(problem, d_lat_us, d_profile_id, trial_lambda, d_replicas,
+                        SolveOpts{kVertical, iter_active}, trial, d_workspace, L.total_bytes, st);
         if (rc != THEMIS_OK) return rc;
         e = launch_fb_update(N, lo, hi, iter_active, trial.status, st);
         if (e != cudaSuccess) return fail_cuda(e);
@@ -363,13 +378,12 @@ int themis_vertical_fallback_batch(const themis_problem_t *problem, const int32_
     // 3. the vertical part at the rate found, straight into the caller's arrays
     e = launch_fb_final_trial(N, resolution_mrps, lo, active, iter_active, trial_lambda, st);
     if (e != cudaSuccess) return fail_cuda(e);
-    g_active = iter_active;
-    rc = solve_impl(problem, d_lat_us, d_profile_id, trial_lambda, d_replicas, 1, out, d_workspace, L.total_bytes, st);
-    g_active = nullptr;
+    rc = solve_impl(problem, d_lat_us, d_profile_id, trial_lambda, d_replicas, SolveOpts{kVertical, iter_active},
+                    out, d_workspace, L.total_bytes, st);
     if (rc != THEMIS_OK) return rc;
     // 4. the rest of the load on extra replicas
     Params P;
-    rc = make_params(problem, 1, d_workspace, L.total_bytes, &P);
+    rc = make_params(problem, SolveOpts{kVertical}, d_workspace, L.total_bytes, &P);
     if (rc != THEMIS_OK) return rc;
     P.lat_us = d_lat_us; P.profile_id = d_profile_id; P.lambda_mrps = d_lambda_mrps; P.replicas = d_replicas;
     P.out = out;
@@ -383,7 +397,7 @@ int themis_solve_horizontal_batch(const themis_problem_t *problem, const int32_t
                                   void *cuda_stream)
 {
     if (problem && problem->c_max != 1) return THEMIS_E_INVALID_ARG;
-    return solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, nullptr, 2, out, d_workspace,
+    return solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, nullptr, SolveOpts{kHorizontal}, out, d_workspace,
                       workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -391,14 +405,15 @@ int themis_score_batch(const themis_problem_t *problem, const int32_t *d_lat_us,
                        const uint32_t *d_lambda_mrps, const int32_t *d_replicas, void *d_workspace,
                        size_t workspace_bytes, void *cuda_stream)
 {
-    return score_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, d_replicas, d_replicas != nullptr,
+    return score_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, d_replicas,
+                      SolveOpts{d_replicas ? kVertical : kJoint},
                       d_workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int themis_minplus_batch(const themis_problem_t *problem, const int32_t *d_replicas, themis_result_t out,
                          void *d_workspace, size_t workspace_bytes, void *cuda_stream)
 {
-    return minplus_impl(problem, d_replicas, d_replicas != nullptr, out, d_workspace, workspace_bytes,
+    return minplus_impl(problem, d_replicas, SolveOpts{d_replicas ? kVertical : kJoint}, out, d_workspace, workspace_bytes,
                         static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -451,7 +466,8 @@ int themis_solve_batch_host(const themis_problem_t *problem, const int32_t *h_la
     rc = solve_impl(problem, reinterpret_cast<const int32_t *>(base + H.lat),
                     h_profile_id ? reinterpret_cast<const int32_t *>(base + H.pid) : nullptr,
                     reinterpret_cast<const uint32_t *>(base + H.lam),
-                    vertical ? reinterpret_cast<const int32_t *>(base + H.rep) : nullptr, vertical, d_out,
+                    vertical ? reinterpret_cast<const int32_t *>(base + H.rep) : nullptr,
+                    SolveOpts{vertical ? kVertical : kJoint}, d_out,
                     d_workspace, L.total_bytes, st);
     if (rc != THEMIS_OK) return rc;
     THEMIS_COPY(h_out.h, d_out.h, N * S * 4, cudaMemcpyDeviceToHost);
@@ -477,7 +493,8 @@ int themis_solve_batch_static(const themis_problem_t *problem, const int32_t *d_
     void *scratch = nullptr;
     rc = static_scratch_ptr(&scratch);
     if (rc != THEMIS_OK) return rc;
-    return solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, d_replicas, vertical, out, scratch,
+    return solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, d_replicas,
+                      SolveOpts{vertical ? kVertical : kJoint}, out, scratch,
                       (size_t)THEMIS_STATIC_SCRATCH_BYTES, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -491,7 +508,7 @@ int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_s
 
 int themis_set_minplus_mode(int mode)
 {
-    if (mode < 0 || mode > 2) return THEMIS_E_INVALID_ARG;
+    if (mode < 0 || mode > 3) return THEMIS_E_INVALID_ARG;
     g_mode = mode;
     return THEMIS_OK;
 }

@@ -76,6 +76,10 @@ cudaError_t launch_score(const Params &p, cudaStream_t stream);
 cudaError_t launch_minplus(const Params &p, int tile, cudaStream_t stream);
 cudaError_t launch_minplus16(const Params &p, int tile, cudaStream_t stream);
 cudaError_t launch_minplus_pruned(const Params &p, cudaStream_t stream);
+// Scoring and recurrence on undominated entries in one kernel (needs lat_us, lambda, out set).
+size_t sparse_smem_bytes(const Params &p);
+cudaError_t launch_solve_sparse(const Params &p, cudaStream_t stream);
+constexpr size_t kMaxDynamicSmem = 227u * 1024u;
 // Dynamic shared memory of the pruned kernel for a row pitch; it cannot run above 227 KB.
 inline size_t pruned_smem_bytes(int pitch) { return sizeof(uint32_t) * (5u * (size_t)pitch + 4 + 32); }
 cudaError_t launch_fb_init(int N, uint32_t res, const int32_t *status, const uint32_t *lambda, uint32_t *lo,

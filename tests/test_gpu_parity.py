@@ -49,7 +49,7 @@ def _assert_results_equal(gpu, ref, idx=None):
 MODE = {"mode": 0}   # min-plus kernel under test: 0 packed 16-bit (default), 1 32-bit, 2 pruned
 
 
-@pytest.fixture(params=[0, 1, 2], ids=["packed16", "wide32", "pruned"])
+@pytest.fixture(params=[0, 1, 2, 3], ids=["packed16", "wide32", "pruned", "sparse"])
 def mode(request, S):
     S.themis_set_minplus_mode(request.param)
     MODE["mode"] = request.param
@@ -62,6 +62,8 @@ def _assert_tables_equal(S, gpu, ref):
     """G, Garg everywhere; F (last prefix) where the instance is solved; then
     32-bit kernel: A where F_s[t] is reachable (0 elsewhere);
     packed kernel: every prefix table F_s[t], saturated at 0x7FFF."""
+    if MODE["mode"] == 3:      # one fused kernel: the workspace holds fronts, not the dense tables
+        return
     assert np.array_equal(gpu["G"], ref["G"])
     assert np.array_equal(gpu["Garg"], ref["Garg"])
     assert (gpu["G_pad"] == S.G_INF).all()
@@ -319,10 +321,10 @@ def test_repeatable_and_tile_independent(S, mode):
 
 
 def test_all_kernels_agree(S):
-    """Packed 16-bit, 32-bit and pruned min-plus kernels: the same results, word for word."""
+    """Packed 16-bit, 32-bit, pruned and fused sparse kernels: the same results, word for word."""
     for wl in (W.make_workload(3, 300), W.make_workload(4, 96), W.make_workload(2, 512)):
         runs = []
-        for m in (1, 0, 2):
+        for m in (1, 0, 2, 3):
             S.themis_set_minplus_mode(m)
             runs.append(_gpu_solve(S, wl))
         S.themis_set_minplus_mode(0)
