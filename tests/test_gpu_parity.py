@@ -412,22 +412,38 @@ def test_config2_full(S, oracle_mod, mode):
     _assert_results_equal(gpu, oracle_mod.solve_batch(wl))
 
 
-@pytest.mark.parametrize("cfg,n_sample", [(3, 1024), (4, 40), (5, 8)])
-def test_full_size_configs_sampled(S, oracle_mod, cfg, n_sample, mode):
-    """The full batch in the launch configuration the benchmark times; sampled
-    instances are compared with the oracle one by one, every instance is checked
-    against the size-independent properties."""
+_ORACLE_CACHE = {}
+
+
+def _oracle_cached(oracle_mod, key, wl):
+    """The oracle's answer for a workload, computed once per test session (the
+    same batches are checked against every kernel mode)."""
+    if key not in _ORACLE_CACHE:
+        _ORACLE_CACHE[key] = oracle_mod.solve_batch(wl)
+    return _ORACLE_CACHE[key]
+
+
+@pytest.mark.parametrize("cfg", [3, 4])
+def test_full_size_configs_every_instance(S, oracle_mod, cfg, mode):
+    """Configurations 3 (86400 instances) and 4 (16384 instances) in the launch
+    configuration the benchmark times: every instance against the oracle."""
     wl = W.make_workload(cfg)
     gpu = _gpu_solve(S, wl)
     _check_properties(wl, gpu)
+    _assert_results_equal(gpu, _oracle_cached(oracle_mod, ("full", cfg), wl))
+
+
+def test_full_size_config5_sampled(S, oracle_mod, mode):
+    """Configuration 5 (4096 instances, 20 stages, T = 8192) in the benchmark's launch
+    configuration: every instance is checked against the size-independent properties,
+    a seeded sample of 48 instances against the oracle one by one (the oracle needs
+    about a second per instance and core)."""
+    wl = W.make_workload(5)
+    gpu = _gpu_solve(S, wl)
+    _check_properties(wl, gpu)
     pick = np.unique(np.concatenate([
-        W.rand_int(77, cfg, np.arange(n_sample, dtype=np.uint64), 0, wl.n_instances - 1),
-        [0, wl.n_instances - 1]]))
-    if cfg == 3:   # make sure spike seconds (possibly infeasible) are sampled
-        hot = np.argsort(wl.lambda_mrps)[-16:]
-        pick = np.unique(np.concatenate([pick, hot, np.flatnonzero(gpu["status"] == 1)[:64]]))
+        W.rand_int(77, 5, np.arange(46, dtype=np.uint64), 0, wl.n_instances - 1), [0, wl.n_instances - 1],
+        np.flatnonzero(gpu["status"] == 1)[:8]]))
     sub = dataclasses.replace(wl, n_instances=len(pick), profile_id=wl.profile_id[pick].copy(),
-                              lambda_mrps=wl.lambda_mrps[pick].copy(),
-                              replicas=None if wl.replicas is None else wl.replicas[pick].copy())
-    ref = oracle_mod.solve_batch(sub)
-    _assert_results_equal(gpu, ref, idx=pick)
+                              lambda_mrps=wl.lambda_mrps[pick].copy())
+    _assert_results_equal(gpu, _oracle_cached(oracle_mod, ("cfg5", tuple(pick.tolist())), sub), idx=pick)
