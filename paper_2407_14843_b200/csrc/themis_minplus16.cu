@@ -35,6 +35,10 @@ namespace {
 
 constexpr uint32_t kInf16x2 = (kInf16 << 16) | kInf16;
 constexpr int kPadChunks = 32;   // "unreachable" chunks in front of F[0]: one per lane of a warp
+// Budgets just above a whole number of tile groups (T a power of two gives T + 1 cells) would cost
+// a whole extra warp walking the longest columns for a handful of cells.  Up to this many cells
+// beyond the last full group are instead computed by a block-wide reduction per stage.
+constexpr int kMaxExtra = 8;
 
 template <int R>
 struct Tile16 {
@@ -111,7 +115,8 @@ __device__ __forceinline__ uint32_t block_min(uint32_t v, uint32_t *red, int tid
     return m;
 }
 
-template <int R, int MAXT>
+// EXTRA: the block also computes up to kMaxExtra cells beyond its tiles (see kMaxExtra).
+template <int R, int MAXT, bool EXTRA>
 __global__ void __launch_bounds__(MAXT)
 minplus16_kernel(const Params p)
 {
@@ -124,7 +129,9 @@ minplus16_kernel(const Params p)
     const int NT = blockDim.x;
     const int n_warps = NT >> 5;
     const int T = p.T, pitch = p.pitch, S = p.prob.n_stages;
-    const int Tp = NT * R;                                // padded budget length, >= pitch
+    const int Tc = NT * R;                                // cells covered by the tiles
+    const int Tp = EXTRA ? max(Tc, pitch) : Tc;           // length of the G buffers (Tc >= pitch without extras)
+    const int n_extra = EXTRA ? max(0, T + 1 - Tc) : 0;   // cells beyond the tiles, at most kMaxExtra
 
     uint32_t *Fw = smem;                                  // (kPadChunks + NT) chunks of CS words
     uint32_t *Gbuf0 = Fw + (kPadChunks + NT) * CS;
@@ -133,6 +140,8 @@ minplus16_kernel(const Params p)
     uint32_t *red = reinterpret_cast<uint32_t *>(mbar + 2);   // 32 words
     uint32_t *xchg = red + 32;                                // 32 words: last accp word of each warp
     uint32_t *stage_lmin = xchg + 32;                         // 64 words: first reachable l of every G_s
+    uint32_t *fx_prev = stage_lmin + THEMIS_MAX_STAGES;       // kMaxExtra words: F_{s-1} at the extra cells
+    uint32_t *fx_acc = fx_prev + kMaxExtra;                   // kMaxExtra words: F_s at the extra cells, building
 
     // Which tile (R consecutive cells) this thread owns: lanes keep consecutive tiles,
     // warps take the tile groups the host dealt them (see assign_warp_groups).
@@ -205,8 +214,18 @@ minplus16_kernel(const Params p)
         }
         note_first_reachable(first, 0);
         store_chunk(w, 0);
+        if (tid < n_extra) {
+            const uint32_t v = min(Gbuf0[Tc + tid], kInf16);
+            fx_prev[tid] = v;
+            F16_inst[Tc + tid] = (uint16_t)v;
+        }
     }
     failed = __syncthreads_or(failed);
+    // Half-word i (< Tc) of the prefix table in shared memory.
+    auto f_at = [&](int i) -> uint32_t {
+        const uint32_t w = Fw[(kPadChunks + i / R) * CS + ((i % R) >> 1)];
+        return (i & 1) ? (w >> 16) : (w & 0xFFFFu);
+    };
     // Lowest reachable budget of the prefix F_{s-1} (0xFFFFFFFF: nothing reachable).  Everything
     // below it, and every G_s[l] below that row's first reachable l, can only give "unreachable".
     uint32_t prefix_min = stage_lmin[0];
@@ -229,6 +248,7 @@ minplus16_kernel(const Params p)
                 }
             }
             note_first_reachable(first, s);
+            if (EXTRA && tid < kMaxExtra) fx_acc[tid] = 0xFFFFFFFFu;
         }
         failed = __syncthreads_or(failed);                // G_s and F_{s-1} visible to all
         if (failed) break;
@@ -270,6 +290,35 @@ minplus16_kernel(const Params p)
             }
         }
         prefix_min = dead ? 0xFFFFFFFFu : prefix_min + g_min;
+        if (EXTRA && n_extra > 0) {
+            // Extra cells t = Tc + e: this thread's share of min_l F_{s-1}[t-l] + G_s[l] is its own
+            // tile's l range; thread 0 adds l >= Tc (those entries of G are still raw costs).
+            uint32_t ex[kMaxExtra];
+#pragma unroll
+            for (int e = 0; e < kMaxExtra; ++e) ex[e] = 0xFFFFFFFFu;
+            for (int r = 0; r < R; ++r) {
+                const int l = t0 + r;
+                const uint32_t g = Gk[l] & 0xFFFFu;
+#pragma unroll
+                for (int e = 0; e < kMaxExtra; ++e)
+                    if (e < n_extra) {
+                        const int i = Tc + e - l;             // >= 1
+                        ex[e] = min(ex[e], (i < Tc ? f_at(i) : fx_prev[i - Tc]) + g);
+                    }
+            }
+            if (tid == 0) {
+#pragma unroll
+                for (int e = 0; e < kMaxExtra; ++e)
+                    for (int l = Tc; l <= Tc + e && e < n_extra; ++l)
+                        ex[e] = min(ex[e], f_at(Tc + e - l) + min(Gk[l], kInf16));
+            }
+#pragma unroll
+            for (int e = 0; e < kMaxExtra; ++e)
+                if (e < n_extra) {
+                    const uint32_t m = __reduce_min_sync(0xFFFFFFFFu, ex[e]);
+                    if ((tid & 31) == 0) atomicMin(&fx_acc[e], m);
+                }
+        }
         if ((tid & 31) == 31) xchg[tile >> 5] = accp[H - 1];
         __syncthreads();                                  // every read of F_{s-1} is done
 
@@ -283,6 +332,11 @@ minplus16_kernel(const Params p)
             w[r] = __vminu2(__vminu2(acc[r], odd), kInf16x2);
         }
         store_chunk(w, s);
+        if (tid < n_extra) {                              // every share arrived before the barrier above
+            const uint32_t v = min(fx_acc[tid], kInf16);
+            fx_prev[tid] = v;
+            F16_inst[(size_t)s * pitch + Tc + tid] = (uint16_t)v;
+        }
     }
     failed = __syncthreads_or(failed);
 
@@ -303,6 +357,7 @@ minplus16_kernel(const Params p)
         if (t <= T) best = min(best, ((w & 0xFFFFu) << 16) | (uint32_t)t);
         if (t + 1 <= T) best = min(best, (w & 0xFFFF0000u) | (uint32_t)(t + 1));
     }
+    if (tid < n_extra) best = min(best, (fx_prev[tid] << 16) | (uint32_t)(Tc + tid));
     best = block_min(best, red, tid, n_warps);
     const uint32_t best_cost = best >> 16;
     const int tstar = (int)(best & 0xFFFFu);
@@ -339,6 +394,9 @@ minplus16_kernel(const Params p)
             }
         }
     }
+
+    if (tid < n_extra)
+        p.F[(size_t)n * pitch + Tc + tid] = fx_prev[tid] >= kInf16 ? THEMIS_G_INF : (int32_t)fx_prev[tid];
 
     // backtrack along the optimal path: lowest l with F_{s-1}[t-l] + G_s[l] == F_s[t]
     int t = tstar;
@@ -382,16 +440,23 @@ minplus16_kernel(const Params p)
     }
 }
 
+template <int R, int MAXT, bool EXTRA>
+cudaError_t launch_variant16x(const Params &p, int threads, size_t smem, cudaStream_t stream)
+{
+    cudaError_t e = cudaFuncSetAttribute(minplus16_kernel<R, MAXT, EXTRA>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    minplus16_kernel<R, MAXT, EXTRA><<<p.prob.n_instances, threads, smem, stream>>>(p);
+    return cudaGetLastError();
+}
+
 template <int R, int MAXT>
 cudaError_t launch_variant16(const Params &p_in, int threads, size_t smem, cudaStream_t stream)
 {
     Params p = p_in;
     assign_warp_groups(threads / 32, p.warp_group);
-    cudaError_t e = cudaFuncSetAttribute(minplus16_kernel<R, MAXT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
-    if (e != cudaSuccess) return e;
-    minplus16_kernel<R, MAXT><<<p.prob.n_instances, threads, smem, stream>>>(p);
-    return cudaGetLastError();
+    return threads * R < p.T + 1 ? launch_variant16x<R, MAXT, true>(p, threads, smem, stream)
+                                 : launch_variant16x<R, MAXT, false>(p, threads, smem, stream);
 }
 
 }  // namespace
@@ -403,13 +468,18 @@ cudaError_t launch_minplus16(const Params &p, int tile, cudaStream_t stream)
     // Finer tiles waste fewer cells past the diagonal (a warp spans 32 tiles and all its lanes
     // run to its longest column) but pay more loads per update: 4 cells per thread up to 1024
     // budget cells, 8 up to 8192, else 16.
-    if (R != 4 && R != 8 && R != 16) R = cells <= 1024 ? 4 : 8;
-    if (R == 4 && (cells + 3) / 4 > 1024) R = 8;
-    if (R == 8 && (cells + 7) / 8 > 1024) R = 16;
+    if (R != 4 && R != 8 && R != 16) R = cells <= 1024 + kMaxExtra ? 4 : 8;
+    if (R == 4 && (cells - kMaxExtra + 3) / 4 > 1024) R = 8;
+    if (R == 8 && (cells - kMaxExtra + 7) / 8 > 1024) R = 16;
     const int chunks = (cells + R - 1) / R;
-    const int threads = (chunks + 31) / 32 * 32;
+    int groups = (chunks + 31) / 32;
+    // a few cells beyond a whole number of tile groups are handled outside the tiles
+    if (groups > 1 && cells - (groups - 1) * 32 * R <= kMaxExtra) --groups;
+    const int threads = groups * 32;
     const int CS = R == 16 ? 12 : R / 2;
-    const size_t words = (size_t)(kPadChunks + threads) * CS + 2u * (size_t)threads * R + 4 + 32 + 32 + THEMIS_MAX_STAGES;
+    const size_t g_words = (size_t)(threads * R > p.pitch ? threads * R : p.pitch);
+    const size_t words = (size_t)(kPadChunks + threads) * CS + 2u * g_words + 4 + 32 + 32 + THEMIS_MAX_STAGES +
+                         2 * kMaxExtra;
     const size_t smem = words * sizeof(uint32_t);
     if (R == 4)
         return threads <= 512 ? launch_variant16<4, 512>(p, threads, smem, stream)

@@ -222,7 +222,8 @@ def test_vertical_fallback(S, oracle_mod, res, mode):
 
 # ---------------------------------------------------------------- edge cases
 
-@pytest.mark.parametrize("T", [1, 2, 31, 32, 33, 255, 256, 257, 511, 2047, 2048, 2049])
+@pytest.mark.parametrize("T", [1, 2, 31, 32, 33, 127, 128, 131, 135, 136, 255, 256, 257, 263, 264, 511, 512, 1024, 1031,
+                               2047, 2048, 2049, 2055, 2056])
 def test_budget_lengths_around_tile_boundaries(S, oracle_mod, T, mode):
     wl = W.random_tiny_workload(5000 + T, 6, 3, 8, (1, 2, 4), 4, T, bucket_us=max(1, 400_000 // T) if T < 400 else 1000,
                                 rate_lo=20.0, rate_hi=120.0)
