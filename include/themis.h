@@ -264,6 +264,29 @@ int themis_solve_batch_static(const themis_problem_t *problem, const int32_t *d_
                               const int32_t *d_replicas, themis_result_t out, void *cuda_stream);
 
 /*
+ * Profile fit (Eq. 1): least-squares fit of
+ *     l(b, c) = gamma * b / c + epsilon / c + delta * b + eta      [milliseconds]
+ * to measured samples, one model (pipeline stage) at a time, and the latency table
+ * the solvers take as input, evaluated from the fitted coefficients.
+ *   d_sample_b, d_sample_c  [n_samples] int32: the (batch size, cores) grid the models
+ *                           were run on (shared by all models), values >= 1
+ *   d_latency_ms            [n_models][n_samples] double: measured latency per model
+ *   d_batch_sizes           [n_batch] int32 (device): the table's batch sizes
+ *   d_coeffs                [n_models][4] double out: gamma, epsilon, delta, eta
+ *   d_lat_us                [n_models][c_max][n_batch] int32 out: ceil(1000 * l(b, c)),
+ *                           at least 1; this is the layout of one profile's stages
+ *                           in the solvers' d_lat_us when models are its stages
+ *   d_status                [n_models] int32 out: 0, or THEMIS_STATUS_BAD_INPUT when the
+ *                           samples do not determine the four coefficients (table = 0)
+ * Double precision throughout (normal equations, Gaussian elimination with partial
+ * pivoting).  n_samples >= 4.
+ */
+int themis_fit_profiles_batch(int32_t n_models, int32_t n_samples, const int32_t *d_sample_b,
+                              const int32_t *d_sample_c, const double *d_latency_ms, int32_t c_max,
+                              int32_t n_batch, const int32_t *d_batch_sizes, double *d_coeffs,
+                              int32_t *d_lat_us, int32_t *d_status, void *cuda_stream);
+
+/*
  * Integer-ALU throughput probe (not part of the method): every thread runs
  * `iters` rounds of 16 independent add-then-min updates, the operation pair of
  * the recurrence, in one of three instruction forms:

@@ -498,6 +498,20 @@ int themis_solve_batch_static(const themis_problem_t *problem, const int32_t *d_
                       (size_t)THEMIS_STATIC_SCRATCH_BYTES, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int themis_fit_profiles_batch(int32_t n_models, int32_t n_samples, const int32_t *d_sample_b,
+                              const int32_t *d_sample_c, const double *d_latency_ms, int32_t c_max,
+                              int32_t n_batch, const int32_t *d_batch_sizes, double *d_coeffs,
+                              int32_t *d_lat_us, int32_t *d_status, void *cuda_stream)
+{
+    if (n_models < 1 || n_samples < 4 || c_max < 1 || n_batch < 1 || n_batch > THEMIS_MAX_BATCH_SIZES ||
+        !d_sample_b || !d_sample_c || !d_latency_ms || !d_batch_sizes || !d_coeffs || !d_lat_us || !d_status)
+        return THEMIS_E_INVALID_ARG;
+    cudaError_t e = launch_fit_profiles(n_models, n_samples, d_sample_b, d_sample_c, d_latency_ms, c_max, n_batch,
+                                        d_batch_sizes, d_coeffs, d_lat_us, d_status,
+                                        static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
+}
+
 int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_sink, void *cuda_stream)
 {
     if (mode < 0 || mode > 4 || blocks < 1 || threads < 32 || threads > 1024 || iters < 1 || !d_sink)

@@ -92,6 +92,9 @@ cudaError_t launch_fb_final_trial(int N, uint32_t res, const uint32_t *lo, const
                                   int32_t *iter_active, uint32_t *trial_lambda, cudaStream_t st);
 cudaError_t launch_fb_finish(const Params &p, uint32_t res, const uint32_t *lo, const uint32_t *hi,
                              const int32_t *active, uint32_t *lambda_vertical, int32_t *extra, cudaStream_t st);
+cudaError_t launch_fit_profiles(int n_models, int n_samples, const int32_t *sample_b, const int32_t *sample_c,
+                                const double *latency_ms, int c_max, int n_batch, const int32_t *d_batch_sizes,
+                                double *coeffs, int32_t *lat_us, int32_t *status, cudaStream_t st);
 cudaError_t launch_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *sink,
                              cudaStream_t stream);
 

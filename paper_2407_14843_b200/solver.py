@@ -34,6 +34,7 @@ EXPORTS = (
     "themis_host_workspace_bytes", "themis_solve_batch_host", "themis_alu_probe",
     "themis_set_minplus_tile", "themis_solve_batch_static", "themis_set_minplus_mode",
     "themis_solve_horizontal_batch", "themis_fallback_workspace_bytes", "themis_vertical_fallback_batch",
+    "themis_fit_profiles_batch",
 )
 
 
@@ -105,6 +106,8 @@ def _load() -> ctypes.CDLL:
     lib.themis_minplus_batch.argtypes = [PP, vp, Result, vp, sz, vp]
     lib.themis_solve_batch_host.argtypes = [PP, vp, vp, vp, vp, Result, vp, sz, vp]
     lib.themis_solve_batch_static.argtypes = [PP, vp, vp, vp, vp, Result, vp]
+    lib.themis_fit_profiles_batch.argtypes = [ctypes.c_int32, ctypes.c_int32, vp, vp, vp, ctypes.c_int32,
+                                              ctypes.c_int32, vp, vp, vp, vp, vp]
     lib.themis_alu_probe.argtypes = [ctypes.c_int] * 4 + [vp, vp]
     lib.themis_set_minplus_tile.argtypes = [ctypes.c_int]
     lib.themis_set_minplus_mode.argtypes = [ctypes.c_int]
@@ -245,6 +248,18 @@ def themis_solve_batch_static(problem: Problem, lat_us, profile_id, lambda_mrps,
         ctypes.byref(problem), _dptr(lat_us, torch.int32, "lat_us"), _dptr(profile_id, torch.int32, "profile_id"),
         _dptr(lambda_mrps, torch.uint32, "lambda_mrps"), _dptr(replicas, torch.int32, "replicas"), _result(out),
         _stream()), "themis_solve_batch_static")
+
+
+def themis_fit_profiles_batch(sample_b, sample_c, latency_ms, c_max: int, batch_sizes, coeffs, lat_us, status) -> None:
+    """Eq. 1 fit for ``latency_ms.shape[0]`` models; all arguments are CUDA tensors
+    (``batch_sizes`` int32 on the device)."""
+    n_models, n_samples = latency_ms.shape
+    _check(_lib.themis_fit_profiles_batch(
+        n_models, n_samples, _dptr(sample_b, torch.int32, "sample_b"), _dptr(sample_c, torch.int32, "sample_c"),
+        _dptr(latency_ms, torch.float64, "latency_ms"), int(c_max), batch_sizes.numel(),
+        _dptr(batch_sizes, torch.int32, "batch_sizes"), _dptr(coeffs, torch.float64, "coeffs"),
+        _dptr(lat_us, torch.int32, "lat_us"), _dptr(status, torch.int32, "status"), _stream()),
+        "themis_fit_profiles_batch")
 
 
 def themis_alu_probe(mode: int, blocks: int, threads: int, iters: int, sink) -> None:

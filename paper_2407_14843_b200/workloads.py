@@ -287,3 +287,21 @@ def random_tiny_workload(seed: int, n_instances: int, n_stages: int, c_max: int,
         slo_us=T * bucket_us, bucket_us=bucket_us, flags=flags, vertical=vertical, lat_us=lat,
         profile_id=np.arange(n_instances, dtype=np.int32), lambda_mrps=_to_mrps(rate),
         replicas=replicas, seed=seed)
+
+
+def profile_samples(seed: int, n_models: int, noise: float = 0.02):
+    """Synthetic profiling runs for the Eq. 1 fit: every model is "measured" on the
+    grid b in {1,2,4,8,16} x c in {1,2,4,8,16}; its true coefficients are drawn
+    gamma~U[5,40], epsilon~U[2,20], delta~U[0.1,2], eta~U[1,10] (milliseconds) and
+    each measurement carries multiplicative log-normal noise.  Returns
+    (sample_b int32 [25], sample_c int32 [25], latency_ms float64 [M][25], true coeffs [M][4])."""
+    grid = (1, 2, 4, 8, 16)
+    sample_b = np.repeat(np.asarray(grid, np.int32), len(grid))
+    sample_c = np.tile(np.asarray(grid, np.int32), len(grid))
+    m = np.arange(n_models, dtype=np.uint64)
+    true = np.stack([rand_uniform(seed, 11, m, 5.0, 40.0), rand_uniform(seed, 12, m, 2.0, 20.0),
+                     rand_uniform(seed, 13, m, 0.1, 2.0), rand_uniform(seed, 14, m, 1.0, 10.0)], axis=1)
+    b, c = sample_b.astype(np.float64), sample_c.astype(np.float64)
+    clean = (true[:, 0:1] * b / c + true[:, 1:2] / c + true[:, 2:3] * b + true[:, 3:4])
+    z = rand_normal(seed, 15, np.arange(n_models * b.size, dtype=np.uint64)).reshape(n_models, b.size)
+    return sample_b, sample_c, clean * np.exp(noise * z), true

@@ -101,7 +101,7 @@ def test_pointer_and_workspace_checks(S):
     assert lib.themis_alu_probe(9, 1, 32, 1, one, None) == S.E_INVALID_ARG
     assert lib.themis_set_minplus_tile(12) == S.E_INVALID_ARG
     assert lib.themis_set_minplus_tile(0) == S.OK
-    assert lib.themis_set_minplus_mode(3) == S.E_INVALID_ARG and lib.themis_set_minplus_mode(0) == S.OK
+    assert lib.themis_set_minplus_mode(4) == S.E_INVALID_ARG and lib.themis_set_minplus_mode(0) == S.OK
 
 
 def test_strerror(S):
