@@ -220,7 +220,7 @@ class ClockSampler:
 def probe_alu_peak(solver, torch, mode):
     """Add-min throughput sustained by themis_alu_probe in TOP/s (two operations
     per cell update): mode 1 = fused 32-bit add-min, mode 3 = packed 2 x 16-bit."""
-    blocks, threads, iters = N_SMS * 8, 256, 4000
+    blocks, threads, iters = N_SMS * 8, 256, 20000          # about 0.1 s per form
     cells_per_update = 2 if mode == 3 else 1
     sink = torch.empty(blocks * threads, dtype=torch.uint32, device="cuda")
     solver.themis_alu_probe(mode, blocks, threads, 50, sink)
@@ -407,6 +407,8 @@ def run_ours(args):
         "kernels_ms": {"score_kernel": score_ms, ("minplus16_kernel" if packed else "minplus_kernel"): minplus_ms},
         "infeasible_instances": n_infeasible, "device_error_instances": n_error,
         "input_checksums": wl.checksums(),
+        "device": {"name": torch.cuda.get_device_name(local_rank),
+                   "sms": torch.cuda.get_device_properties(local_rank).multi_processor_count},
         "roofline": {
             "kernel": "minplus16_kernel" if packed else "minplus_kernel", "bound": "alu",
             "achieved": achieved_tops, "peak": alu_peak,
