@@ -96,7 +96,6 @@ int make_params(const themis_problem_t *pr, const SolveOpts &opts, void *ws, siz
     P->T = L.T;
     P->pitch = L.row_pitch;
     P->vertical = vertical ? 1 : 0;
-    P->K = (vertical ? 1 : pr->h_max) * pr->c_max * pr->n_batch;
     P->horizontal = opts.mode == kHorizontal ? 1 : 0;
     P->active = opts.active;
     char *base = static_cast<char *>(ws);

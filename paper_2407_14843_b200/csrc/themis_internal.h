@@ -38,7 +38,6 @@ struct Params {
     int32_t vertical;   // 1: h fixed per stage from replicas[]
     int32_t horizontal; // 1: Algorithm 2, one candidate per batch size with the fewest replicas
                         //    that sustain lambda; candidate index = batch index, stage cost = h
-    int32_t K;          // candidates per stage
     int32_t only_flagged;  // wide min-plus kernel: solve only instances flagged kFlagNeedsWide
     uint8_t warp_group[32];  // min-plus kernels: tile group (32 tiles) owned by each warp
     const int32_t *lat_us;

@@ -1,8 +1,6 @@
 """Parity of the CUDA path (called through the C ABI) with the CPU oracle,
 element by element and bit-exact, on the same seeded inputs."""
 import dataclasses
-import json
-import os
 
 import numpy as np
 import pytest
