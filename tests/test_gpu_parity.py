@@ -252,6 +252,30 @@ def test_stage_counts(S, oracle_mod, n_stages, mode):
     _assert_results_equal(gpu, ref)
 
 
+SHAPES = [  # n_stages, c_max, batch sizes, h_max, T, bucket_us, vertical, rate range (rps)
+    (2, 1, tuple(range(1, 17)), 512, 300, 1000, False, (50.0, 4000.0)),      # widest replica table
+    (3, 100, (1,), 3, 77, 2000, False, (5.0, 90.0)),                         # one batch size, ragged core count
+    (4, 33, (1, 2, 5), 7, 1025, 500, True, (20.0, 300.0)),                   # one cell beyond a tile group
+    (2, 2, (1, 2), 2, 16383, 100, False, (5.0, 30.0)),                       # longest budget, 8 candidates
+    (64, 3, (1, 4), 2, 2500, 1000, False, (5.0, 60.0)),                      # most stages
+    (5, 64, (1, 2, 4, 8, 16, 32, 64, 128), 16, 4096, 250, False, (100.0, 900.0)),   # T a power of two
+    (6, 16, (1, 2, 4, 8), 64, 2056, 500, False, (200.0, 3000.0)),            # eight cells beyond the tiles
+    (3, 7, (2, 3), 5, 263, 1000, True, (10.0, 80.0)),
+]
+
+
+@pytest.mark.parametrize("shape", SHAPES, ids=[f"S{s[0]}_C{s[1]}_B{len(s[2])}_H{s[3]}_T{s[4]}" for s in SHAPES])
+def test_assorted_shapes(S, oracle_mod, shape, mode):
+    """Shapes at the edges of the supported ranges, every kernel mode, every table the mode exposes."""
+    n_stages, c_max, batches, h_max, T, bucket_us, vertical, (lo, hi) = shape
+    wl = W.random_tiny_workload(9000 + T + n_stages, 7, n_stages, c_max, batches, h_max, T, bucket_us=bucket_us,
+                                vertical=vertical, rate_lo=lo, rate_hi=hi)
+    ref = oracle_mod.solve_batch(wl, dumps=True)
+    gpu = _gpu_solve(S, wl, tables=True)
+    _assert_tables_equal(S, gpu, ref)
+    _assert_results_equal(gpu, ref)
+
+
 def test_single_instance_single_candidate(S, oracle_mod):
     wl = W.random_tiny_workload(5300, 1, 2, 1, (1,), 1, 100, rate_lo=5.0, rate_hi=6.0)
     ref = oracle_mod.solve_batch(wl)
