@@ -38,10 +38,23 @@ def _gpu_solve(S, wl, tables=False, horizontal=False):
 RESULT_KEYS = ("status", "total_cost", "latency_buckets", "h", "c", "b")
 
 
+def _diagnose(gpu, ref, idx):
+    """On a mismatch: is the CUDA answer at least optimal (same status and cost, so only a
+    tie was broken differently), or is it a different optimum altogether?"""
+    pick = (lambda a: a) if idx is None else (lambda a: a[idx])
+    st, cost = pick(gpu["status"]), pick(gpu["total_cost"])
+    same_opt = (st == ref["status"]) & (cost == ref["total_cost"])
+    cfg_equal = np.all(pick(gpu["h"]) == ref["h"], axis=1) & np.all(pick(gpu["c"]) == ref["c"], axis=1) \
+        & np.all(pick(gpu["b"]) == ref["b"], axis=1) & (pick(gpu["latency_buckets"]) == ref["latency_buckets"])
+    return (f"{int((~same_opt).sum())} instances with a different status or cost (optimality), "
+            f"{int((same_opt & ~cfg_equal).sum())} with the same cost but another configuration or latency (tie-break)")
+
+
 def _assert_results_equal(gpu, ref, idx=None):
     for k in RESULT_KEYS:
         a = gpu[k] if idx is None else gpu[k][idx]
-        assert np.array_equal(a, ref[k]), f"{k} differs at instances {np.argwhere(a != ref[k])[:5].tolist()}"
+        assert np.array_equal(a, ref[k]), (f"{k} differs at instances {np.argwhere(a != ref[k])[:5].tolist()}: "
+                                           + _diagnose(gpu, ref, idx))
 
 
 MODE = {"mode": 0}   # min-plus kernel under test: 0 packed 16-bit (default), 1 32-bit, 2 pruned
