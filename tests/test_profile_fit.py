@@ -47,6 +47,8 @@ def test_cuda_fit_matches_the_oracle():
     import torch
     if not torch.cuda.is_available():
         pytest.fail("the gpu tests need a CUDA device")
+    from paper_2407_14843_b200 import build
+    build.build_library()
     from paper_2407_14843_b200 import solver as S
     for n_models, c_max, batches in ((1, 4, (1,)), (37, 16, (1, 2, 4, 8, 16)), (640, 64, (1, 2, 4, 8, 16, 32, 64))):
         sb, sc, lat, _ = W.profile_samples(40 + n_models, n_models)

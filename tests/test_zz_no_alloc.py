@@ -33,6 +33,8 @@ def test_static_scratch_entry_point_matches_workspace_entry_point():
     import torch
     if not torch.cuda.is_available():
         pytest.fail("the gpu tests need a CUDA device")
+    from paper_2407_14843_b200 import build
+    build.build_library()
     from paper_2407_14843_b200 import solver as S
     # first call: joint problem, 3 stages, T = 500
     first = W.make_workload(1)
@@ -58,6 +60,8 @@ def test_static_scratch_entry_point_refuses_large_problems():
     import torch
     if not torch.cuda.is_available():
         pytest.fail("the gpu tests need a CUDA device")
+    from paper_2407_14843_b200 import build
+    build.build_library()
     from paper_2407_14843_b200 import solver as S
     wl = W.make_workload(4, 64)                          # 64 * 8 * 4032 * 8 B = 16.5 MB: fits
     prob = S.Problem.of_workload(wl)
