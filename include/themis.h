@@ -71,7 +71,9 @@ extern "C" {
 #define THEMIS_STATUS_INFEASIBLE 1
 #define THEMIS_STATUS_SPLIT 2          /* themis_vertical_fallback_batch: part of the load is served
                                           by the replicas in place, the rest needs extra replicas */
-#define THEMIS_STATUS_BAD_INPUT (-1)   /* lambda = 0, a latency <= 0 or replicas < 1 */
+#define THEMIS_STATUS_BAD_INPUT (-1)   /* lambda = 0, a latency <= 0, replicas < 1, replicas * c_max > 65535,
+                                          sum of replicas * c_max > THEMIS_MAX_TOTAL_COST, profile id out
+                                          of range */
 #define THEMIS_STATUS_TIMEOUT (-2)     /* a bounded on-device wait expired */
 
 /* value of an empty bucket in the G table of the workspace */
@@ -287,14 +289,19 @@ int themis_fit_profiles_batch(int32_t n_models, int32_t n_samples, const int32_t
                               int32_t *d_lat_us, int32_t *d_status, void *cuda_stream);
 
 /*
- * Integer-ALU throughput probe (not part of the method): every thread runs
- * `iters` rounds of 16 independent add-then-min updates, the operation pair of
- * the recurrence, in one of three instruction forms:
- *   mode 0: separate 32-bit add and unsigned min;
- *   mode 1: the fused add-min instruction (one instruction per update);
- *   mode 2: one add per update and one three-input min per two updates.
- * Launches `blocks` x `threads` and writes one word per thread to d_sink
- * (blocks*threads uint32).  Updates performed = blocks*threads*iters*16.
+ * Integer-ALU throughput probe (not part of the method, and the paper has no
+ * counterpart): every thread keeps 16 independent chains in registers and runs
+ * `iters` iterations of 4 rounds, each round one add-then-min update per chain (the
+ * operation pair of the recurrence), every update reading two values produced one
+ * round earlier.  Instruction form by mode:
+ *   0: separate 32-bit add and unsigned min;
+ *   1: fused 32-bit add-min (one instruction per update);
+ *   2: two adds and one three-input min per two updates;
+ *   3: fused add-min on packed 2 x 16-bit (two cell updates per instruction);
+ *   4: single-precision add and min.
+ * Launches `blocks` x `threads` (32..1024) and writes one word per thread to d_sink
+ * (blocks*threads uint32).  Updates performed = blocks * threads * iters * 64
+ * (x 2 cells in mode 3).
  */
 int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_sink,
                      void *cuda_stream);
