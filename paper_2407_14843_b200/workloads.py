@@ -305,3 +305,29 @@ def profile_samples(seed: int, n_models: int, noise: float = 0.02):
     clean = (true[:, 0:1] * b / c + true[:, 1:2] / c + true[:, 2:3] * b + true[:, 3:4])
     z = rand_normal(seed, 15, np.arange(n_models * b.size, dtype=np.uint64)).reshape(n_models, b.size)
     return sample_b, sample_c, clean * np.exp(noise * z), true
+
+
+def arbitrary_tables_workload(seed: int, n_instances: int, n_stages: int, c_max: int,
+                              batch_sizes: Sequence[int], h_max: int, T: int, bucket_us: int,
+                              flags: int, vertical: bool, lat_lo_us: int = 700, lat_hi_us: int = 90_000,
+                              rate_lo: float = 3.0, rate_hi: float = 400.0, repeat_prob: float = 0.3) -> Workload:
+    """Instances whose latency tables follow no model at all: every entry is an
+    independent draw in [lat_lo_us, lat_hi_us] microseconds (not monotone in cores or
+    batch size, not multiples of the bucket), with a share of entries copied from the
+    neighbouring core count so that equal latencies occur.  For robustness checks."""
+    shape = (n_instances, n_stages, c_max, len(batch_sizes))
+    idx = np.arange(int(np.prod(shape)), dtype=np.uint64)
+    lat = rand_int(seed, 21, idx, lat_lo_us, lat_hi_us).reshape(shape)
+    copy = rand_uniform(seed, 22, idx).reshape(shape) < repeat_prob
+    for c in range(1, c_max):
+        lat[:, :, c, :] = np.where(copy[:, :, c, :], lat[:, :, c - 1, :], lat[:, :, c, :])
+    rate = rand_uniform(seed, 4, np.arange(n_instances, dtype=np.uint64), rate_lo, rate_hi)
+    replicas = None
+    if vertical:
+        replicas = rand_int(seed, 8, np.arange(n_instances * n_stages, dtype=np.uint64), 1, h_max)
+        replicas = replicas.reshape(n_instances, n_stages).astype(np.int32)
+    return Workload(
+        name=f"arbitrary_{seed}", n_instances=n_instances, n_stages=n_stages, n_profiles=n_instances,
+        c_max=c_max, batch_sizes=tuple(batch_sizes), h_max=h_max, slo_us=T * bucket_us, bucket_us=bucket_us,
+        flags=flags, vertical=vertical, lat_us=np.ascontiguousarray(lat.astype(np.int32)),
+        profile_id=np.arange(n_instances, dtype=np.int32), lambda_mrps=_to_mrps(rate), replicas=replicas, seed=seed)

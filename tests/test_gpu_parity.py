@@ -291,6 +291,21 @@ def test_assorted_shapes(S, oracle_mod, shape, mode):
     _assert_results_equal(gpu, ref)
 
 
+@pytest.mark.parametrize("vertical", [False, True])
+@pytest.mark.parametrize("flags", [0, W.QUEUE_PER_REPLICA])
+def test_arbitrary_latency_tables(S, oracle_mod, flags, vertical, mode):
+    """Latency tables that follow no model (not monotone in cores or batch size, entries
+    repeated between neighbouring core counts, odd bucket widths, batch sizes that are not
+    powers of two): every table the mode exposes and every result."""
+    for seed, (bucket, T, batches, c_max, h_max) in enumerate([
+            (777, 400, (1, 3, 5, 6), 40, 9), (1300, 1100, (2, 7), 70, 5), (333, 2600, (1, 2, 3, 4, 9, 17), 17, 33)]):
+        wl = W.arbitrary_tables_workload(8100 + seed, 12, 2 + seed, c_max, batches, h_max, T, bucket, flags, vertical)
+        ref = oracle_mod.solve_batch(wl, dumps=True)
+        gpu = _gpu_solve(S, wl, tables=True)
+        _assert_tables_equal(S, gpu, ref)
+        _assert_results_equal(gpu, ref)
+
+
 def test_single_instance_single_candidate(S, oracle_mod):
     wl = W.random_tiny_workload(5300, 1, 2, 1, (1,), 1, 100, rate_lo=5.0, rate_hi=6.0)
     ref = oracle_mod.solve_batch(wl)

@@ -468,3 +468,22 @@ def test_full_queue_model_reduces_to_the_simplified_one():
                             assert max(Fraction(b - 1) / lam, second) == Fraction(b - 1) / lam
                             checked += 1
     assert checked > 500
+
+
+# ---------------------------------------------------------------- tables that follow no model
+
+@pytest.mark.parametrize("vertical", [False, True])
+@pytest.mark.parametrize("flags", [0, W.QUEUE_PER_REPLICA])
+def test_arbitrary_tables_vs_rational_brute_force(oracle_mod, flags, vertical):
+    """Latency entries drawn independently (not monotone in cores or batch size, odd
+    bucket widths, batch sizes that are not powers of two): DP oracle, exact-rational
+    brute force and the paper's scatter order agree."""
+    solved = 0
+    for seed, (bucket, T, batches) in enumerate([(777, 150, (1, 3, 5)), (1300, 90, (2, 7)), (250, 500, (1, 2, 3, 4))]):
+        wl = W.arbitrary_tables_workload(8000 + seed, 20, 1 + seed, 5, batches, 3, T, bucket, flags, vertical)
+        r = oracle_mod.solve_batch(wl)
+        for n in range(wl.n_instances):
+            _assert_same(r, n, pyref.solve_instance(wl, n), f"seed {seed} instance {n}")
+            _assert_same(r, n, oracle_mod.alg1_scatter(wl, n), f"scatter seed {seed} instance {n}")
+        solved += int((r["status"] == 0).sum())
+    assert solved > 10
