@@ -400,7 +400,9 @@ def run_ours(args):
         "metric": METRIC, "value": N_total * args.steps / (total_ms * 1e-3), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
         "ms_per_step_best": step_ms[0], "ms_per_step_median": step_ms[len(step_ms) // 2],
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        # arithmetic of the dominant kernel: packed pairs of unsigned 16-bit costs, or 32-bit keys
+        "dtype": "u16" if packed else "u32",
         "data": "synthetic", "config": workload_config(wl, args, world),
         "cell_updates_per_s": world * cells_per_launch * args.steps / (total_ms * 1e-3),
         "minplus_cell_updates_per_s_kernel": cells_per_launch / (minplus_ms * 1e-3),
