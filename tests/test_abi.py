@@ -109,3 +109,40 @@ def test_strerror(S):
     assert "workspace" in S.themis_strerror(-3)
     assert "CUDA" in S.themis_strerror(-4)
     assert "unknown" in S.themis_strerror(-99)
+
+
+def test_header_is_plain_c_and_links_from_c(S, tmp_path):
+    """include/themis.h compiles as strict C99 and a C program linked against the
+    library can call the host-side entry points (nothing is launched)."""
+    import subprocess
+    src = tmp_path / "use_themis.c"
+    src.write_text(r'''
+#include <stdio.h>
+#include <string.h>
+#include "themis.h"
+int main(void) {
+    themis_problem_t p;
+    themis_workspace_layout_t lay;
+    size_t bytes = 0;
+    memset(&p, 0, sizeof p);
+    p.n_instances = 10; p.n_stages = 5; p.n_profiles = 1; p.c_max = 16; p.n_batch = 3;
+    p.batch_sizes[0] = 1; p.batch_sizes[1] = 2; p.batch_sizes[2] = 4;
+    p.h_max = 8; p.slo_us = 1000000; p.bucket_us = 1000; p.flags = THEMIS_QUEUE_PER_REPLICA;
+    if (themis_version() != THEMIS_VERSION) return 1;
+    if (themis_workspace_bytes(&p, 0, &bytes) != THEMIS_OK || bytes == 0) return 2;
+    if (themis_workspace_layout(&p, 0, &lay) != THEMIS_OK || lay.T != 1000 || lay.row_pitch != 1024) return 3;
+    p.bucket_us = 0;
+    if (themis_workspace_bytes(&p, 0, &bytes) != THEMIS_E_INVALID_ARG) return 4;
+    if (strcmp(themis_strerror(THEMIS_OK), "ok") != 0) return 5;
+    printf("%lu\n", (unsigned long)lay.total_bytes);
+    return 0;
+}
+''')
+    exe = tmp_path / "use_themis"
+    lib_dir = os.path.dirname(S.LIB_PATH)
+    subprocess.check_call(["gcc", "-std=c99", "-pedantic", "-Wall", "-Wextra", "-Werror",
+                           "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe),
+                           "-L", lib_dir, "-l:libthemis.so", f"-Wl,-rpath,{lib_dir}"])
+    out = subprocess.check_output([str(exe)]).decode().strip()
+    assert int(out) == S.themis_workspace_bytes(_good(S, n_instances=10, n_stages=5, n_profiles=1, c_max=16,
+                                                      batch_sizes=(1, 2, 4), h_max=8, slo_us=1_000_000), False)
