@@ -206,6 +206,16 @@ int themis_solve_horizontal_batch(const themis_problem_t *problem, const int32_t
                                   void *cuda_stream);
 
 /*
+ * Stability test of the transition policy (Section "Transition", vertical to
+ * horizontal: when): the workload counts as stable when the horizontal solver
+ * returns the same configuration for the current and for the predicted arrival
+ * rate.  Given the results of two solves of the same N pipelines (device arrays),
+ *   d_stable[n] = 1 iff both have status 0 and equal (h, c, b) at every stage, else 0.
+ */
+int themis_configs_equal_batch(int32_t n_instances, int32_t n_stages, themis_result_t current,
+                               themis_result_t predicted, int32_t *d_stable, void *cuda_stream);
+
+/*
  * The two halves of the solvers, for checking and timing each step on its own.
  * themis_score_batch fills G and Garg of the workspace (candidate scoring: the
  * inner loops of Algorithm 1 with Eq. 4 and the throughput test of Eq. 6);

@@ -400,6 +400,17 @@ int themis_solve_horizontal_batch(const themis_problem_t *problem, const int32_t
                       workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int themis_configs_equal_batch(int32_t n_instances, int32_t n_stages, themis_result_t current,
+                               themis_result_t predicted, int32_t *d_stable, void *cuda_stream)
+{
+    if (n_instances < 1 || n_stages < 1 || !d_stable || !current.h || !current.c || !current.b || !current.status ||
+        !predicted.h || !predicted.c || !predicted.b || !predicted.status)
+        return THEMIS_E_INVALID_ARG;
+    cudaError_t e = launch_configs_equal(n_instances, n_stages, current, predicted, d_stable,
+                                         static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
+}
+
 int themis_score_batch(const themis_problem_t *problem, const int32_t *d_lat_us, const int32_t *d_profile_id,
                        const uint32_t *d_lambda_mrps, const int32_t *d_replicas, void *d_workspace,
                        size_t workspace_bytes, void *cuda_stream)

@@ -88,7 +88,26 @@ __global__ void fb_finish_kernel(const Params p, uint32_t res, const uint32_t *l
     }
 }
 
+// stable[n] = 1 iff both solves succeeded and chose the same (h, c, b) at every stage.
+__global__ void configs_equal_kernel(int N, int S, themis_result_t a, themis_result_t b, int32_t *stable)
+{
+    const int n = blockIdx.x * kThreads + threadIdx.x;
+    if (n >= N) return;
+    int same = a.status[n] == THEMIS_STATUS_OK && b.status[n] == THEMIS_STATUS_OK;
+    for (int s = 0; s < S && same; ++s) {
+        const size_t i = (size_t)n * S + s;
+        same = a.h[i] == b.h[i] && a.c[i] == b.c[i] && a.b[i] == b.b[i];
+    }
+    stable[n] = same;
+}
+
 }  // namespace
+
+cudaError_t launch_configs_equal(int N, int S, themis_result_t a, themis_result_t b, int32_t *stable, cudaStream_t st)
+{
+    configs_equal_kernel<<<(N + kThreads - 1) / kThreads, kThreads, 0, st>>>(N, S, a, b, stable);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_fb_init(int N, uint32_t res, const int32_t *status, const uint32_t *lambda, uint32_t *lo,
                            uint32_t *hi, int32_t *active, cudaStream_t st)

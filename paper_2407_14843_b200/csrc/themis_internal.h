@@ -81,6 +81,7 @@ cudaError_t launch_solve_sparse(const Params &p, cudaStream_t stream);
 constexpr size_t kMaxDynamicSmem = 227u * 1024u;
 // Dynamic shared memory of the pruned kernel for a row pitch; it cannot run above 227 KB.
 inline size_t pruned_smem_bytes(int pitch) { return sizeof(uint32_t) * (5u * (size_t)pitch + 4 + 32); }
+cudaError_t launch_configs_equal(int N, int S, themis_result_t a, themis_result_t b, int32_t *stable, cudaStream_t st);
 cudaError_t launch_fb_init(int N, uint32_t res, const int32_t *status, const uint32_t *lambda, uint32_t *lo,
                            uint32_t *hi, int32_t *active, cudaStream_t st);
 cudaError_t launch_fb_trial(int N, uint32_t res, const uint32_t *lo, const uint32_t *hi, const int32_t *active,

@@ -34,7 +34,7 @@ EXPORTS = (
     "themis_host_workspace_bytes", "themis_solve_batch_host", "themis_alu_probe",
     "themis_set_minplus_tile", "themis_solve_batch_static", "themis_set_minplus_mode",
     "themis_solve_horizontal_batch", "themis_fallback_workspace_bytes", "themis_vertical_fallback_batch",
-    "themis_fit_profiles_batch",
+    "themis_fit_profiles_batch", "themis_configs_equal_batch",
 )
 
 
@@ -106,6 +106,7 @@ def _load() -> ctypes.CDLL:
     lib.themis_minplus_batch.argtypes = [PP, vp, Result, vp, sz, vp]
     lib.themis_solve_batch_host.argtypes = [PP, vp, vp, vp, vp, Result, vp, sz, vp]
     lib.themis_solve_batch_static.argtypes = [PP, vp, vp, vp, vp, Result, vp]
+    lib.themis_configs_equal_batch.argtypes = [ctypes.c_int32, ctypes.c_int32, Result, Result, vp, vp]
     lib.themis_fit_profiles_batch.argtypes = [ctypes.c_int32, ctypes.c_int32, vp, vp, vp, ctypes.c_int32,
                                               ctypes.c_int32, vp, vp, vp, vp, vp]
     lib.themis_alu_probe.argtypes = [ctypes.c_int] * 4 + [vp, vp]
@@ -248,6 +249,14 @@ def themis_solve_batch_static(problem: Problem, lat_us, profile_id, lambda_mrps,
         ctypes.byref(problem), _dptr(lat_us, torch.int32, "lat_us"), _dptr(profile_id, torch.int32, "profile_id"),
         _dptr(lambda_mrps, torch.uint32, "lambda_mrps"), _dptr(replicas, torch.int32, "replicas"), _result(out),
         _stream()), "themis_solve_batch_static")
+
+
+def themis_configs_equal_batch(current: dict, predicted: dict, stable) -> None:
+    """``stable[n] = 1`` iff both result sets are solved and equal at every stage."""
+    n, s = current["h"].shape
+    _check(_lib.themis_configs_equal_batch(n, s, _result(current), _result(predicted),
+                                           _dptr(stable, torch.int32, "stable"), _stream()),
+           "themis_configs_equal_batch")
 
 
 def themis_fit_profiles_batch(sample_b, sample_c, latency_ms, c_max: int, batch_sizes, coeffs, lat_us, status) -> None:

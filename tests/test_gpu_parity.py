@@ -233,6 +233,25 @@ def test_vertical_fallback(S, oracle_mod, res, mode):
     assert (st[ref["status"] == 2] == S.STATUS_BAD_INPUT).all() and (st[ref["status"] == 0] == 0).all()
 
 
+def test_stability_test_of_the_transition_policy(S, oracle_mod):
+    """Horizontal solves at the current and at a predicted rate, compared on the device:
+    stable exactly where the oracle's two configurations coincide."""
+    import torch
+    wl = W.random_tiny_workload(7500, 200, 3, 1, (1, 2, 4, 8), 40, 260, rate_lo=20.0, rate_hi=300.0)
+    growth = 1.0 + 0.3 * W.rand_uniform(7501, 1, np.arange(200, dtype=np.uint64))      # up to 30 % more load
+    pred = dataclasses.replace(wl, lambda_mrps=(wl.lambda_mrps * growth).astype(np.uint32))
+    now_out, _ = S.solve(wl, horizontal=True)
+    pred_out, _ = S.solve(pred, horizontal=True)
+    stable = torch.empty(200, dtype=torch.int32, device="cuda")
+    S.themis_configs_equal_batch(now_out, pred_out, stable)
+    torch.cuda.synchronize()
+    a, b = oracle_mod.solve_batch(wl, horizontal=True), oracle_mod.solve_batch(pred, horizontal=True)
+    expect = (a["status"] == 0) & (b["status"] == 0) & np.all(a["h"] == b["h"], axis=1) \
+        & np.all(a["b"] == b["b"], axis=1) & np.all(a["c"] == b["c"], axis=1)
+    assert np.array_equal(stable.cpu().numpy().astype(bool), expect)
+    assert expect.any() and (~expect).any()
+
+
 # ---------------------------------------------------------------- edge cases
 
 @pytest.mark.parametrize("T", [1, 2, 31, 32, 33, 127, 128, 131, 135, 136, 255, 256, 257, 263, 264, 511, 512, 1024, 1031,
