@@ -316,8 +316,9 @@ int themis_fit_profiles_batch(int32_t n_models, int32_t n_samples, const int32_t
 int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_sink,
                      void *cuda_stream);
 
-/* Which min-plus kernel themis_minplus_batch and the solvers run.  Results do not
- * depend on it; the layout of the A rows of the workspace does.
+/* Which min-plus kernel themis_minplus_batch and the solvers run (an implementation
+ * choice; the paper has no counterpart).  Results do not depend on it; what the rows
+ * of the workspace hold does.
  *   0 (default): packed 16-bit kernel (two budget cells per register).  The A
  *      rows then hold the prefix tables themselves, uint16 F_s[t] with
  *      0x7FFF = unreachable or >= 32767, and the backtrack recovers the argmin
@@ -340,12 +341,12 @@ int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_s
  *      shared memory (about 12 * row_pitch bytes plus tables) does not fit. */
 int themis_set_minplus_mode(int mode);
 
-/* Tuning knob of the dense min-plus kernels: consecutive budget cells per thread
+/* Tuning knob of the dense min-plus kernels (no counterpart in the paper): consecutive budget cells per thread
  * (4, 8 or 16; the 32-bit kernel treats 4 as its default); 0 restores the built-in
  * choice.  Results do not depend on it. */
 int themis_set_minplus_tile(int cells_per_thread);
 
-/* Text for a return code; for THEMIS_E_CUDA includes the last CUDA error seen by
+/* Library housekeeping (no counterpart in the paper).  Text for a return code; for THEMIS_E_CUDA includes the last CUDA error seen by
  * the calling thread.  The pointer stays valid until the thread's next call. */
 const char *themis_strerror(int code);
 int themis_version(void);
