@@ -59,6 +59,8 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--alu-probe", action="store_true",
+                    help="only run the integer-ALU probe in its five instruction forms and print the rates")
     ap.add_argument("--minplus-mode", type=int, default=0, choices=[0, 1],
                     help="0: packed 16-bit min-plus kernel (default); 1: 32-bit kernel")
     ap.add_argument("--pruned-steps", type=int, default=5,
@@ -220,7 +222,7 @@ class ClockSampler:
 def probe_alu_peak(solver, torch, mode):
     """Add-min throughput sustained by themis_alu_probe in TOP/s (two operations
     per cell update): mode 1 = fused 32-bit add-min, mode 3 = packed 2 x 16-bit."""
-    blocks, threads, iters = N_SMS * 8, 256, 20000          # about 0.1 s per form
+    blocks, threads, iters = N_SMS * 8, 256, 20000          # about 20 ms per form
     cells_per_update = 2 if mode == 3 else 1
     sink = torch.empty(blocks * threads, dtype=torch.uint32, device="cuda")
     solver.themis_alu_probe(mode, blocks, threads, 50, sink)
@@ -438,9 +440,40 @@ def run_ours(args):
     print(json.dumps(line), flush=True)
 
 
+def run_alu_probe():
+    """Rates of themis_alu_probe in all five instruction forms (updates per SM per clock at
+    the boost clock, and TOP/s counting two operations per cell update)."""
+    import torch
+    from paper_2407_14843_b200 import build as _build
+    _build.build_library()
+    from paper_2407_14843_b200 import solver
+    torch.cuda.set_device(0)
+    forms = {0: "32-bit add, then unsigned min", 1: "fused 32-bit add-min", 2: "two adds + one three-input min per two updates",
+             3: "fused add-min on packed 2 x 16-bit", 4: "single-precision add, then min"}
+    blocks, threads, iters = N_SMS * 8, 256, 20000
+    sink = torch.empty(blocks * threads, dtype=torch.uint32, device="cuda")
+    out = {}
+    for mode, what in forms.items():
+        solver.themis_alu_probe(mode, blocks, threads, 50, sink)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        solver.themis_alu_probe(mode, blocks, threads, iters, sink)
+        b.record()
+        torch.cuda.synchronize()
+        cells = (2 if mode == 3 else 1) * blocks * threads * iters * 64
+        rate = cells / (a.elapsed_time(b) * 1e-3)
+        out[f"mode{mode}"] = {"form": what, "ms": a.elapsed_time(b), "cell_updates_per_s": rate,
+                              "tops": 2.0 * rate / 1e12,
+                              "cell_updates_per_sm_per_clock_at_1965mhz": rate / N_SMS / (SM_GHZ * 1e9)}
+    print(json.dumps({"alu_probe": out, "derived_peak_tops": {"int32": ALU_PEAK_TOPS_INT32,
+                                                              "int16x2": ALU_PEAK_TOPS_INT16X2}}), flush=True)
+
+
 def main():
     args = parse_args()
-    if args.impl == "reference":
+    if args.alu_probe:
+        run_alu_probe()
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
