@@ -63,6 +63,8 @@ def parse_args():
                     help="only run the integer-ALU probe in its five instruction forms and print the rates")
     ap.add_argument("--minplus-mode", type=int, default=0, choices=[0, 1],
                     help="0: packed 16-bit min-plus kernel (default); 1: 32-bit kernel")
+    ap.add_argument("--minplus-tile", type=int, default=0, choices=[0, 4, 8, 16],
+                    help="cells per thread tile of the recurrence kernels (0: the library's choice)")
     ap.add_argument("--pruned-steps", type=int, default=5,
                     help="extra steps with the recurrence restricted to undominated entries (0: skip)")
     return ap.parse_args()
@@ -269,6 +271,7 @@ def run_ours(args):
     from paper_2407_14843_b200 import solver
 
     solver.themis_set_minplus_mode(args.minplus_mode)
+    solver.themis_set_minplus_tile(args.minplus_tile)
     packed = args.minplus_mode == 0
     prob = solver.Problem.of_workload(wl)
     dev = solver.workload_to_device(wl)

@@ -39,7 +39,8 @@ struct Params {
     int32_t horizontal; // 1: Algorithm 2, one candidate per batch size with the fewest replicas
                         //    that sustain lambda; candidate index = batch index, stage cost = h
     int32_t only_flagged;  // wide min-plus kernel: solve only instances flagged kFlagNeedsWide
-    uint8_t warp_group[32];  // min-plus kernels: tile group (32 tiles) owned by each warp
+    uint8_t warp_group[32];  // 32-bit min-plus kernel: tile group (32 tiles) owned by each warp
+    int32_t n_half_groups;   // packed min-plus kernel: half-groups of 16 tiles
     const int32_t *lat_us;
     const int32_t *profile_id;
     const uint32_t *lambda_mrps;

@@ -23,6 +23,14 @@
 // backtrack recovers, stage by stage along the optimal path only, the lowest l
 // with F_{s-1}[t-l] + G_s[l] == F_s[t] by a block-wide scan.
 //
+// Folding.  Tiles are grouped in half-groups of 16 (one per half-warp).  Column length
+// grows with the tile index, and all lanes of a half-warp run to their half-group's
+// longest column, so every half-warp takes a long half-group and then a short one,
+// (last, first), (last-1, second), ...: all half-warps of the block do the same number
+// of chunk steps, and the two halves of a warp may stand at different l (two broadcast
+// addresses instead of one).  A finished tile's result waits in registers for the stage's
+// barrier; only the word that spills into the next tile goes through shared memory.
+//
 // Saturation.  If the best total is 0x7FFF the instance is either infeasible
 // (decided exactly: the fastest configurations of all stages do not fit the
 // budget) or too expensive for 16 bits; the latter is flagged and redone by the
@@ -129,28 +137,35 @@ minplus16_kernel(const Params p)
     const int NT = blockDim.x;
     const int n_warps = NT >> 5;
     const int T = p.T, pitch = p.pitch, S = p.prob.n_stages;
-    const int Tc = NT * R;                                // cells covered by the tiles
-    const int Tp = EXTRA ? max(Tc, pitch) : Tc;           // length of the G buffers (Tc >= pitch without extras)
+    const int NHG = p.n_half_groups;                      // half-groups of 16 tiles
+    const int n_tiles = NHG * 16;
+    const int Tc = n_tiles * R;                           // cells covered by the tiles
+    const int Tp = max(Tc, pitch);                        // length of the G buffers
     const int n_extra = EXTRA ? max(0, T + 1 - Tc) : 0;   // cells beyond the tiles, at most kMaxExtra
+    // The tiling is right-aligned: the first n_dummy tiles lie in front of cell 0 and stay
+    // "unreachable", so that the columns the padding adds are the shortest, not the longest.
+    const int n_dummy = max(0, Tc - (T + 1)) / R;
 
-    uint32_t *Fw = smem;                                  // (kPadChunks + NT) chunks of CS words
-    uint32_t *Gbuf0 = Fw + (kPadChunks + NT) * CS;
+    uint32_t *Fw = smem;                                  // (kPadChunks + n_tiles) chunks of CS words
+    uint32_t *Gbuf0 = Fw + (kPadChunks + n_tiles) * CS;
     uint32_t *Gbuf1 = Gbuf0 + Tp;
-    uint64_t *mbar = reinterpret_cast<uint64_t *>(Gbuf1 + Tp);
+    uint32_t *xchg = Gbuf1 + Tp;                          // n_tiles words: every tile's last odd-l word
+    uint64_t *mbar = reinterpret_cast<uint64_t *>(xchg + n_tiles);
     uint32_t *red = reinterpret_cast<uint32_t *>(mbar + 2);   // 32 words
-    uint32_t *xchg = red + 32;                                // 32 words: last accp word of each warp
-    uint32_t *stage_lmin = xchg + 32;                         // 64 words: first reachable l of every G_s
+    uint32_t *stage_lmin = red + 32;                          // 64 words: first reachable l of every G_s
     uint32_t *fx_prev = stage_lmin + THEMIS_MAX_STAGES;       // kMaxExtra words: F_{s-1} at the extra cells
     uint32_t *fx_acc = fx_prev + kMaxExtra;                   // kMaxExtra words: F_s at the extra cells, building
 
-    // Which tile (R consecutive cells) this thread owns: lanes keep consecutive tiles,
-    // warps take the tile groups the host dealt them (see assign_warp_groups).
-    const int tile = ((int)p.warp_group[tid >> 5] << 5) | (tid & 31);
-    const int t0 = tile * R;
-    uint32_t *my_chunk = Fw + (kPadChunks + tile) * CS;
+    // The two tiles of this thread: its half-warp takes half-group NHG-1-slot (long columns)
+    // first and half-group slot (short columns) second; the middle one, if any, stands alone.
+    const int slot = tid >> 4, lane16 = tid & 15;
+    const int hg_a = NHG - 1 - slot, hg_b = slot;
+    const bool has_a = hg_a >= hg_b, has_b = hg_b < hg_a;
+    const int tile_a = hg_a * 16 + lane16, tile_b = hg_b * 16 + lane16;
     const uint32_t row_bytes = (uint32_t)pitch * 4u;
     const int32_t *G_inst = p.G + (size_t)n * S * pitch;
     uint16_t *F16_inst = p.A + (size_t)n * S * pitch;     // prefix tables F_s as uint16 rows
+    auto chunk_of = [&](int tile) -> uint32_t * { return Fw + (kPadChunks + tile) * CS; };
 
     int32_t *h_o = p.out.h + (size_t)n * S, *c_o = p.out.c + (size_t)n * S, *b_o = p.out.b + (size_t)n * S;
     auto write_unsolved = [&](int status) {
@@ -188,10 +203,11 @@ minplus16_kernel(const Params p)
     int failed = 0;                                       // a bounded wait ran out
     int pend0 = 0, pend1 = S > 1 ? 0 : -1;                // phase parity of a copy in flight, or -1
 
-    // Stores the thread's H words of F_s to shared memory and to the uint16 table.
-    auto store_chunk = [&](const uint32_t (&w)[H], int s) {
-        store_words<H>(w, my_chunk);
-        if (t0 + R <= pitch)
+    // Stores a tile's H words of F_s to shared memory and to the uint16 table.
+    auto store_chunk = [&](int tile, const uint32_t (&w)[H], int s) {
+        store_words<H>(w, chunk_of(tile));
+        const int t0 = (tile - n_dummy) * R;
+        if (t0 >= 0 && t0 + R <= pitch)
             store_words<H>(w, reinterpret_cast<uint32_t *>(F16_inst + (size_t)s * pitch + t0));
     };
 
@@ -203,17 +219,24 @@ minplus16_kernel(const Params p)
         if ((tid & 31) == 0 && first != 0xFFFFFFFFu) atomicMin(&stage_lmin[s], first);
     };
     {
-        uint32_t w[H], first = 0xFFFFFFFFu;
+        uint32_t first = 0xFFFFFFFFu;
+        auto init_tile = [&](int tile) {
+            const int t0 = (tile - n_dummy) * R;
+            uint32_t w[H];
 #pragma unroll
-        for (int r = H - 1; r >= 0; --r) {
-            // raw costs; entries beyond the loaded row hold kInf16x2, far above kInf16
-            const uint32_t lo = min(Gbuf0[t0 + 2 * r], kInf16), hi = min(Gbuf0[t0 + 2 * r + 1], kInf16);
-            w[r] = lo | (hi << 16);
-            if (hi < kInf16) first = (uint32_t)(t0 + 2 * r + 1);
-            if (lo < kInf16) first = (uint32_t)(t0 + 2 * r);
-        }
+            for (int r = H - 1; r >= 0; --r) {
+                // raw costs; entries beyond the loaded row hold kInf16x2, far above kInf16
+                const uint32_t lo = t0 < 0 ? kInf16 : min(Gbuf0[t0 + 2 * r], kInf16);
+                const uint32_t hi = t0 < 0 ? kInf16 : min(Gbuf0[t0 + 2 * r + 1], kInf16);
+                w[r] = lo | (hi << 16);
+                if (hi < kInf16) first = min(first, (uint32_t)(t0 + 2 * r + 1));
+                if (lo < kInf16) first = min(first, (uint32_t)(t0 + 2 * r));
+            }
+            store_chunk(tile, w, 0);
+        };
+        if (has_a) init_tile(tile_a);
+        if (has_b) init_tile(tile_b);
         note_first_reachable(first, 0);
-        store_chunk(w, 0);
         if (tid < n_extra) {
             const uint32_t v = min(Gbuf0[Tc + tid], kInf16);
             fx_prev[tid] = v;
@@ -223,7 +246,7 @@ minplus16_kernel(const Params p)
     failed = __syncthreads_or(failed);
     // Half-word i (< Tc) of the prefix table in shared memory.
     auto f_at = [&](int i) -> uint32_t {
-        const uint32_t w = Fw[(kPadChunks + i / R) * CS + ((i % R) >> 1)];
+        const uint32_t w = Fw[(kPadChunks + n_dummy + i / R) * CS + ((i % R) >> 1)];
         return (i & 1) ? (w >> 16) : (w & 0xFFFFu);
     };
     // Lowest reachable budget of the prefix F_{s-1} (0xFFFFFFFF: nothing reachable).  Everything
@@ -239,13 +262,16 @@ minplus16_kernel(const Params p)
         // raw costs -> saturated cost duplicated into both half-words, in place
         {
             uint32_t first = 0xFFFFFFFFu;
-            if (t0 < pitch) {
+            for (int l4 = tid * 4; l4 < pitch; l4 += NT * 4) {
+                uint4 v4 = *reinterpret_cast<const uint4 *>(Gk + l4);
+                uint32_t *v = reinterpret_cast<uint32_t *>(&v4);
 #pragma unroll
-                for (int r = R - 1; r >= 0; --r) {
-                    const uint32_t v = min(Gk[t0 + r], kInf16);
-                    Gk[t0 + r] = v | (v << 16);
-                    if (v < kInf16) first = (uint32_t)(t0 + r);
+                for (int i = 3; i >= 0; --i) {
+                    const uint32_t c = min(v[i], kInf16);
+                    v[i] = c | (c << 16);
+                    if (c < kInf16) first = min(first, (uint32_t)(l4 + i));
                 }
+                *reinterpret_cast<uint4 *>(Gk + l4) = v4;
             }
             note_first_reachable(first, s);
             if (EXTRA && tid < kMaxExtra) fx_acc[tid] = 0xFFFFFFFFu;
@@ -263,54 +289,91 @@ minplus16_kernel(const Params p)
         }
 
         uint32_t acc[H], accp[H], wa[H], wb[H];
-#pragma unroll
-        for (int r = 0; r < H; ++r) { acc[r] = 0xFFFFFFFFu; accp[r] = 0xFFFFFFFFu; }
-        // All lanes of a warp walk the same l so that G is a broadcast; lanes that run
+        // All lanes of a half-warp walk the same l so that G is a broadcast; lanes that run
         // past their own range read the "unreachable" chunks in front of F[0].  Chunks of
         // l below G_s's first reachable entry, and chunks that only meet F_{s-1} below its
         // first reachable budget, are skipped (whole steps of U chunks, block-uniform).
         const uint32_t g_min = stage_lmin[s];
         const bool dead = g_min == 0xFFFFFFFFu || prefix_min == 0xFFFFFFFFu;
         const int q_lo = dead ? 0 : (int)(g_min / R) & ~(U - 1);
-        const int q_hi = dead ? -1 : (tile | 31) - ((int)(prefix_min / R) & ~(U - 1));
-        if (q_lo <= q_hi) {
-            const uint32_t *f_hi = my_chunk - q_lo * CS;  // chunk tile - q_lo: at worst a pad chunk
+        const int q_shift = dead ? 0 : ((int)(prefix_min / R) + n_dummy) & ~(U - 1);   // in tiles
+        auto steps_of = [&](int tile) { return dead ? 0 : max(0, (tile | 15) - q_shift - q_lo + 1); };
+        const int steps_a = has_a ? steps_of(tile_a) : 0, steps_b = has_b ? steps_of(tile_b) : 0;
+        const uint32_t *f_lo = Fw, *g = Gk;
+        auto begin_tile = [&](int tile) {
 #pragma unroll
-            for (int r = 0; r < H; ++r) wa[r] = f_hi[r];
-            const uint32_t *f_lo = f_hi - CS;
-            const uint32_t *g = Gk + q_lo * R;
-            for (int q = q_lo; q <= q_hi; q += U) {
+            for (int r = 0; r < H; ++r) { acc[r] = 0xFFFFFFFFu; accp[r] = 0xFFFFFFFFu; }
+            const uint32_t *f_hi = chunk_of(tile) - q_lo * CS;   // chunk tile - q_lo: at worst a pad chunk
+            if (steps_of(tile) > 0) load_words<H>(wa, f_hi);
+            f_lo = f_hi - CS;
+            g = Gk + q_lo * R;
+        };
+        // Parks a finished tile in registers: cell 2j comes from acc[j].lo and accp[j-1].hi, cell
+        // 2j+1 from acc[j].hi and accp[j].lo.  The last odd-l word also holds cell 0 of the tile to
+        // the right, which picks it up from shared memory after the barrier.
+        uint32_t res_a[H], res_b[H];
+        auto park_tile = [&](uint32_t (&dst)[H], int tile) {
 #pragma unroll
-                for (int u = 0; u < U; u += 2) {
-                    chunk_step16<R>(wa, wb, acc, accp, f_lo - u * CS, g + u * R);
-                    chunk_step16<R>(wb, wa, acc, accp, f_lo - (u + 1) * CS, g + (u + 1) * R);
+            for (int r = 0; r < H; ++r)
+                dst[r] = __vminu2(acc[r], __byte_perm(r == 0 ? 0xFFFFFFFFu : accp[r - 1], accp[r], 0x5432));
+            xchg[tile] = accp[H - 1];
+        };
+        int phase = 0, remaining = steps_a;          // phase 0: first tile, 1: second tile, 2: done
+        if (has_a) begin_tile(tile_a);
+        auto advance = [&]() {
+            while (phase < 2 && remaining == 0) {
+                if (phase == 0 && has_a) park_tile(res_a, tile_a);
+                if (phase == 1 && has_b) park_tile(res_b, tile_b);
+                ++phase;
+                if (phase == 1 && has_b) { begin_tile(tile_b); remaining = steps_b; }
+            }
+        };
+        advance();
+        // Segments with a warp-uniform trip count: up to the next moment at which a half-warp
+        // finishes a tile (both halves on long tiles; one long, one short; both on short tiles).
+        for (;;) {
+            const unsigned n_seg = __reduce_min_sync(0xFFFFFFFFu, remaining > 0 ? (unsigned)remaining : 0xFFFFFFFFu);
+            if (n_seg == 0xFFFFFFFFu) break;
+            if (remaining > 0) {
+                for (unsigned q = 0; q < n_seg; q += U) {
+#pragma unroll
+                    for (int u = 0; u < U; u += 2) {
+                        chunk_step16<R>(wa, wb, acc, accp, f_lo - u * CS, g + u * R);
+                        chunk_step16<R>(wb, wa, acc, accp, f_lo - (u + 1) * CS, g + (u + 1) * R);
+                    }
+                    f_lo -= U * CS;
+                    g += U * R;
                 }
-                f_lo -= U * CS;
-                g += U * R;
+                remaining -= (int)n_seg;
+                advance();
             }
         }
         prefix_min = dead ? 0xFFFFFFFFu : prefix_min + g_min;
         if (EXTRA && n_extra > 0) {
             // Extra cells t = Tc + e: this thread's share of min_l F_{s-1}[t-l] + G_s[l] is its own
-            // tile's l range; thread 0 adds l >= Tc (those entries of G are still raw costs).
+            // tile's l range; thread 0 adds l >= Tc.
             uint32_t ex[kMaxExtra];
 #pragma unroll
             for (int e = 0; e < kMaxExtra; ++e) ex[e] = 0xFFFFFFFFu;
-            for (int r = 0; r < R; ++r) {
-                const int l = t0 + r;
-                const uint32_t g = Gk[l] & 0xFFFFu;
+            auto share_of_tile = [&](int tile) {
+                for (int r = 0; r < R; ++r) {
+                    const int l = tile * R + r;
+                    const uint32_t gl = Gk[l] & 0xFFFFu;
 #pragma unroll
-                for (int e = 0; e < kMaxExtra; ++e)
-                    if (e < n_extra) {
-                        const int i = Tc + e - l;             // >= 1
-                        ex[e] = min(ex[e], (i < Tc ? f_at(i) : fx_prev[i - Tc]) + g);
-                    }
-            }
+                    for (int e = 0; e < kMaxExtra; ++e)
+                        if (e < n_extra) {
+                            const int i = Tc + e - l;         // >= 1
+                            ex[e] = min(ex[e], (i < Tc ? f_at(i) : fx_prev[i - Tc]) + gl);
+                        }
+                }
+            };
+            if (has_a) share_of_tile(tile_a);
+            if (has_b) share_of_tile(tile_b);
             if (tid == 0) {
 #pragma unroll
                 for (int e = 0; e < kMaxExtra; ++e)
                     for (int l = Tc; l <= Tc + e && e < n_extra; ++l)
-                        ex[e] = min(ex[e], f_at(Tc + e - l) + min(Gk[l], kInf16));
+                        ex[e] = min(ex[e], f_at(Tc + e - l) + (Gk[l] & 0xFFFFu));
             }
 #pragma unroll
             for (int e = 0; e < kMaxExtra; ++e)
@@ -319,19 +382,17 @@ minplus16_kernel(const Params p)
                     if ((tid & 31) == 0) atomicMin(&fx_acc[e], m);
                 }
         }
-        if ((tid & 31) == 31) xchg[tile >> 5] = accp[H - 1];
-        __syncthreads();                                  // every read of F_{s-1} is done
+        __syncthreads();                                  // every read of F_{s-1} is done, every tile parked
 
-        // merge: cell 2j comes from acc[j].lo and accp[j-1].hi, cell 2j+1 from acc[j].hi and accp[j].lo
-        uint32_t left = __shfl_up_sync(0xFFFFFFFFu, accp[H - 1], 1);
-        if ((tid & 31) == 0) left = tile == 0 ? 0xFFFFFFFFu : xchg[(tile >> 5) - 1];
-        uint32_t w[H];
+        auto finish_tile = [&](uint32_t (&w)[H], int tile) {
+            const uint32_t left = tile == 0 ? 0xFFFFFFFFu : xchg[tile - 1];
+            w[0] = __vminu2(w[0], __byte_perm(left, 0xFFFFFFFFu, 0x5432));
 #pragma unroll
-        for (int r = 0; r < H; ++r) {
-            const uint32_t odd = __byte_perm(r == 0 ? left : accp[r - 1], accp[r], 0x5432);
-            w[r] = __vminu2(__vminu2(acc[r], odd), kInf16x2);
-        }
-        store_chunk(w, s);
+            for (int r = 0; r < H; ++r) w[r] = __vminu2(w[r], kInf16x2);
+            store_chunk(tile, w, s);
+        };
+        if (has_a) finish_tile(res_a, tile_a);
+        if (has_b) finish_tile(res_b, tile_b);
         if (tid < n_extra) {                              // every share arrived before the barrier above
             const uint32_t v = min(fx_acc[tid], kInf16);
             fx_prev[tid] = v;
@@ -350,13 +411,19 @@ minplus16_kernel(const Params p)
 
     // final scan: cheapest total, lowest total latency among equals
     uint32_t best = 0xFFFFFFFFu;
+    auto scan_tile = [&](int tile) {
+        const uint32_t *chunk = chunk_of(tile);
 #pragma unroll
-    for (int r = 0; r < H; ++r) {
-        const uint32_t w = my_chunk[r];
-        const int t = t0 + 2 * r;
-        if (t <= T) best = min(best, ((w & 0xFFFFu) << 16) | (uint32_t)t);
-        if (t + 1 <= T) best = min(best, (w & 0xFFFF0000u) | (uint32_t)(t + 1));
-    }
+        for (int r = 0; r < H; ++r) {
+            const uint32_t w = chunk[r];
+            const int t = (tile - n_dummy) * R + 2 * r;
+            if (t < 0) continue;
+            if (t <= T) best = min(best, ((w & 0xFFFFu) << 16) | (uint32_t)t);
+            if (t + 1 <= T) best = min(best, (w & 0xFFFF0000u) | (uint32_t)(t + 1));
+        }
+    };
+    if (has_a) scan_tile(tile_a);
+    if (has_b) scan_tile(tile_b);
     if (tid < n_extra) best = min(best, (fx_prev[tid] << 16) | (uint32_t)(Tc + tid));
     best = block_min(best, red, tid, n_warps);
     const uint32_t best_cost = best >> 16;
@@ -384,59 +451,91 @@ minplus16_kernel(const Params p)
     // last prefix table as int32 (same table the 32-bit kernel leaves)
     {
         int32_t *F_row = p.F + (size_t)n * pitch;
+        auto write_tile = [&](int tile) {
+            const uint32_t *chunk = chunk_of(tile);
 #pragma unroll
-        for (int r = 0; r < H; ++r) {
-            const uint32_t w = my_chunk[r];
-            const int t = t0 + 2 * r;
-            if (t < pitch) {
-                F_row[t] = (w & 0xFFFFu) >= kInf16 ? THEMIS_G_INF : (int32_t)(w & 0xFFFFu);
-                F_row[t + 1] = (w >> 16) >= kInf16 ? THEMIS_G_INF : (int32_t)(w >> 16);
+            for (int r = 0; r < H; ++r) {
+                const uint32_t w = chunk[r];
+                const int t = (tile - n_dummy) * R + 2 * r;
+                if (t >= 0 && t < pitch) {
+                    F_row[t] = (w & 0xFFFFu) >= kInf16 ? THEMIS_G_INF : (int32_t)(w & 0xFFFFu);
+                    F_row[t + 1] = (w >> 16) >= kInf16 ? THEMIS_G_INF : (int32_t)(w >> 16);
+                }
             }
-        }
+        };
+        if (has_a) write_tile(tile_a);
+        if (has_b) write_tile(tile_b);
     }
 
     if (tid < n_extra)
         p.F[(size_t)n * pitch + Tc + tid] = fx_prev[tid] >= kInf16 ? THEMIS_G_INF : (int32_t)fx_prev[tid];
 
-    // backtrack along the optimal path: lowest l with F_{s-1}[t-l] + G_s[l] == F_s[t]
+    // backtrack along the optimal path: lowest l with F_{s-1}[t-l] + G_s[l] == F_s[t].
+    // The block scans l upward, kScanGroups * 4 * NT values a round (four consecutive l per
+    // thread and group: one 16-byte load of G), and stops at the first round with a match.
+    // The reduction key (l << 16 | F_{s-1}[t-l]) brings the next stage's target along;
+    // the two reduction buffers alternate, so a round costs one barrier.
+    constexpr int kScanGroups = 2;
     int t = tstar;
     uint32_t target = best_cost;
-    for (int s = S - 1; s >= 1; --s) {
+    uint32_t *red_alt = stage_lmin;                       // the stage minima are no longer needed
+    uint32_t *ell_of = Gbuf0;                             // the G buffers are free: l_s of the path
+    int round = 0;
+    for (int s = S - 1; s >= 1 && !failed; --s) {
         const int32_t *G_row = G_inst + (size_t)s * pitch;
         const uint16_t *Fprev = F16_inst + (size_t)(s - 1) * pitch;
-        uint32_t cand = 0xFFFFFFFFu;
-        for (int l = tid; l <= t; l += NT) {
-            const uint32_t g = min((uint32_t)G_row[l], kInf16);
-            if ((uint32_t)Fprev[t - l] + g == target) { cand = (uint32_t)l; break; }
+        uint32_t key = 0xFFFFFFFFu;
+        for (int base = 0; base <= t; base += kScanGroups * 4 * NT) {
+            uint32_t cand = 0xFFFFFFFFu;
+#pragma unroll
+            for (int k = kScanGroups - 1; k >= 0; --k) {
+                const int l4 = base + (k * NT + tid) * 4;
+                if (l4 <= t) {
+                    const int4 g4 = *reinterpret_cast<const int4 *>(G_row + l4);   // pitch covers l4 + 3
+                    const int32_t gv[4] = {g4.x, g4.y, g4.z, g4.w};
+#pragma unroll
+                    for (int i = 3; i >= 0; --i)
+                        if (l4 + i <= t) {
+                            const uint32_t f = Fprev[t - l4 - i];
+                            if (f + min((uint32_t)gv[i], kInf16) == target) cand = ((uint32_t)(l4 + i) << 16) | f;
+                        }
+                }
+            }
+            cand = __reduce_min_sync(0xFFFFFFFFu, cand);
+            uint32_t *rbuf = (round++ & 1) ? red_alt : red;
+            if ((tid & 31) == 0) rbuf[tid >> 5] = cand;
+            __syncthreads();
+            key = rbuf[0];
+            for (int w = 1; w < n_warps; ++w) key = min(key, rbuf[w]);
+            if (key != 0xFFFFFFFFu) break;
         }
-        const uint32_t ell = block_min(cand, red, tid, n_warps);
-        if (ell > (uint32_t)t) { failed = 1; break; }     // cannot happen for consistent tables
-        t -= (int)ell;
-        target = Fprev[t];
-        if (tid == 0) {
-            const int idx = (int)p.Garg[((size_t)n * S + s) * pitch + ell];
-            const int C = p.prob.c_max, NB = p.prob.n_batch;
-            const int bi = idx % NB, rest = idx / NB;
-            b_o[s] = p.prob.batch_sizes[bi];
-            c_o[s] = rest % C + 1;
-            h_o[s] = p.vertical ? p.replicas[(size_t)n * S + s]
-                       : p.horizontal ? G_inst[(size_t)s * pitch + ell] : rest / C + 1;
-        }
+        if (key == 0xFFFFFFFFu) { failed = 1; break; }    // cannot happen for consistent tables
+        const int ell = (int)(key >> 16);
+        if (tid == 0) ell_of[s] = (uint32_t)ell;
+        t -= ell;
+        target = key & 0xFFFFu;
+    }
+    if (tid == 0) ell_of[0] = (uint32_t)t;
+    __syncthreads();
+    if (failed) {
+        if (tid == 0) write_unsolved(THEMIS_STATUS_TIMEOUT);
+        return;
+    }
+    // one thread per stage turns (s, l_s) into the stage's configuration
+    for (int s = tid; s < S; s += NT) {
+        const int ell = (int)ell_of[s];
+        const int idx = (int)p.Garg[((size_t)n * S + s) * pitch + ell];
+        const int C = p.prob.c_max, NB = p.prob.n_batch;
+        const int bi = idx % NB, rest = idx / NB;
+        b_o[s] = p.prob.batch_sizes[bi];
+        c_o[s] = rest % C + 1;
+        h_o[s] = p.vertical ? p.replicas[(size_t)n * S + s]
+                   : p.horizontal ? G_inst[(size_t)s * pitch + ell] : rest / C + 1;
     }
     if (tid == 0) {
-        if (failed) {
-            write_unsolved(THEMIS_STATUS_TIMEOUT);
-        } else {
-            const int idx = (int)p.Garg[(size_t)n * S * pitch + t];
-            const int C = p.prob.c_max, NB = p.prob.n_batch;
-            const int bi = idx % NB, rest = idx / NB;
-            b_o[0] = p.prob.batch_sizes[bi];
-            c_o[0] = rest % C + 1;
-            h_o[0] = p.vertical ? p.replicas[(size_t)n * S] : p.horizontal ? G_inst[t] : rest / C + 1;
-            p.out.total_cost[n] = (int32_t)best_cost;
-            p.out.latency_buckets[n] = tstar;
-            p.out.status[n] = THEMIS_STATUS_OK;
-        }
+        p.out.total_cost[n] = (int32_t)best_cost;
+        p.out.latency_buckets[n] = tstar;
+        p.out.status[n] = THEMIS_STATUS_OK;
     }
 }
 
@@ -450,45 +549,59 @@ cudaError_t launch_variant16x(const Params &p, int threads, size_t smem, cudaStr
     return cudaGetLastError();
 }
 
+// Shape of a launch: cells per tile, half-groups of 16 tiles, threads (16 per pair of
+// half-groups, whole warps), whether a few cells are left to the block-wide reduction.
+struct Shape16 { int R, half_groups, threads; bool extra; size_t smem; };
+
+Shape16 shape_of(int cells, int pitch, int tile)
+{
+    Shape16 sh;
+    // Finer tiles waste fewer cells past the diagonal (all lanes of a half-warp run to its
+    // longest column) but pay more loads per update: 4 cells per tile up to about 1024 budget
+    // cells, else 8; 16 only on request.
+    sh.R = (tile == 4 || tile == 8 || tile == 16) ? tile : (cells <= 1024 + kMaxExtra ? 4 : 8);
+    for (;;) {
+        const int tiles = (cells + sh.R - 1) / sh.R;
+        sh.half_groups = (tiles + 15) / 16;
+        sh.extra = false;
+        // a few cells beyond a whole number of half-groups are handled outside the tiles
+        if (sh.half_groups > 1 && cells - (sh.half_groups - 1) * 16 * sh.R <= kMaxExtra) {
+            --sh.half_groups;
+            sh.extra = true;
+        }
+        const int slots = (sh.half_groups + 1) / 2;          // half-warps, two half-groups each
+        sh.threads = (slots + 1) / 2 * 32;
+        if (sh.threads <= 1024 || sh.R == 16) break;
+        sh.R *= 2;
+    }
+    const int n_tiles = sh.half_groups * 16;
+    const int CS = sh.R == 16 ? 12 : sh.R / 2;
+    const size_t g_words = (size_t)(n_tiles * sh.R > pitch ? n_tiles * sh.R : pitch);
+    const size_t words = (size_t)(kPadChunks + n_tiles) * CS + 2u * g_words + (size_t)n_tiles + 4 + 32 + THEMIS_MAX_STAGES +
+                         2 * kMaxExtra;
+    sh.smem = words * sizeof(uint32_t);
+    return sh;
+}
+
 template <int R, int MAXT>
-cudaError_t launch_variant16(const Params &p_in, int threads, size_t smem, cudaStream_t stream)
+cudaError_t launch_variant16(const Params &p_in, const Shape16 &sh, cudaStream_t stream)
 {
     Params p = p_in;
-    assign_warp_groups(threads / 32, p.warp_group);
-    return threads * R < p.T + 1 ? launch_variant16x<R, MAXT, true>(p, threads, smem, stream)
-                                 : launch_variant16x<R, MAXT, false>(p, threads, smem, stream);
+    p.n_half_groups = sh.half_groups;
+    return sh.extra ? launch_variant16x<R, MAXT, true>(p, sh.threads, sh.smem, stream)
+                    : launch_variant16x<R, MAXT, false>(p, sh.threads, sh.smem, stream);
 }
 
 }  // namespace
 
 cudaError_t launch_minplus16(const Params &p, int tile, cudaStream_t stream)
 {
-    const int cells = p.T + 1;
-    int R = tile;
-    // Finer tiles waste fewer cells past the diagonal (a warp spans 32 tiles and all its lanes
-    // run to its longest column) but pay more loads per update: 4 cells per thread up to 1024
-    // budget cells, 8 up to 8192, else 16.
-    if (R != 4 && R != 8 && R != 16) R = cells <= 1024 + kMaxExtra ? 4 : 8;
-    if (R == 4 && (cells - kMaxExtra + 3) / 4 > 1024) R = 8;
-    if (R == 8 && (cells - kMaxExtra + 7) / 8 > 1024) R = 16;
-    const int chunks = (cells + R - 1) / R;
-    int groups = (chunks + 31) / 32;
-    // a few cells beyond a whole number of tile groups are handled outside the tiles
-    if (groups > 1 && cells - (groups - 1) * 32 * R <= kMaxExtra) --groups;
-    const int threads = groups * 32;
-    const int CS = R == 16 ? 12 : R / 2;
-    const size_t g_words = (size_t)(threads * R > p.pitch ? threads * R : p.pitch);
-    const size_t words = (size_t)(kPadChunks + threads) * CS + 2u * g_words + 4 + 32 + 32 + THEMIS_MAX_STAGES +
-                         2 * kMaxExtra;
-    const size_t smem = words * sizeof(uint32_t);
-    if (R == 4)
-        return threads <= 512 ? launch_variant16<4, 512>(p, threads, smem, stream)
-                              : launch_variant16<4, 1024>(p, threads, smem, stream);
-    if (R == 8)
-        return threads <= 512 ? launch_variant16<8, 512>(p, threads, smem, stream)
-                              : launch_variant16<8, 1024>(p, threads, smem, stream);
-    return threads <= 512 ? launch_variant16<16, 512>(p, threads, smem, stream)
-                          : launch_variant16<16, 1024>(p, threads, smem, stream);
+    const Shape16 sh = shape_of(p.T + 1, p.pitch, tile);
+    if (sh.R == 4)
+        return sh.threads <= 512 ? launch_variant16<4, 512>(p, sh, stream) : launch_variant16<4, 1024>(p, sh, stream);
+    if (sh.R == 8)
+        return sh.threads <= 512 ? launch_variant16<8, 512>(p, sh, stream) : launch_variant16<8, 1024>(p, sh, stream);
+    return sh.threads <= 512 ? launch_variant16<16, 512>(p, sh, stream) : launch_variant16<16, 1024>(p, sh, stream);
 }
 
 }  // namespace themis
