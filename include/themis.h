@@ -319,11 +319,13 @@ int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_s
 /* Which min-plus kernel themis_minplus_batch and the solvers run (an implementation
  * choice; the paper has no counterpart).  Results do not depend on it; what the rows
  * of the workspace hold does.
- *   0 (default): packed 16-bit kernel (two budget cells per register).  The A
- *      rows then hold the prefix tables themselves, uint16 F_s[t] with
- *      0x7FFF = unreachable or >= 32767, and the backtrack recovers the argmin
- *      along the optimal path only.  Instances whose optimum does not fit 16
- *      bits are redone by the 32-bit kernel in a second launch.
+ *   0 (default): packed 16-bit kernel (two budget cells per register).  It works
+ *      on costs relative to every stage's cheapest entry, and the A rows then hold
+ *      the prefix tables themselves, uint16
+ *          F_s[t] - sum_{k<=s} min_l G_k[l]     (0x7FFF: unreachable or >= 32767),
+ *      while the backtrack recovers the argmin along the optimal path only.
+ *      Instances whose optimum lies 32767 or more above the sum of the stages'
+ *      cheapest entries are redone by the 32-bit kernel in a second launch.
  *   1: 32-bit kernel only; the A rows hold the argmin tables described above.
  *   2: recurrence restricted to the undominated entries of every G_s (an entry is
  *      dominated when a smaller l has a cost at most as high; such entries never

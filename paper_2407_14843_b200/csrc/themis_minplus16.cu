@@ -8,15 +8,19 @@
 // non-negative, so any total below 0x7FFF only ever sums exact parts: the
 // saturating tables equal the true ones wherever the true value is below 0x7FFF.
 // Two half-words add without a carry into the neighbour (at most 0xFFFE).
+// Every row G_s enters relative to its cheapest entry, G_s[l] - min G_s, which
+// shifts F_s by the running sum of those minima and changes no argmin: the 15
+// bits then only have to hold what the latency budget costs on top of the
+// cheapest configurations.  The sum is added back to the reported total and to
+// the last prefix table; the stored uint16 tables stay relative.
 //
 // Packing.  Word k of F holds (F[2k], F[2k+1]).  For an even l = 2e the operand
 // pair of output word j, (F[2j-l], F[2j+1-l]), is the aligned word j-e.  For an
 // odd l = 2e+1 the same word j-e is the operand pair of outputs (2j+1, 2j+2), so
 // every thread keeps two accumulator sets, acc for even l (cells 2j, 2j+1) and
 // accp for odd l (cells 2j+1, 2j+2), and merges them once per stage with a
-// half-word shift; the half-word that belongs to the next thread travels by a
-// warp shuffle (and through shared memory across warps).  G is stored with each
-// cost duplicated into both halves.
+// half-word shift; the half-word that belongs to the next tile travels through
+// shared memory.  G is stored with each cost duplicated into both halves.
 //
 // Argmin.  No argmin is carried.  The prefix tables F_s are kept (uint16, in the
 // workspace rows that the 32-bit kernel uses for its argmin tables) and the
@@ -155,6 +159,7 @@ minplus16_kernel(const Params p)
     uint32_t *stage_lmin = red + 32;                          // 64 words: first reachable l of every G_s
     uint32_t *fx_prev = stage_lmin + THEMIS_MAX_STAGES;       // kMaxExtra words: F_{s-1} at the extra cells
     uint32_t *fx_acc = fx_prev + kMaxExtra;                   // kMaxExtra words: F_s at the extra cells, building
+    uint32_t *stage_cmin = fx_acc + kMaxExtra;                // 64 words: cheapest entry of every G_s
 
     // The two tiles of this thread: its half-warp takes half-group NHG-1-slot (long columns)
     // first and half-group slot (short columns) second; the middle one, if any, stands alone.
@@ -185,7 +190,10 @@ minplus16_kernel(const Params p)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = tid; i < kPadChunks * CS; i += NT) Fw[i] = kInf16x2;
-    for (int i = tid; i < THEMIS_MAX_STAGES; i += NT) stage_lmin[i] = 0xFFFFFFFFu;
+    for (int i = tid; i < THEMIS_MAX_STAGES; i += NT) {
+        stage_lmin[i] = 0xFFFFFFFFu;
+        stage_cmin[i] = 0xFFFFFFFFu;
+    }
     for (int l = pitch + tid; l < Tp; l += NT) {
         Gbuf0[l] = kInf16x2;
         Gbuf1[l] = kInf16x2;
@@ -211,8 +219,35 @@ minplus16_kernel(const Params p)
             store_words<H>(w, reinterpret_cast<uint32_t *>(F16_inst + (size_t)s * pitch + t0));
     };
 
-    // stage 0: F_0 = G_0
+    // The kernel works on costs relative to every row's cheapest entry, G_s[l] - min G_s, so that
+    // the 15 bits hold the cost paid beyond the cheapest configurations rather than the whole
+    // total.  note_row_cmin adds this thread's share of the raw row s in Gk to stage_cmin[s]
+    // (complete after the next block barrier); row_cmin reads it (0 for a row without a candidate).
+    auto note_row_cmin = [&](const uint32_t *Gk, int s) {
+        uint32_t m = 0xFFFFFFFFu;
+        for (int l4 = tid * 4; l4 < pitch; l4 += NT * 4) {
+            const uint4 v = *reinterpret_cast<const uint4 *>(Gk + l4);
+            m = min(m, min(min(v.x, v.y), min(v.z, v.w)));
+        }
+        m = __reduce_min_sync(0xFFFFFFFFu, m);
+        if ((tid & 31) == 0) atomicMin(&stage_cmin[s], m);
+    };
+    auto row_cmin = [&](int s) -> uint32_t {
+        const uint32_t m = stage_cmin[s];
+        return m >= (uint32_t)THEMIS_G_INF ? 0u : m;
+    };
+    uint32_t cost_offset = 0;                             // sum of the rows' cheapest entries so far
+
+    // stage 0: F_0 = G_0 (relative to its cheapest entry); both first rows are waited for here
     if (!mbar_wait(&mbar[0], 0)) failed = 1; else pend0 = -1;
+    note_row_cmin(Gbuf0, 0);
+    if (S > 1) {
+        if (!mbar_wait(&mbar[1], 0)) failed = 1; else pend1 = -1;
+        note_row_cmin(Gbuf1, 1);
+    }
+    __syncthreads();
+    const uint32_t c_off0 = row_cmin(0);
+    cost_offset += c_off0;
     // Records the lowest reachable index among this thread's R entries of row s.
     auto note_first_reachable = [&](uint32_t first, int s) {
         first = __reduce_min_sync(0xFFFFFFFFu, first);
@@ -226,8 +261,8 @@ minplus16_kernel(const Params p)
 #pragma unroll
             for (int r = H - 1; r >= 0; --r) {
                 // raw costs; entries beyond the loaded row hold kInf16x2, far above kInf16
-                const uint32_t lo = t0 < 0 ? kInf16 : min(Gbuf0[t0 + 2 * r], kInf16);
-                const uint32_t hi = t0 < 0 ? kInf16 : min(Gbuf0[t0 + 2 * r + 1], kInf16);
+                const uint32_t lo = t0 < 0 ? kInf16 : min(Gbuf0[t0 + 2 * r] - c_off0, kInf16);
+                const uint32_t hi = t0 < 0 ? kInf16 : min(Gbuf0[t0 + 2 * r + 1] - c_off0, kInf16);
                 w[r] = lo | (hi << 16);
                 if (hi < kInf16) first = min(first, (uint32_t)(t0 + 2 * r + 1));
                 if (lo < kInf16) first = min(first, (uint32_t)(t0 + 2 * r));
@@ -238,7 +273,7 @@ minplus16_kernel(const Params p)
         if (has_b) init_tile(tile_b);
         note_first_reachable(first, 0);
         if (tid < n_extra) {
-            const uint32_t v = min(Gbuf0[Tc + tid], kInf16);
+            const uint32_t v = min(Gbuf0[Tc + tid] - c_off0, kInf16);
             fx_prev[tid] = v;
             F16_inst[Tc + tid] = (uint16_t)v;
         }
@@ -253,13 +288,16 @@ minplus16_kernel(const Params p)
     // below it, and every G_s[l] below that row's first reachable l, can only give "unreachable".
     uint32_t prefix_min = stage_lmin[0];
 
-    for (int s = 1; s < S && !failed; ++s) {
+    // `failed` is block-uniform here and after every __syncthreads_or below; between those it is
+    // a thread's own, so the loop may only leave at the uniform test.
+    for (int s = 1; s < S; ++s) {
+        if (s == 1 && failed) break;
         const int cur = s & 1;
         uint32_t *Gk = cur ? Gbuf1 : Gbuf0;
-        const int parity = (s >> 1) & 1;
-        if (!mbar_wait(&mbar[cur], (uint32_t)parity)) failed = 1;
-        else if (cur) pend1 = -1; else pend0 = -1;
-        // raw costs -> saturated cost duplicated into both half-words, in place
+        // raw costs -> saturated relative cost duplicated into both half-words, in place
+        // (the row has arrived and its cheapest entry is known: see the end of the stage before)
+        const uint32_t c_off = row_cmin(s);
+        cost_offset += c_off;
         {
             uint32_t first = 0xFFFFFFFFu;
             for (int l4 = tid * 4; l4 < pitch; l4 += NT * 4) {
@@ -267,7 +305,7 @@ minplus16_kernel(const Params p)
                 uint32_t *v = reinterpret_cast<uint32_t *>(&v4);
 #pragma unroll
                 for (int i = 3; i >= 0; --i) {
-                    const uint32_t c = min(v[i], kInf16);
+                    const uint32_t c = min(v[i] - c_off, kInf16);
                     v[i] = c | (c << 16);
                     if (c < kInf16) first = min(first, (uint32_t)(l4 + i));
                 }
@@ -382,6 +420,12 @@ minplus16_kernel(const Params p)
                     if ((tid & 31) == 0) atomicMin(&fx_acc[e], m);
                 }
         }
+        if (s + 1 < S) {                                  // the next row arrived long ago: its cheapest entry
+            const int nxt = cur ^ 1;
+            if (!mbar_wait(&mbar[nxt], (uint32_t)(((s + 1) >> 1) & 1))) failed = 1;
+            else if (nxt) pend1 = -1; else pend0 = -1;
+            note_row_cmin(nxt ? Gbuf1 : Gbuf0, s + 1);
+        }
         __syncthreads();                                  // every read of F_{s-1} is done, every tile parked
 
         auto finish_tile = [&](uint32_t (&w)[H], int tile) {
@@ -458,8 +502,8 @@ minplus16_kernel(const Params p)
                 const uint32_t w = chunk[r];
                 const int t = (tile - n_dummy) * R + 2 * r;
                 if (t >= 0 && t < pitch) {
-                    F_row[t] = (w & 0xFFFFu) >= kInf16 ? THEMIS_G_INF : (int32_t)(w & 0xFFFFu);
-                    F_row[t + 1] = (w >> 16) >= kInf16 ? THEMIS_G_INF : (int32_t)(w >> 16);
+                    F_row[t] = (w & 0xFFFFu) >= kInf16 ? THEMIS_G_INF : (int32_t)((w & 0xFFFFu) + cost_offset);
+                    F_row[t + 1] = (w >> 16) >= kInf16 ? THEMIS_G_INF : (int32_t)((w >> 16) + cost_offset);
                 }
             }
         };
@@ -468,7 +512,8 @@ minplus16_kernel(const Params p)
     }
 
     if (tid < n_extra)
-        p.F[(size_t)n * pitch + Tc + tid] = fx_prev[tid] >= kInf16 ? THEMIS_G_INF : (int32_t)fx_prev[tid];
+        p.F[(size_t)n * pitch + Tc + tid] =
+            fx_prev[tid] >= kInf16 ? THEMIS_G_INF : (int32_t)(fx_prev[tid] + cost_offset);
 
     // backtrack along the optimal path: lowest l with F_{s-1}[t-l] + G_s[l] == F_s[t].
     // The block scans l upward, kScanGroups * 4 * NT values a round (four consecutive l per
@@ -484,6 +529,7 @@ minplus16_kernel(const Params p)
     for (int s = S - 1; s >= 1 && !failed; --s) {
         const int32_t *G_row = G_inst + (size_t)s * pitch;
         const uint16_t *Fprev = F16_inst + (size_t)(s - 1) * pitch;
+        const uint32_t c_off = stage_cmin[s] >= (uint32_t)THEMIS_G_INF ? 0u : stage_cmin[s];
         uint32_t key = 0xFFFFFFFFu;
         for (int base = 0; base <= t; base += kScanGroups * 4 * NT) {
             uint32_t cand = 0xFFFFFFFFu;
@@ -497,7 +543,7 @@ minplus16_kernel(const Params p)
                     for (int i = 3; i >= 0; --i)
                         if (l4 + i <= t) {
                             const uint32_t f = Fprev[t - l4 - i];
-                            if (f + min((uint32_t)gv[i], kInf16) == target) cand = ((uint32_t)(l4 + i) << 16) | f;
+                            if (f + min((uint32_t)gv[i] - c_off, kInf16) == target) cand = ((uint32_t)(l4 + i) << 16) | f;
                         }
                 }
             }
@@ -533,7 +579,7 @@ minplus16_kernel(const Params p)
                    : p.horizontal ? G_inst[(size_t)s * pitch + ell] : rest / C + 1;
     }
     if (tid == 0) {
-        p.out.total_cost[n] = (int32_t)best_cost;
+        p.out.total_cost[n] = (int32_t)(best_cost + cost_offset);
         p.out.latency_buckets[n] = tstar;
         p.out.status[n] = THEMIS_STATUS_OK;
     }
@@ -557,9 +603,9 @@ Shape16 shape_of(int cells, int pitch, int tile)
 {
     Shape16 sh;
     // Finer tiles waste fewer cells past the diagonal (all lanes of a half-warp run to its
-    // longest column) but pay more loads per update: 4 cells per tile up to about 1024 budget
+    // longest column) but pay more loads per update: 4 cells per tile up to about 900 budget
     // cells, else 8; 16 only on request.
-    sh.R = (tile == 4 || tile == 8 || tile == 16) ? tile : (cells <= 1024 + kMaxExtra ? 4 : 8);
+    sh.R = (tile == 4 || tile == 8 || tile == 16) ? tile : (cells <= 896 + kMaxExtra ? 4 : 8);
     for (;;) {
         const int tiles = (cells + sh.R - 1) / sh.R;
         sh.half_groups = (tiles + 15) / 16;
@@ -577,8 +623,8 @@ Shape16 shape_of(int cells, int pitch, int tile)
     const int n_tiles = sh.half_groups * 16;
     const int CS = sh.R == 16 ? 12 : sh.R / 2;
     const size_t g_words = (size_t)(n_tiles * sh.R > pitch ? n_tiles * sh.R : pitch);
-    const size_t words = (size_t)(kPadChunks + n_tiles) * CS + 2u * g_words + (size_t)n_tiles + 4 + 32 + THEMIS_MAX_STAGES +
-                         2 * kMaxExtra;
+    const size_t words = (size_t)(kPadChunks + n_tiles) * CS + 2u * g_words + (size_t)n_tiles + 4 + 32 +
+                         2 * THEMIS_MAX_STAGES + 2 * kMaxExtra;
     sh.smem = words * sizeof(uint32_t);
     return sh;
 }

@@ -86,7 +86,12 @@ def _assert_tables_equal(S, gpu, ref):
         solved = ref["status"] == 0
         assert np.array_equal(gpu["F"][solved], ref["F"][solved, -1, :])
         assert (ref["F"][ref["F"] != S.G_INF] < S.INF16).all(), "use the saturation test for such inputs"
-        assert np.array_equal(gpu["A"], np.minimum(ref["F"], S.INF16).astype(np.uint16))
+        # prefix tables relative to the running sum of the stages' cheapest entries
+        cheapest = ref["G"].astype(np.int64).min(axis=2)
+        cheapest[cheapest == S.G_INF] = 0
+        rel = ref["F"].astype(np.int64) - np.cumsum(cheapest, axis=1)[:, :, None]
+        rel[ref["F"] == S.G_INF] = S.INF16
+        assert np.array_equal(gpu["A"], rel.astype(np.uint16))
         return
     assert np.array_equal(gpu["F"], ref["F"][:, -1, :])
     reach = ref["F"] != S.G_INF
@@ -406,20 +411,30 @@ def test_all_kernels_agree(S):
 
 
 def test_totals_beyond_16_bits_fall_back_to_the_wide_kernel(S, oracle_mod):
-    """Vertical problem with thousands of replicas per stage: optimal totals of
-    40000 and more do not fit the packed kernel's 15-bit costs; those instances
-    are redone by the 32-bit kernel.  Mixed with cheap instances and with
-    infeasible ones in the same batch."""
-    base = W.random_tiny_workload(5600, 24, 6, 2, (1, 2, 4), 4, 420, vertical=True, rate_lo=10.0, rate_hi=60.0)
+    """Vertical problem with thousands of replicas per stage.  The packed kernel holds, in 15
+    bits, what an instance pays beyond the sum of its stages' cheapest entries.  One group of
+    instances has totals of 36000 and more but pays little beyond those entries (solved by the
+    packed kernel); another must take the dearer core count in all six stages, 36000 beyond
+    them, and is redone by the 32-bit kernel.  Mixed with cheap and with infeasible instances."""
+    base = W.random_tiny_workload(5600, 32, 6, 2, (1, 2, 4), 4, 420, vertical=True, rate_lo=10.0, rate_hi=60.0)
     rep = base.replicas.copy()
-    rep[0::3] = 6000                        # 6 stages x 6000 x c: totals of 36000 .. 72000
-    rep[1::3] = np.maximum(rep[1::3], 1)
+    rep[0::4] = 6000                        # 6 stages x 6000 x c: totals of 36000 .. 72000
+    rep[1::4] = np.maximum(rep[1::4], 1)
+    rep[3::4] = 6000
     lam = base.lambda_mrps.copy()
-    lam[2::3] = 4_000_000                   # 4000 rps on a handful of replicas: infeasible
-    wl = dataclasses.replace(base, replicas=rep, lambda_mrps=lam)
-    ref = oracle_mod.solve_batch(wl)
-    assert (ref["total_cost"] >= S.INF16).any() and (ref["status"] == 1).any()
+    lam[2::4] = 4_000_000                   # 4000 rps on a handful of replicas: infeasible
+    lat = base.lat_us.copy()                # one profile per instance: [N][S][c][b]
+    lat[3::4, :, 0, :] = 130_000            # one core: 130 buckets; two cores: 65; budget 420, so
+    lat[3::4, :, 1, :] = 65_000             # six stages only fit with two cores everywhere
+    lat[3::4, :, :, 1:] = 900_000           # larger batches never fit
+    wl = dataclasses.replace(base, replicas=rep, lambda_mrps=lam, lat_us=lat)
+    ref = oracle_mod.solve_batch(wl, dumps=True)
+    assert (ref["status"] == 1).any()
     assert ((ref["total_cost"] > 0) & (ref["total_cost"] < S.INF16)).any()
+    beyond = ref["total_cost"] - ref["G"].astype(np.int64).min(axis=2).sum(axis=1)
+    solved = ref["status"] == 0
+    assert (solved & (ref["total_cost"] >= S.INF16) & (beyond < S.INF16)).any()
+    assert (solved[3::4] & (beyond[3::4] >= S.INF16)).all()
     S.themis_set_minplus_mode(0)
     _assert_results_equal(_gpu_solve(S, wl), ref)
 
