@@ -308,10 +308,14 @@ int themis_fit_profiles_batch(int32_t n_models, int32_t n_samples, const int32_t
  *   1: fused 32-bit add-min (one instruction per update);
  *   2: two adds and one three-input min per two updates;
  *   3: fused add-min on packed 2 x 16-bit (two cell updates per instruction);
- *   4: single-precision add and min.
+ *   4: single-precision add and min;
+ *   5: the packed recurrence kernel's own inner step, operands loaded from shared
+ *      memory as there but without stages, barriers or global traffic: every
+ *      thread walks `iters` columns of 256 chunk steps of 8 x 8 cells (threads
+ *      must be 256; 128 fused instructions per 4 steps as in mode 3).
  * Launches `blocks` x `threads` (32..1024) and writes one word per thread to d_sink
  * (blocks*threads uint32).  Updates performed = blocks * threads * iters * 64
- * (x 2 cells in mode 3).
+ * (x 2 cells in mode 3; blocks * 256 * iters * 256 * 64 cells in mode 5).
  */
 int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_sink,
                      void *cuda_stream);

@@ -14,7 +14,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 LIB_PATH = os.path.join(_PKG, "libthemis.so")
 SOURCES = sorted(glob.glob(os.path.join(_PKG, "csrc", "*.cu")))
-HEADERS = sorted(glob.glob(os.path.join(_PKG, "csrc", "*.h"))) + [os.path.join(_ROOT, "include", "themis.h")]
+HEADERS = sorted(glob.glob(os.path.join(_PKG, "csrc", "*.h")) + glob.glob(os.path.join(_PKG, "csrc", "*.cuh"))) + [os.path.join(_ROOT, "include", "themis.h")]
 
 
 def _nvcc() -> str:

@@ -524,7 +524,7 @@ int themis_fit_profiles_batch(int32_t n_models, int32_t n_samples, const int32_t
 
 int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_sink, void *cuda_stream)
 {
-    if (mode < 0 || mode > 4 || blocks < 1 || threads < 32 || threads > 1024 || iters < 1 || !d_sink)
+    if (mode < 0 || mode > 5 || (mode == 5 && threads != 256) || blocks < 1 || threads < 32 || threads > 1024 || iters < 1 || !d_sink)
         return THEMIS_E_INVALID_ARG;
     cudaError_t e = launch_alu_probe(mode, blocks, threads, iters, d_sink, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);

@@ -41,6 +41,7 @@
 // 32-bit kernel in a second launch.
 #include "themis_async.cuh"
 #include "themis_internal.h"
+#include "themis_minplus16_step.cuh"
 
 namespace themis {
 namespace {
@@ -51,69 +52,6 @@ constexpr int kPadChunks = 32;   // "unreachable" chunks in front of F[0]: one p
 // a whole extra warp walking the longest columns for a handful of cells.  Up to this many cells
 // beyond the last full group are instead computed by a block-wide reduction per stage.
 constexpr int kMaxExtra = 8;
-
-template <int R>
-struct Tile16 {
-    static constexpr int H = R / 2;                       // words per chunk
-    static constexpr int CS = (H % 8 == 0) ? H + 4 : H;   // chunk stride: keeps 16-byte loads of
-                                                          // consecutive lanes in distinct bank groups
-};
-
-// H consecutive words (H = 2, 4 or 8) from / to 8- or 16-byte aligned memory.
-template <int H>
-__device__ __forceinline__ void load_words(uint32_t (&w)[H], const uint32_t *src)
-{
-    if constexpr (H == 2) {
-        const uint2 x = *reinterpret_cast<const uint2 *>(src);
-        w[0] = x.x; w[1] = x.y;
-    } else {
-#pragma unroll
-        for (int v = 0; v < H / 4; ++v) {
-            const uint4 x = *reinterpret_cast<const uint4 *>(src + 4 * v);
-            w[4 * v + 0] = x.x; w[4 * v + 1] = x.y; w[4 * v + 2] = x.z; w[4 * v + 3] = x.w;
-        }
-    }
-}
-
-template <int H>
-__device__ __forceinline__ void store_words(const uint32_t (&w)[H], uint32_t *dst)
-{
-    if constexpr (H == 2) {
-        *reinterpret_cast<uint2 *>(dst) = make_uint2(w[0], w[1]);
-    } else {
-#pragma unroll
-        for (int v = 0; v < H / 4; ++v)
-            *reinterpret_cast<uint4 *>(dst + 4 * v) = make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
-    }
-}
-
-// One chunk step: R values of l (H even/odd pairs) against the thread's R cells.
-// w_hi holds words m .. m+H-1 of F, w_lo receives words m-H .. m-1 (m = J - q*H).
-template <int R>
-__device__ __forceinline__ void chunk_step16(const uint32_t (&w_hi)[R / 2], uint32_t (&w_lo)[R / 2],
-                                             uint32_t (&acc)[R / 2], uint32_t (&accp)[R / 2],
-                                             const uint32_t *f_chunk, const uint32_t *g_chunk)
-{
-    constexpr int H = R / 2;
-    load_words<H>(w_lo, f_chunk);
-#pragma unroll
-    for (int v = 0; v < R / 4; ++v) {
-        const uint4 g4 = *reinterpret_cast<const uint4 *>(g_chunk + 4 * v);   // l = l0+4v .. l0+4v+3
-        const uint32_t g_even[2] = {g4.x, g4.z};
-        const uint32_t g_odd[2] = {g4.y, g4.w};
-#pragma unroll
-        for (int kk = 0; kk < 2; ++kk) {
-            const int k = 2 * v + kk;                      // pair index within the chunk
-#pragma unroll
-            for (int r = 0; r < H; ++r) {
-                const int i = H + r - k;                   // 1 .. 2H-1
-                const uint32_t f = i >= H ? w_hi[i - H] : w_lo[i];
-                acc[r] = __viaddmin_u16x2(f, g_even[kk], acc[r]);
-                accp[r] = __viaddmin_u16x2(f, g_odd[kk], accp[r]);
-            }
-        }
-    }
-}
 
 // Block-wide unsigned minimum; every thread gets the result.  Two barriers.
 __device__ __forceinline__ uint32_t block_min(uint32_t v, uint32_t *red, int tid, int n_warps)
@@ -129,12 +67,12 @@ __device__ __forceinline__ uint32_t block_min(uint32_t v, uint32_t *red, int tid
 
 // EXTRA: the block also computes up to kMaxExtra cells beyond its tiles (see kMaxExtra).
 template <int R, int MAXT, bool EXTRA>
-__global__ void __launch_bounds__(MAXT)
+__global__ void __launch_bounds__(MAXT, (R == 16 || MAXT > 512) ? 1 : 2)   // 64 registers: two blocks of 512
 minplus16_kernel(const Params p)
 {
     extern __shared__ __align__(128) uint32_t smem[];
     constexpr int H = Tile16<R>::H, CS = Tile16<R>::CS;
-    constexpr int U = 32 / R;                             // chunk steps per loop iteration (2, 4 or 8)
+    constexpr int U = R == 16 ? 2 : 64 / R;               // chunk steps per iteration of the main loop
     const int n = blockIdx.x;
     if (p.active && !p.active[n]) return;
     const int tid = threadIdx.x;
@@ -330,11 +268,11 @@ minplus16_kernel(const Params p)
         // All lanes of a half-warp walk the same l so that G is a broadcast; lanes that run
         // past their own range read the "unreachable" chunks in front of F[0].  Chunks of
         // l below G_s's first reachable entry, and chunks that only meet F_{s-1} below its
-        // first reachable budget, are skipped (whole steps of U chunks, block-uniform).
+        // first reachable budget, are skipped (pairs of chunks, block-uniform).
         const uint32_t g_min = stage_lmin[s];
         const bool dead = g_min == 0xFFFFFFFFu || prefix_min == 0xFFFFFFFFu;
-        const int q_lo = dead ? 0 : (int)(g_min / R) & ~(U - 1);
-        const int q_shift = dead ? 0 : ((int)(prefix_min / R) + n_dummy) & ~(U - 1);   // in tiles
+        const int q_lo = dead ? 0 : (int)(g_min / R) & ~1;
+        const int q_shift = dead ? 0 : ((int)(prefix_min / R) + n_dummy) & ~1;   // in tiles
         auto steps_of = [&](int tile) { return dead ? 0 : max(0, (tile | 15) - q_shift - q_lo + 1); };
         const int steps_a = has_a ? steps_of(tile_a) : 0, steps_b = has_b ? steps_of(tile_b) : 0;
         const uint32_t *f_lo = Fw, *g = Gk;
@@ -373,7 +311,8 @@ minplus16_kernel(const Params p)
             const unsigned n_seg = __reduce_min_sync(0xFFFFFFFFu, remaining > 0 ? (unsigned)remaining : 0xFFFFFFFFu);
             if (n_seg == 0xFFFFFFFFu) break;
             if (remaining > 0) {
-                for (unsigned q = 0; q < n_seg; q += U) {
+                unsigned q = 0;
+                for (; q + U <= n_seg; q += U) {
 #pragma unroll
                     for (int u = 0; u < U; u += 2) {
                         chunk_step16<R>(wa, wb, acc, accp, f_lo - u * CS, g + u * R);
@@ -381,6 +320,12 @@ minplus16_kernel(const Params p)
                     }
                     f_lo -= U * CS;
                     g += U * R;
+                }
+                for (; q < n_seg; q += 2) {               // segments are even, not multiples of U
+                    chunk_step16<R>(wa, wb, acc, accp, f_lo, g);
+                    chunk_step16<R>(wb, wa, acc, accp, f_lo - CS, g + R);
+                    f_lo -= 2 * CS;
+                    g += 2 * R;
                 }
                 remaining -= (int)n_seg;
                 advance();

@@ -3,7 +3,12 @@
 // instruction forms.  Every update reads two values produced one round earlier,
 // so nothing can be hoisted and no memory is touched.  It measures what the
 // arithmetic pipes sustain; it is not part of the method.
+//
+// Form 5 times the packed kernel's own inner step instead (themis_minplus16_step.cuh):
+// columns of 256 chunk steps with the operands loaded from shared memory exactly as in
+// the recurrence kernel, but no stages, barriers or global traffic around them.
 #include "themis_internal.h"
+#include "themis_minplus16_step.cuh"
 
 namespace themis {
 namespace {
@@ -69,6 +74,42 @@ __global__ void alu_probe_kernel(int iters, uint32_t *sink)
     sink[blockIdx.x * blockDim.x + threadIdx.x] = r;
 }
 
+// 256 threads; thread i owns tile 256 + i of a 512-tile row and walks 256 chunks of l per
+// column, `iters` columns.  One column = 256 * R * R / ... cell updates: 256 steps x R x R cells.
+template <int R>
+__global__ void __launch_bounds__(256) step_probe_kernel(int iters, uint32_t *sink)
+{
+    constexpr int H = Tile16<R>::H, CS = Tile16<R>::CS;
+    constexpr int kTiles = 512, kSteps = 256, U = 32 / R;
+    __shared__ __align__(16) uint32_t Fw[kTiles * CS];
+    __shared__ __align__(16) uint32_t G[kSteps * R];
+    const int tid = threadIdx.x;
+    for (int i = tid; i < kTiles * CS; i += 256) Fw[i] = ((uint32_t)(i * 37 + blockIdx.x) & 0x3FFFu) * 0x00010001u;
+    for (int i = tid; i < kSteps * R; i += 256) G[i] = ((uint32_t)(i * 11 + 5) & 0x0FFFu) * 0x00010001u;
+    __syncthreads();
+    uint32_t acc[H], accp[H], wa[H], wb[H];
+#pragma unroll
+    for (int r = 0; r < H; ++r) { acc[r] = 0xFFFFFFFFu; accp[r] = 0xFFFFFFFFu; }
+    const uint32_t *f_hi = Fw + (256 + tid) * CS;
+    for (int it = 0; it < iters; ++it) {
+        load_words<H>(wa, f_hi);
+        const uint32_t *f_lo = f_hi - CS, *g = G;
+        for (int q = 0; q < kSteps; q += U) {
+#pragma unroll
+            for (int u = 0; u < U; u += 2) {
+                chunk_step16<R>(wa, wb, acc, accp, f_lo - u * CS, g + u * R);
+                chunk_step16<R>(wb, wa, acc, accp, f_lo - (u + 1) * CS, g + (u + 1) * R);
+            }
+            f_lo -= U * CS;
+            g += U * R;
+        }
+    }
+    uint32_t r = 0;
+#pragma unroll
+    for (int i = 0; i < H; ++i) r ^= acc[i] ^ accp[i];
+    sink[blockIdx.x * blockDim.x + tid] = r;
+}
+
 }  // namespace
 
 cudaError_t launch_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *sink, cudaStream_t stream)
@@ -78,6 +119,10 @@ cudaError_t launch_alu_probe(int mode, int blocks, int threads, int iters, uint3
         case 1: alu_probe_kernel<1><<<blocks, threads, 0, stream>>>(iters, sink); break;
         case 2: alu_probe_kernel<2><<<blocks, threads, 0, stream>>>(iters, sink); break;
         case 3: alu_probe_kernel<3><<<blocks, threads, 0, stream>>>(iters, sink); break;
+        case 5:
+            if (threads != 256) return cudaErrorInvalidValue;
+            step_probe_kernel<8><<<blocks, 256, 0, stream>>>(iters, sink);
+            break;
         default: alu_probe_kernel<4><<<blocks, threads, 0, stream>>>(iters, sink); break;
     }
     return cudaGetLastError();
