@@ -42,10 +42,12 @@ HBM_FALLBACK_GBS = 6650.0
 # DRAM bytes (read + write) of one min-plus launch from the ncu capture summarised
 # under profiles/, per instance of the captured workload.  Traffic is proportional
 # to the instance count (one block per instance, no reuse across blocks).  The
-# figure is only reported while the kernel source still has the recorded hash.
+# figure is only reported while the kernel sources still have the recorded hash.
 NCU_TRAFFIC = {
-    "config": 4, "bytes_per_instance": (308.140032e6 + 159.183360e6) / 2368,
-    "source": "paper_2407_14843_b200/csrc/themis_minplus16.cu", "sha256_16": "509f368d0155c510",
+    "config": 4, "bytes_per_instance": (315.242240e6 + 156.358656e6) / 2368,
+    "sources": ("paper_2407_14843_b200/csrc/themis_minplus16.cu",
+                "paper_2407_14843_b200/csrc/themis_minplus16_step.cuh"),
+    "sha256_16": "ffd7c90af1cd82cd",
 }
 
 
@@ -73,9 +75,12 @@ def parse_args():
 def ncu_traffic_bytes(cfg: int, n_instances: int):
     import hashlib
     try:
-        with open(os.path.join(ROOT, NCU_TRAFFIC["source"]), "rb") as f:
-            if hashlib.sha256(f.read()).hexdigest()[:16] != NCU_TRAFFIC["sha256_16"]:
-                return None
+        h = hashlib.sha256()
+        for src in NCU_TRAFFIC["sources"]:
+            with open(os.path.join(ROOT, src), "rb") as f:
+                h.update(f.read())
+        if h.hexdigest()[:16] != NCU_TRAFFIC["sha256_16"]:
+            return None
     except OSError:
         return None
     return NCU_TRAFFIC["bytes_per_instance"] * n_instances if cfg == NCU_TRAFFIC["config"] else None
@@ -444,26 +449,32 @@ def run_ours(args):
 
 
 def run_alu_probe():
-    """Rates of themis_alu_probe in all five instruction forms (updates per SM per clock at
-    the boost clock, and TOP/s counting two operations per cell update)."""
+    """Rates of themis_alu_probe in all its forms (updates per SM per clock at the boost
+    clock, and TOP/s counting two operations per cell update).  Forms 0-4 keep their
+    operands in registers; form 5 is the packed kernel's inner step with its operand
+    loads from shared memory."""
     import torch
     from paper_2407_14843_b200 import build as _build
     _build.build_library()
     from paper_2407_14843_b200 import solver
     torch.cuda.set_device(0)
     forms = {0: "32-bit add, then unsigned min", 1: "fused 32-bit add-min", 2: "two adds + one three-input min per two updates",
-             3: "fused add-min on packed 2 x 16-bit", 4: "single-precision add, then min"}
-    blocks, threads, iters = N_SMS * 8, 256, 20000
-    sink = torch.empty(blocks * threads, dtype=torch.uint32, device="cuda")
+             3: "fused add-min on packed 2 x 16-bit", 4: "single-precision add, then min",
+             5: "inner step of the packed recurrence kernel (operands from shared memory)"}
+    threads = 256
     out = {}
     for mode, what in forms.items():
-        solver.themis_alu_probe(mode, blocks, threads, 50, sink)
+        # form 5: 4 blocks per SM as the recurrence kernel runs, 256 steps x 64 cells per iteration
+        blocks, warm, iters = (N_SMS * 4, 2, 300) if mode == 5 else (N_SMS * 8, 50, 20000)
+        sink = torch.empty(blocks * threads, dtype=torch.uint32, device="cuda")
+        solver.themis_alu_probe(mode, blocks, threads, warm, sink)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         solver.themis_alu_probe(mode, blocks, threads, iters, sink)
         b.record()
         torch.cuda.synchronize()
-        cells = (2 if mode == 3 else 1) * blocks * threads * iters * 64
+        per_iter = 256 * 64 if mode == 5 else (128 if mode == 3 else 64)
+        cells = blocks * threads * iters * per_iter
         rate = cells / (a.elapsed_time(b) * 1e-3)
         out[f"mode{mode}"] = {"form": what, "ms": a.elapsed_time(b), "cell_updates_per_s": rate,
                               "tops": 2.0 * rate / 1e12,

@@ -80,7 +80,7 @@ template <int R>
 __global__ void __launch_bounds__(256) step_probe_kernel(int iters, uint32_t *sink)
 {
     constexpr int H = Tile16<R>::H, CS = Tile16<R>::CS;
-    constexpr int kTiles = 512, kSteps = 256, U = 32 / R;
+    constexpr int kTiles = 512, kSteps = 256, U = 64 / R;
     __shared__ __align__(16) uint32_t Fw[kTiles * CS];
     __shared__ __align__(16) uint32_t G[kSteps * R];
     const int tid = threadIdx.x;
