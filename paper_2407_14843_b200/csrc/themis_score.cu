@@ -10,14 +10,22 @@
 //                 satisfies  h * b / l >= lambda                           (Eq. 6)
 // (joint problem: one table for all stages; vertical variant: one row pair per
 // stage, for that stage's fixed replica count), all filled before the first stage.
-// A candidate then costs a compare, an add, a multiply-add and a shared-memory
-// atomic min on the packed word (cost << 16 | candidate index), whose ordering
-// gives "cheapest, then lowest index" directly.
+// A candidate is then two compares, a multiply-add and a shared-memory atomic
+// min on the packed word (cost << 16 | candidate index), whose ordering gives
+// "cheapest, then lowest index" directly.
 //
-// Work is dealt to warps as (one batch size) x (32 consecutive core counts), so
-// all lanes of a warp read the same table rows (no bank conflicts) and walk the
-// replica count upward from the fewest replicas that sustain lambda.  Two key
-// rows alternate between stages, so a stage costs one block barrier.
+// A warp task is (one batch size) x (32 consecutive core counts).  Its lanes
+// first take one (c, b) pair each: load the latency, drop the pair if one core
+// fewer has the same latency or if the latency alone exceeds the budget, and
+// round it up to buckets.  Then
+//  - where the queuing delay grows with the replica count (joint problem, flag
+//    THEMIS_QUEUE_PER_REPLICA, b > 1), the surviving pairs are compacted into a
+//    warp-private list and the lanes switch to one replica count each: every
+//    list entry is broadcast and each lane scores its (h, c, b);
+//  - elsewhere more replicas only cost more in the same bucket, so each lane
+//    looks up the fewest replicas that sustain lambda for its pair (binary
+//    search in the Lmax row) and scores that one candidate.
+// Two key rows alternate between stages, so a stage costs one block barrier.
 #include "themis_internal.h"
 
 namespace themis {
@@ -25,13 +33,57 @@ namespace {
 
 constexpr uint32_t kEmptyKey = 0xFFFFFFFFu;
 constexpr int kScoreThreads = 256;
+constexpr int kScoreWarps = kScoreThreads / 32;
+constexpr int kListWords = 64;        // per warp: 32 entries of two words
+constexpr uint32_t kNeverFits = 0xFFFFFFFFu;   // latency of a padding entry: above every Lmax
+
+// atomic min on a shared-memory word given by its 32-bit shared-space address
+__device__ __forceinline__ void red_min_shared(uint32_t addr, uint32_t v)
+{
+    asm volatile("red.shared.min.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+
+// Two list entries {latency [us], 4 * l_b | c << 17} at `entries` against this lane's replica
+// count: q4 = 4 * Q[b][h], lmax = Lmax[b][h], key = c * key_mul + key_add.  A lane whose
+// candidate is infeasible or over budget sends its word to `idle` (a word nobody reads), so
+// the reduction itself is unconditional and the loop body has no branch.
+__device__ __forceinline__ void score_two_entries(uint32_t entries, uint32_t q4, uint32_t lmax, uint32_t t4,
+                                                  uint32_t key_mul, uint32_t key_add, uint32_t keys,
+                                                  uint32_t idle)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        ".reg .b32 e0, e1, e2, e3, x, y, l0, l1, c0, c1, k0, k1;\n\t"
+        "ld.shared.v4.u32 {e0, e1, e2, e3}, [%0];\n\t"
+        "add.u32 x, e1, %1;\n\t"
+        "add.u32 y, e3, %1;\n\t"
+        "and.b32 l0, x, 0x1FFFC;\n\t"
+        "and.b32 l1, y, 0x1FFFC;\n\t"
+        "setp.le.u32 p, e0, %2;\n\t"
+        "setp.le.u32 q, e2, %2;\n\t"
+        "setp.le.and.u32 p, l0, %3, p;\n\t"
+        "setp.le.and.u32 q, l1, %3, q;\n\t"
+        "shr.u32 c0, x, 17;\n\t"
+        "shr.u32 c1, y, 17;\n\t"
+        "mad.lo.u32 k0, c0, %4, %5;\n\t"
+        "mad.lo.u32 k1, c1, %4, %5;\n\t"
+        "add.u32 l0, l0, %6;\n\t"
+        "add.u32 l1, l1, %6;\n\t"
+        "selp.u32 l0, l0, %7, p;\n\t"
+        "selp.u32 l1, l1, %7, q;\n\t"
+        "red.shared.min.u32 [l0], k0;\n\t"
+        "red.shared.min.u32 [l1], k1;\n\t"
+        "}" ::"r"(entries), "r"(q4), "r"(lmax), "r"(t4), "r"(key_mul), "r"(key_add), "r"(keys), "r"(idle)
+        : "memory");
+}
 
 __device__ __forceinline__ uint32_t sat_u32(unsigned long long v, uint32_t cap)
 {
     return v > (unsigned long long)cap ? cap : (uint32_t)v;
 }
 
-__global__ void __launch_bounds__(kScoreThreads)
+__global__ void __launch_bounds__(kScoreThreads, 6)
 score_kernel(const Params p)
 {
     extern __shared__ __align__(16) uint32_t smem[];
@@ -44,16 +96,21 @@ score_kernel(const Params p)
     const int HN = p.vertical ? 1 : p.prob.h_max;   // replica values per table row
     const int SV = p.vertical ? S : 1;              // table sets: one per stage when h is per stage
     const uint32_t w_us = (uint32_t)p.prob.bucket_us;
+    const int lane = tid & 31, warp = tid >> 5;
 
-    uint32_t *keys0 = smem;                     // [pitch]
-    uint32_t *keys1 = keys0 + pitch;            // [pitch]
-    uint32_t *Q = keys1 + pitch;                // [SV][NB][HN]
-    uint32_t *Lmax = Q + SV * NB * HN;          // [SV][NB][HN]
+    // Shared memory, in words (every access is an offset from this one array):
+    // key row 0 [pitch] | key row 1 [pitch] | Q [SV][NB][HN] | Lmax [SV][NB][HN] | pad to 4 |
+    // one list per warp [kListWords] | one idle word per lane [32]
+    const int q_off = 2 * pitch;
+    const int lmax_off = q_off + SV * NB * HN;
+    const int list_base = (lmax_off + SV * NB * HN + 3) & ~3;
+    const int list_off = list_base + warp * kListWords;
+    const uint32_t smem_addr = (uint32_t)__cvta_generic_to_shared(smem);
+    const uint32_t idle_addr = smem_addr + 4u * (uint32_t)(list_base + kScoreWarps * kListWords + lane);
     __shared__ int s_bad;
 
     const uint32_t lambda_m = p.lambda_mrps[n];
     const int pid = p.profile_id ? p.profile_id[n] : 0;
-    const int32_t *lat = p.lat_us + (size_t)pid * S * CB;
     const int32_t *rep = p.vertical ? p.replicas + (size_t)n * S : nullptr;
 
     if (tid == 0) {
@@ -68,10 +125,16 @@ score_kernel(const Params p)
         }
         s_bad = bad;
     }
-    for (int l = tid; l < 2 * pitch; l += kScoreThreads) keys0[l] = kEmptyKey;
+    for (int l4 = tid * 4; l4 < 2 * pitch; l4 += kScoreThreads * 4)
+        *reinterpret_cast<uint4 *>(smem + l4) = make_uint4(kEmptyKey, kEmptyKey, kEmptyKey, kEmptyKey);
     __syncthreads();
     const bool skip_all = s_bad != 0;
+    const int32_t *lat = p.lat_us + (size_t)(skip_all ? 0 : pid) * S * CB;
 
+    // This warp's tasks: (batch index, chunk of 32 core counts) number warp, warp + kScoreWarps, ...
+    const int c_chunks = (C + 31) / 32;
+    const int bi_first = warp / c_chunks, ch_first = warp - bi_first * c_chunks;
+    const int bi_step = kScoreWarps / c_chunks, ch_step = kScoreWarps - bi_step * c_chunks;
     if (!skip_all) {
         const unsigned long long q_den = (unsigned long long)lambda_m * w_us;
         for (int e = tid; e < SV * NB * HN; e += kScoreThreads) {
@@ -82,65 +145,109 @@ score_kernel(const Params p)
             const unsigned long long b = (unsigned long long)p.prob.batch_sizes[bi];
             const unsigned long long m = (p.prob.flags & THEMIS_QUEUE_PER_REPLICA) ? h : 1ull;
             const unsigned long long q_num = (b - 1ull) * m * 1000000000ull;
-            Q[e] = sat_u32((q_num + q_den - 1ull) / q_den, (uint32_t)T + 1u);
-            Lmax[e] = sat_u32(h * b * 1000000000ull / lambda_m, 0x7FFFFFFFu);
+            smem[q_off + e] = sat_u32((q_num + q_den - 1ull) / q_den, (uint32_t)T + 1u);
+            smem[lmax_off + e] = sat_u32(h * b * 1000000000ull / lambda_m, 0x7FFFFFFFu);
         }
     }
     __syncthreads();                            // tables ready, both key rows empty
 
     const bool q_grows_with_h = (p.prob.flags & THEMIS_QUEUE_PER_REPLICA) != 0;
+    // one candidate per (c, b): q does not depend on h, or only one h is a candidate
+    const bool single = !q_grows_with_h || p.horizontal || p.vertical || HN == 1;
     int saw_bad_latency = 0;
-    const int lane = tid & 31, warp = tid >> 5;
-    const int c_chunks = (C + 31) / 32;
-    const int n_tasks = NB * c_chunks;
     const uint32_t w_magic = 0xFFFFFFFFu / w_us;            // floor((2^32 - 1) / w)
+    // In the list loop the lanes of a warp cover HNp replica counts x (32 / HNp) pairs of entries.
+    int hn_log = 1;
+    while ((1 << hn_log) < HN && hn_log < 5) ++hn_log;
+    const int HNp = 1 << hn_log;
+    const int groups = 32 >> hn_log;
+    const int group = lane >> hn_log, hk = lane & (HNp - 1);
+    const uint32_t lanemask_lt = (1u << lane) - 1u;
+    const uint32_t list_addr = smem_addr + 4u * (uint32_t)list_off + 16u * (uint32_t)group;
 
     for (int s = 0; s < S; ++s) {
-        uint32_t *keys = (s & 1) ? keys1 : keys0;
+        const int key_off = (s & 1) * pitch;
+        const uint32_t key_addr = smem_addr + 4u * (uint32_t)key_off;
         if (!skip_all) {
             const int h_lo = p.vertical ? rep[s] : 1;
             const int32_t *lat_s = lat + (size_t)s * CB;
-            const uint32_t *Q_s = Q + (p.vertical ? s * NB : 0);
-            const uint32_t *Lmax_s = Lmax + (p.vertical ? s * NB : 0);
-            for (int task = warp; task < n_tasks; task += kScoreThreads / 32) {
-                const int bi = task / c_chunks;
-                const int c = (task - bi * c_chunks) * 32 + lane + 1;
-                if (c > C) continue;
-                const int pair = (c - 1) * NB + bi;
-                const int32_t l_us = lat_s[pair];
-                if (l_us <= 0) { saw_bad_latency = 1; continue; }
-                // Same latency with one core fewer: that candidate reaches the same buckets with
-                // the same replica counts at a lower cost, so this one can never be a minimum
-                // (latency tables are flat over long runs of core counts).
-                if (c > 1 && lat_s[pair - NB] == l_us) continue;
-                // l_b = ceil(l_us / w): quotient estimate by the precomputed reciprocal, then fix up
-                uint32_t l_q = __umulhi((uint32_t)l_us, w_magic);
-                uint32_t l_r = (uint32_t)l_us - l_q * w_us;
-                while (l_r >= w_us) { l_r -= w_us; ++l_q; }
-                const uint32_t l_b = l_q + (l_r != 0u);
-                if (l_b > (uint32_t)T) continue;
-                const int b = p.prob.batch_sizes[bi];
-                // Stop at the fewest replicas when more of them cannot reach another bucket
-                // more cheaply (q does not depend on h), or when only that count is a candidate.
-                const bool q_const = !q_grows_with_h || b == 1 || p.horizontal;
-                const uint32_t *q_row = Q_s + bi * HN;
-                const uint32_t *lmax_row = Lmax_s + bi * HN;
-                // Fewest replicas that sustain lambda: feasibility is monotone in h.  Start
-                // from a floating-point estimate of lambda * l / b and settle it on the exact
-                // integer table; if the estimate is not provably below the answer, scan from 0.
-                const float need = (float)l_us * ((float)lambda_m / ((float)b * 1.0e9f)) - (float)h_lo;
-                int k = (int)fminf(fmaxf(need, 0.0f), (float)HN) - 1;      // one or two below the answer
-                k = max(k, 0);
-                if (k > 0 && (uint32_t)l_us <= lmax_row[k - 1]) k = 0;     // estimate not below: scan from 0
-                while (k < HN && (uint32_t)l_us > lmax_row[k]) ++k;        // cannot sustain lambda
-                uint32_t cost = (uint32_t)(h_lo + k) * (uint32_t)c;
-                uint32_t idx = (uint32_t)((p.horizontal ? 0 : k * CB) + pair);
-                for (; k < HN; ++k, cost += (uint32_t)c, idx += (uint32_t)CB) {
-                    const uint32_t ell = l_b + q_row[k];
-                    if (ell > (uint32_t)T) break;                  // q never shrinks with h
-                    atomicMin(&keys[ell], (cost << 16) | idx);
-                    if (q_const) break;   // more replicas only cost more in this bucket
+            const int row_s = p.vertical ? s * NB : 0;
+            int bi = bi_first, ch = ch_first;
+            while (bi < NB) {
+                const int cidx = ch * 32 + lane;     // core count - 1
+                const int pair = cidx * NB + bi;
+                bool live = cidx < C;
+                uint32_t l_us = 0, l_b = 0;
+                if (live) {
+                    const int32_t v = lat_s[pair];
+                    const int32_t v_prev = cidx > 0 ? lat_s[pair - NB] : 0;
+                    if (v <= 0) saw_bad_latency = 1;
+                    // Same latency with one core fewer: that candidate reaches the same buckets with
+                    // the same replica counts at a lower cost, so this one is never a minimum
+                    // (latency tables are flat over long runs of core counts).
+                    live = v > 0 && v != v_prev;
+                    l_us = (uint32_t)v;
+                    // l_b = ceil(l_us / w): the reciprocal's quotient is at most one too small
+                    uint32_t l_q = __umulhi(l_us, w_magic);
+                    uint32_t l_r = l_us - l_q * w_us;
+                    if (l_r >= w_us) { l_r -= w_us; ++l_q; }
+                    if (l_r >= w_us) { l_r -= w_us; ++l_q; }
+                    l_b = l_q + (l_r != 0u);
+                    live = live && l_b <= (uint32_t)T;
                 }
+                const int q_row = q_off + (row_s + bi) * HN;
+                const int lmax_row = lmax_off + (row_s + bi) * HN;
+                if (single || p.prob.batch_sizes[bi] == 1) {
+                    // More replicas only cost more in the same bucket: the fewest replicas that
+                    // sustain lambda (feasibility is monotone in h) are the pair's one candidate.
+                    if (live) {
+                        int lo = 0, cnt = HN;
+                        while (cnt > 0) {
+                            const int half = cnt >> 1;
+                            if (smem[lmax_row + lo + half] < l_us) { lo += half + 1; cnt -= half + 1; }
+                            else cnt = half;
+                        }
+                        if (lo < HN) {
+                            const uint32_t ell = l_b + smem[q_row + lo];
+                            if (ell <= (uint32_t)T) {
+                                const uint32_t cost = (uint32_t)(h_lo + lo) * (uint32_t)(cidx + 1);
+                                const uint32_t idx = (uint32_t)((p.horizontal ? 0 : lo * CB) + pair);
+                                red_min_shared(key_addr + 4u * ell, (cost << 16) | idx);
+                            }
+                        }
+                    }
+                } else {
+                    // Joint problem with h_max >= 2 (so c <= 32767: at most 65535 candidates per stage).
+                    for (int h0 = 0; h0 < HN; h0 += HNp) {
+                        // pairs that still fit the budget at this chunk's first replica count ...
+                        const bool fits = live && l_b + smem[q_row + h0] <= (uint32_t)T;
+                        if (__ballot_sync(0xFFFFFFFFu, fits) == 0u) break;     // q never shrinks with h
+                        // ... and sustain lambda at its last
+                        const bool in = fits && l_us <= smem[lmax_row + min(h0 + HNp, HN) - 1];
+                        const uint32_t mask = __ballot_sync(0xFFFFFFFFu, in);
+                        const int cnt = __popc(mask);
+                        // compacted entries first; the other slots hold a latency no replica count sustains
+                        if (lane >= cnt)
+                            *reinterpret_cast<uint2 *>(smem + list_off + 2 * lane) = make_uint2(kNeverFits, 0u);
+                        if (in)
+                            *reinterpret_cast<uint2 *>(smem + list_off + 2 * __popc(mask & lanemask_lt)) =
+                                make_uint2(l_us, (l_b << 2) | ((uint32_t)(cidx + 1) << 17));
+                        __syncwarp();
+                        const int k = h0 + hk;                       // this lane's replica count - 1
+                        const bool kv = k < HN;
+                        const uint32_t q4 = 4u * (kv ? smem[q_row + k] : (uint32_t)T + 1u);
+                        const uint32_t lmax = kv ? smem[lmax_row + k] : 0u;
+                        // key = (h * c) << 16 | (h - 1) * CB + (c - 1) * NB + bi  =  c * key_mul + key_add
+                        const uint32_t key_mul = ((uint32_t)(k + 1) << 16) + (uint32_t)NB;
+                        const uint32_t key_add = (uint32_t)(k * CB - NB + bi);
+                        uint32_t entries = list_addr;
+                        for (int i = 0; i < cnt; i += 2 * groups, entries += 16u * (uint32_t)groups)
+                            score_two_entries(entries, q4, lmax, 4u * (uint32_t)T, key_mul, key_add, key_addr, idle_addr);
+                        __syncwarp();
+                    }
+                }
+                bi += bi_step; ch += ch_step;
+                if (ch >= c_chunks) { ch -= c_chunks; ++bi; }
             }
         }
         __syncthreads();
@@ -149,8 +256,8 @@ score_kernel(const Params p)
         int32_t *G_row = p.G + ((size_t)n * S + s) * pitch;
         uint16_t *Garg_row = p.Garg + ((size_t)n * S + s) * pitch;
         for (int l4 = tid * 4; l4 < pitch; l4 += kScoreThreads * 4) {
-            const uint4 k4 = *reinterpret_cast<const uint4 *>(keys + l4);
-            *reinterpret_cast<uint4 *>(keys + l4) = make_uint4(kEmptyKey, kEmptyKey, kEmptyKey, kEmptyKey);
+            const uint4 k4 = *reinterpret_cast<const uint4 *>(smem + key_off + l4);
+            *reinterpret_cast<uint4 *>(smem + key_off + l4) = make_uint4(kEmptyKey, kEmptyKey, kEmptyKey, kEmptyKey);
             const uint32_t kk[4] = {k4.x, k4.y, k4.z, k4.w};
             int4 g;
             int32_t *gv = reinterpret_cast<int32_t *>(&g);
@@ -159,10 +266,11 @@ score_kernel(const Params p)
             for (int i = 0; i < 4; ++i) {
                 const bool empty = kk[i] == kEmptyKey;
                 gv[i] = empty ? THEMIS_G_INF : (int32_t)(kk[i] >> 16);
-                a[i] = empty ? 0u : (kk[i] & 0xFFFFu);
+                a[i] = empty ? 0u : kk[i];
             }
             *reinterpret_cast<int4 *>(G_row + l4) = g;
-            *reinterpret_cast<uint2 *>(Garg_row + l4) = make_uint2(a[0] | (a[1] << 16), a[2] | (a[3] << 16));
+            *reinterpret_cast<uint2 *>(Garg_row + l4) =
+                make_uint2(__byte_perm(a[0], a[1], 0x5410), __byte_perm(a[2], a[3], 0x5410));
         }
     }
     const int any_bad = __syncthreads_or(saw_bad_latency);
@@ -175,7 +283,7 @@ cudaError_t launch_score(const Params &p, cudaStream_t stream)
 {
     const size_t table = p.vertical ? (size_t)p.prob.n_stages * p.prob.n_batch
                                     : (size_t)p.prob.n_batch * p.prob.h_max;
-    const size_t smem = sizeof(uint32_t) * (2u * (size_t)p.pitch + 2u * table);
+    const size_t smem = sizeof(uint32_t) * (2u * (size_t)p.pitch + 2u * table + 4u + kScoreWarps * kListWords + 32u);
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)smem);
