@@ -300,6 +300,9 @@ SHAPES = [  # n_stages, c_max, batch sizes, h_max, T, bucket_us, vertical, rate 
     (5, 64, (1, 2, 4, 8, 16, 32, 64, 128), 16, 4096, 250, False, (100.0, 900.0)),   # T a power of two
     (6, 16, (1, 2, 4, 8), 64, 2056, 500, False, (200.0, 3000.0)),            # eight cells beyond the tiles
     (3, 7, (2, 3), 5, 263, 1000, True, (10.0, 80.0)),
+    (3, 20, (1, 2, 4), 1, 300, 1000, False, (5.0, 200.0)),                   # joint problem with one replica count
+    (2, 40000, (3,), 1, 500, 1000, False, (5.0, 50.0)),                      # core counts beyond 15 bits
+    (3, 9, (1, 2, 4, 8), 40, 900, 500, False, (50.0, 2500.0)),               # replica counts: a full and a ragged chunk of 32
 ]
 
 
