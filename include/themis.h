@@ -320,6 +320,23 @@ int themis_fit_profiles_batch(int32_t n_models, int32_t n_samples, const int32_t
 int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_sink,
                      void *cuda_stream);
 
+/*
+ * Bounded-wait probe (not part of the method; the paper has no counterpart).  The
+ * recurrence kernels stage every row G_s with an asynchronous bulk copy and wait for
+ * it on a shared-memory barrier; that wait gives up after a fixed number of attempts
+ * and the instance reports THEMIS_STATUS_TIMEOUT instead of hanging.  This entry point
+ * runs the same wait routine in a one-warp kernel on two barriers: one whose 16-byte
+ * copy from d_src16 (16-byte aligned) is issued (waited for with the kernels' own
+ * limit), and one that expects 16 bytes which nothing delivers (waited for with
+ * `max_polls` attempts, 1 .. 2^20).  Results:
+ *   d_status[0] = THEMIS_STATUS_OK and d_dst16[0..3] = d_src16[0..3]  (the copy landed);
+ *   d_status[1] = THEMIS_STATUS_TIMEOUT                               (the wait ran out);
+ * the kernel returns normally in both cases and the context stays usable.
+ * Returns THEMIS_E_INVALID_ARG for a NULL or misaligned pointer or max_polls out of range.
+ */
+int themis_wait_probe(int32_t max_polls, const uint32_t *d_src16, uint32_t *d_dst16, int32_t *d_status,
+                      void *cuda_stream);
+
 /* Which min-plus kernel themis_minplus_batch and the solvers run (an implementation
  * choice; the paper has no counterpart).  Results do not depend on it; what the rows
  * of the workspace hold does.

@@ -530,6 +530,17 @@ int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_s
     return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
 }
 
+int themis_wait_probe(int32_t max_polls, const uint32_t *d_src16, uint32_t *d_dst16, int32_t *d_status,
+                      void *cuda_stream)
+{
+    if (max_polls < 1 || max_polls > (1 << 20) || !d_src16 || !d_dst16 || !d_status ||
+        ((uintptr_t)d_src16 & 15u))
+        return THEMIS_E_INVALID_ARG;
+    cudaError_t e = launch_wait_probe((uint32_t)max_polls, d_src16, d_dst16, d_status,
+                                      static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
+}
+
 int themis_set_minplus_mode(int mode)
 {
     if (mode < 0 || mode > 3) return THEMIS_E_INVALID_ARG;

@@ -98,5 +98,7 @@ cudaError_t launch_fit_profiles(int n_models, int n_samples, const int32_t *samp
                                 double *coeffs, int32_t *lat_us, int32_t *status, cudaStream_t st);
 cudaError_t launch_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *sink,
                              cudaStream_t stream);
+cudaError_t launch_wait_probe(uint32_t max_polls, const uint32_t *src16, uint32_t *dst16, int32_t *status,
+                              cudaStream_t stream);
 
 }  // namespace themis

@@ -7,6 +7,7 @@
 // Form 5 times the packed kernel's own inner step instead (themis_minplus16_step.cuh):
 // columns of 256 chunk steps with the operands loaded from shared memory exactly as in
 // the recurrence kernel, but no stages, barriers or global traffic around them.
+#include "themis_async.cuh"
 #include "themis_internal.h"
 #include "themis_minplus16_step.cuh"
 
@@ -110,6 +111,35 @@ __global__ void __launch_bounds__(256) step_probe_kernel(int iters, uint32_t *si
     sink[blockIdx.x * blockDim.x + tid] = r;
 }
 
+// Bounded-wait probe: the same mbarrier wait the recurrence kernels use, once on a copy that
+// is issued (must complete; the kernels' own limit, so that no copy is in flight when the block
+// leaves) and once on a transaction that nothing delivers (must give up after `max_polls`
+// attempts and report it).  One warp; the kernel returns normally in both cases.
+__global__ void wait_probe_kernel(uint32_t max_polls, const uint32_t *src16, uint32_t *dst16, int32_t *status)
+{
+    __shared__ __align__(16) uint32_t buf[4];
+    __shared__ __align__(8) uint64_t bar[2];
+    if (threadIdx.x == 0) {
+        mbar_init(&bar[0], 1);
+        mbar_init(&bar[1], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_expect_tx(&bar[0], 16);
+        bulk_load(buf, src16, 16, &bar[0]);
+        mbar_expect_tx(&bar[1], 16);              // these 16 bytes never come
+    }
+    const bool arrived = mbar_wait(&bar[0], 0);
+    if (arrived && threadIdx.x < 4) dst16[threadIdx.x] = buf[threadIdx.x];
+    const bool never = mbar_wait(&bar[1], 0, max_polls);
+    if (threadIdx.x == 0) {
+        status[0] = arrived ? THEMIS_STATUS_OK : THEMIS_STATUS_TIMEOUT;
+        status[1] = never ? THEMIS_STATUS_OK : THEMIS_STATUS_TIMEOUT;
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *sink, cudaStream_t stream)
@@ -125,6 +155,13 @@ cudaError_t launch_alu_probe(int mode, int blocks, int threads, int iters, uint3
             break;
         default: alu_probe_kernel<4><<<blocks, threads, 0, stream>>>(iters, sink); break;
     }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_wait_probe(uint32_t max_polls, const uint32_t *src16, uint32_t *dst16, int32_t *status,
+                              cudaStream_t stream)
+{
+    wait_probe_kernel<<<1, 32, 0, stream>>>(max_polls, src16, dst16, status);
     return cudaGetLastError();
 }
 

@@ -31,7 +31,7 @@ INF16 = 0x7FFF
 EXPORTS = (
     "themis_version", "themis_strerror", "themis_workspace_bytes", "themis_workspace_layout",
     "themis_solve_batch", "themis_solve_vertical_batch", "themis_score_batch", "themis_minplus_batch",
-    "themis_host_workspace_bytes", "themis_solve_batch_host", "themis_alu_probe",
+    "themis_host_workspace_bytes", "themis_solve_batch_host", "themis_alu_probe", "themis_wait_probe",
     "themis_set_minplus_tile", "themis_solve_batch_static", "themis_set_minplus_mode",
     "themis_solve_horizontal_batch", "themis_fallback_workspace_bytes", "themis_vertical_fallback_batch",
     "themis_fit_profiles_batch", "themis_configs_equal_batch",
@@ -110,6 +110,7 @@ def _load() -> ctypes.CDLL:
     lib.themis_fit_profiles_batch.argtypes = [ctypes.c_int32, ctypes.c_int32, vp, vp, vp, ctypes.c_int32,
                                               ctypes.c_int32, vp, vp, vp, vp, vp]
     lib.themis_alu_probe.argtypes = [ctypes.c_int] * 4 + [vp, vp]
+    lib.themis_wait_probe.argtypes = [ctypes.c_int32, vp, vp, vp, vp]
     lib.themis_set_minplus_tile.argtypes = [ctypes.c_int]
     lib.themis_set_minplus_mode.argtypes = [ctypes.c_int]
     for name in EXPORTS:
@@ -276,6 +277,11 @@ def themis_alu_probe(mode: int, blocks: int, threads: int, iters: int, sink) -> 
         raise ValueError("sink too small")
     _check(_lib.themis_alu_probe(mode, blocks, threads, iters, _dptr(sink, torch.uint32, "sink"), _stream()),
            "themis_alu_probe")
+
+
+def themis_wait_probe(max_polls: int, src16, dst16, status) -> None:
+    _check(_lib.themis_wait_probe(max_polls, _dptr(src16, torch.uint32, "src16"), _dptr(dst16, torch.uint32, "dst16"),
+                                  _dptr(status, torch.int32, "status"), _stream()), "themis_wait_probe")
 
 
 def themis_set_minplus_mode(mode: int) -> None:

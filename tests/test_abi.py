@@ -99,6 +99,9 @@ def test_pointer_and_workspace_checks(S):
     assert lib.themis_solve_vertical_batch(ctypes.byref(p), one, None, one, None, res, one, need, None) == S.E_INVALID_ARG
     assert lib.themis_solve_batch_host(ctypes.byref(p), one, None, one, None, res, one, need, None) == S.E_WORKSPACE_TOO_SMALL
     assert lib.themis_alu_probe(9, 1, 32, 1, one, None) == S.E_INVALID_ARG
+    assert lib.themis_wait_probe(0, one, one, one, None) == S.E_INVALID_ARG
+    assert lib.themis_wait_probe(100, ctypes.c_void_p(260), one, one, None) == S.E_INVALID_ARG
+    assert lib.themis_wait_probe(100, one, None, one, None) == S.E_INVALID_ARG
     assert lib.themis_set_minplus_tile(12) == S.E_INVALID_ARG
     assert lib.themis_set_minplus_tile(0) == S.OK
     assert lib.themis_set_minplus_mode(4) == S.E_INVALID_ARG and lib.themis_set_minplus_mode(0) == S.OK

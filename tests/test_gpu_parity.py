@@ -537,3 +537,19 @@ def test_full_size_config5_sampled(S, oracle_mod, mode):
     sub = dataclasses.replace(wl, n_instances=len(pick), profile_id=wl.profile_id[pick].copy(),
                               lambda_mrps=wl.lambda_mrps[pick].copy())
     _assert_results_equal(gpu, _oracle_cached(oracle_mod, ("cfg5", tuple(pick.tolist())), sub), idx=pick)
+
+
+def test_bounded_wait_gives_up_and_reports(S, oracle_mod):
+    """The recurrence kernels' barrier wait, run on a transaction that nothing delivers: it
+    gives up after its attempts, the kernel returns THEMIS_STATUS_TIMEOUT for that barrier and
+    the copy that was issued still lands; the context stays usable (a solve right after)."""
+    import torch
+    src = torch.arange(11, 15, dtype=torch.int32, device="cuda").view(torch.uint32)
+    dst = torch.zeros(4, dtype=torch.uint32, device="cuda")
+    status = torch.full((2,), 99, dtype=torch.int32, device="cuda")
+    S.themis_wait_probe(2000, src, dst, status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [S.STATUS_OK, S.STATUS_TIMEOUT]
+    assert dst.view(torch.int32).cpu().tolist() == [11, 12, 13, 14]
+    wl = W.make_workload(1)
+    _assert_results_equal(_gpu_solve(S, wl), oracle_mod.solve_batch(wl))
