@@ -32,8 +32,6 @@ namespace themis {
 namespace {
 
 constexpr uint32_t kEmptyKey = 0xFFFFFFFFu;
-constexpr int kScoreThreads = 256;
-constexpr int kScoreWarps = kScoreThreads / 32;
 constexpr int kListWords = 64;        // per warp: 32 entries of two words
 constexpr uint32_t kNeverFits = 0xFFFFFFFFu;   // latency of a padding entry: above every Lmax
 
@@ -83,9 +81,13 @@ __device__ __forceinline__ uint32_t sat_u32(unsigned long long v, uint32_t cap)
     return v > (unsigned long long)cap ? cap : (uint32_t)v;
 }
 
-__global__ void __launch_bounds__(kScoreThreads, 6)
+// THREADS: 256, or 128 for short budgets, where a stage is so little work that the per-warp
+// cost of a stage (loop, barrier, row addresses) shows; registers for 1536 threads per SM.
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS, 1536 / THREADS)
 score_kernel(const Params p)
 {
+    constexpr int kScoreThreads = THREADS, kScoreWarps = THREADS / 32;
     extern __shared__ __align__(16) uint32_t smem[];
     const int n = blockIdx.x;
     if (p.active && !p.active[n]) return;
@@ -283,13 +285,14 @@ cudaError_t launch_score(const Params &p, cudaStream_t stream)
 {
     const size_t table = p.vertical ? (size_t)p.prob.n_stages * p.prob.n_batch
                                     : (size_t)p.prob.n_batch * p.prob.h_max;
-    const size_t smem = sizeof(uint32_t) * (2u * (size_t)p.pitch + 2u * table + 4u + kScoreWarps * kListWords + 32u);
+    const int threads = p.pitch <= 1024 ? 128 : 256;
+    const size_t smem = sizeof(uint32_t) * (2u * (size_t)p.pitch + 2u * table + 4u + (threads / 32) * kListWords + 32u);
+    auto kernel = threads == 128 ? score_kernel<128> : score_kernel<256>;
     if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    score_kernel<<<p.prob.n_instances, kScoreThreads, smem, stream>>>(p);
+    kernel<<<p.prob.n_instances, threads, smem, stream>>>(p);
     return cudaGetLastError();
 }
 
