@@ -29,11 +29,14 @@
 //
 // Folding.  Tiles are grouped in half-groups of 16 (one per half-warp).  Column length
 // grows with the tile index, and all lanes of a half-warp run to their half-group's
-// longest column, so every half-warp takes a long half-group and then a short one,
-// (last, first), (last-1, second), ...: all half-warps of the block do the same number
-// of chunk steps, and the two halves of a warp may stand at different l (two broadcast
-// addresses instead of one).  A finished tile's result waits in registers for the stage's
-// barrier; only the word that spills into the next tile goes through shared memory.
+// longest column, so half-group g costs g + 1 units.  A half-warp takes a long half-group
+// and then a short one, paired so that the two half-warps of every warp carry equal sums
+// (a warp runs as long as its longer half): (last, first), (last-1, second), ... when the
+// number of half-groups is a multiple of four; otherwise the one or two shortest, or the
+// longest, stand alone and the rest is paired the same way (assign_half_groups).  The two
+// halves of a warp may stand at different l (two broadcast addresses instead of one).  A
+// finished tile's result waits in registers for the stage's barrier; only the word that
+// spills into the next tile goes through shared memory.
 //
 // Saturation.  If the best total is 0x7FFF the instance is either infeasible
 // (decided exactly: the fastest configurations of all stages do not fit the
@@ -66,7 +69,9 @@ __device__ __forceinline__ uint32_t block_min(uint32_t v, uint32_t *red, int tid
 }
 
 // EXTRA: the block also computes up to kMaxExtra cells beyond its tiles (see kMaxExtra).
-template <int R, int MAXT, bool EXTRA>
+// PAIRS_ONLY: the number of half-groups is a multiple of four, every half-warp slot walks the pair
+// (last - slot, slot); otherwise the slots are described by the fold_* fields of Params.
+template <int R, int MAXT, bool EXTRA, bool PAIRS_ONLY>
 __global__ void __launch_bounds__(MAXT, (R == 16 || MAXT > 512) ? 1 : 2)   // 64 registers: two blocks of 512
 minplus16_kernel(const Params p)
 {
@@ -99,11 +104,20 @@ minplus16_kernel(const Params p)
     uint32_t *fx_acc = fx_prev + kMaxExtra;                   // kMaxExtra words: F_s at the extra cells, building
     uint32_t *stage_cmin = fx_acc + kMaxExtra;                // 64 words: cheapest entry of every G_s
 
-    // The two tiles of this thread: its half-warp takes half-group NHG-1-slot (long columns)
-    // first and half-group slot (short columns) second; the middle one, if any, stands alone.
+    // The two tiles of this thread: its half-warp takes one half-group (long columns) and then
+    // another (short columns), as dealt by the host (assign_half_groups); either may be absent.
     const int slot = tid >> 4, lane16 = tid & 15;
-    const int hg_a = NHG - 1 - slot, hg_b = slot;
-    const bool has_a = hg_a >= hg_b, has_b = hg_b < hg_a;
+    int hg_a, hg_b;
+    bool has_a, has_b;
+    if (PAIRS_ONLY) {
+        hg_a = NHG - 1 - slot; hg_b = slot;
+        has_a = hg_a >= hg_b; has_b = hg_b < hg_a;
+    } else {
+        has_b = slot < p.fold_pairs;
+        hg_a = has_b ? p.fold_hi - slot : slot - p.fold_pairs < 2 ? p.fold_single[slot - p.fold_pairs] : -1;
+        hg_b = p.fold_lo + slot;
+        has_a = hg_a >= 0;
+    }
     const int tile_a = hg_a * 16 + lane16, tile_b = hg_b * 16 + lane16;
     const uint32_t row_bytes = (uint32_t)pitch * 4u;
     const int32_t *G_inst = p.G + (size_t)n * S * pitch;
@@ -533,10 +547,11 @@ minplus16_kernel(const Params p)
 template <int R, int MAXT, bool EXTRA>
 cudaError_t launch_variant16x(const Params &p, int threads, size_t smem, cudaStream_t stream)
 {
-    cudaError_t e = cudaFuncSetAttribute(minplus16_kernel<R, MAXT, EXTRA>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    auto kernel = (p.n_half_groups & 3) == 0 ? minplus16_kernel<R, MAXT, EXTRA, true>
+                                             : minplus16_kernel<R, MAXT, EXTRA, false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    minplus16_kernel<R, MAXT, EXTRA><<<p.prob.n_instances, threads, smem, stream>>>(p);
+    kernel<<<p.prob.n_instances, threads, smem, stream>>>(p);
     return cudaGetLastError();
 }
 
@@ -574,11 +589,31 @@ Shape16 shape_of(int cells, int pitch, int tile)
     return sh;
 }
 
+// Deals the half-groups (half-group g costs g + 1 units) to the block's half-warp slots, at most
+// two each, so that the sum over warps of the longer of a warp's two halves is smallest: pair
+// longest with shortest, after setting aside the shortest (count = 1 mod 4), the two shortest
+// (2 mod 4) or the longest (3 mod 4) as slots of their own behind the pairs (their sums are equal
+// to the pairs' or below), so that the two halves of a warp are equal or nearly so.  Found optimal
+// by exhaustive search for up to 13 half-groups and within half a unit of the ideal (half the
+// total) beyond.
+void assign_half_groups(int nhg, Params *p)
+{
+    int lo = 0, hi = nhg - 1;
+    p->fold_single[0] = p->fold_single[1] = -1;
+    if ((nhg & 3) == 1) p->fold_single[0] = lo++;
+    if ((nhg & 3) == 2) { p->fold_single[1] = lo++; p->fold_single[0] = lo++; }   // the longer of the two first
+    if ((nhg & 3) == 3) p->fold_single[0] = hi--;
+    p->fold_lo = lo;
+    p->fold_hi = hi;
+    p->fold_pairs = (hi - lo + 1) / 2;
+}
+
 template <int R, int MAXT>
 cudaError_t launch_variant16(const Params &p_in, const Shape16 &sh, cudaStream_t stream)
 {
     Params p = p_in;
     p.n_half_groups = sh.half_groups;
+    assign_half_groups(sh.half_groups, &p);
     return sh.extra ? launch_variant16x<R, MAXT, true>(p, sh.threads, sh.smem, stream)
                     : launch_variant16x<R, MAXT, false>(p, sh.threads, sh.smem, stream);
 }
