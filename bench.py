@@ -67,6 +67,11 @@ def parse_args():
                     help="0: packed 16-bit min-plus kernel (default); 1: 32-bit kernel")
     ap.add_argument("--minplus-tile", type=int, default=0, choices=[0, 4, 8, 16],
                     help="cells per thread tile of the recurrence kernels (0: the library's choice)")
+    ap.add_argument("--entry", default="solve", choices=["solve", "fallback", "horizontal", "fit"],
+                    help="solve: the headline step (default).  The others time one of the further entry points "
+                         "on one GPU with the CPU oracle beside it: fallback = themis_vertical_fallback_batch on the "
+                         "day-long trace; horizontal = Algorithm 2 at the current and a predicted rate plus the "
+                         "stability test; fit = themis_fit_profiles_batch")
     ap.add_argument("--pruned-steps", type=int, default=5,
                     help="extra steps with the recurrence restricted to undominated entries (0: skip)")
     return ap.parse_args()
@@ -448,6 +453,162 @@ def run_ours(args):
     print(json.dumps(line), flush=True)
 
 
+# --------------------------------------------------------------------------- further entry points
+
+def _timed(torch, fn, steps, warmup):
+    """Average milliseconds of fn() over `steps` calls after `warmup` calls (CUDA events on the
+    current stream, synchronised on both sides)."""
+    for _ in range(max(1, warmup)):
+        fn()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(steps):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / steps
+
+
+def run_entry(args):
+    """One of the entry points beyond the headline solve: device time per call on resident inputs,
+    the oracle's time on a sample of the same inputs, and whether the two agree on that sample."""
+    import dataclasses
+    import numpy as np
+    import torch
+    from paper_2407_14843_b200 import build as _build, workloads
+    _build.build_library()
+    import oracle
+    oracle.build()
+    cores = os.cpu_count() or 1
+    base = {"n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "higher_is_better": True, "data": "synthetic",
+            "vs_baseline": None}
+
+    if args.entry == "fit":
+        from oracle import profile_fit
+        n_models = args.instances or 65536
+        c_max, batches = 64, (1, 2, 4, 8, 16, 32, 64)
+        sb, sc, lat, _ = workloads.profile_samples(77, n_models)
+        n_ref = min(n_models, 2048)
+        t = time.perf_counter()
+        ref_c, ref_t, ref_s = profile_fit.fit_profiles(sb, sc, lat[:n_ref], c_max, batches)
+        cpu_s = time.perf_counter() - t
+        torch.cuda.set_device(0)
+        from paper_2407_14843_b200 import solver
+        dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+        d_sb, d_sc, d_lat, d_b = dev(sb), dev(sc), dev(lat), dev(np.asarray(batches, np.int32))
+        coeffs = torch.empty((n_models, 4), dtype=torch.float64, device="cuda")
+        tab = torch.empty((n_models, c_max, len(batches)), dtype=torch.int32, device="cuda")
+        status = torch.empty(n_models, dtype=torch.int32, device="cuda")
+        ms = _timed(torch, lambda: solver.themis_fit_profiles_batch(d_sb, d_sc, d_lat, c_max, d_b, coeffs, tab, status),
+                    args.steps, args.warmup)
+        diff = np.abs(tab[:n_ref].cpu().numpy().astype(np.int64) - ref_t)
+        same = bool(np.allclose(coeffs[:n_ref].cpu().numpy(), ref_c, rtol=1e-8, atol=1e-10) and diff.max() <= 1
+                    and np.array_equal(status[:n_ref].cpu().numpy(), ref_s))
+        table_bytes = tab.numel() * 4 + lat.nbytes
+        hbm_peak, hbm_kind = measured_hbm_peak()
+        line = dict(base, metric="profile_fits_per_s", value=n_models / (ms * 1e-3), unit="models/s", ms_per_step=ms,
+                    dtype="f64", scaling="weak",
+                    config={"workload": f"Eq. 1 fit: {n_models} models x {lat.shape[1]} profiled (b, c) points, tables "
+                                        f"{c_max} x {len(batches)}"},
+                    roofline={"kernel": "fit_profiles_kernel", "bound": "hbm", "achieved": table_bytes / (ms * 1e-3) / 1e9,
+                              "peak": hbm_peak, "unit": "GB/s", "frac": table_bytes / (ms * 1e-3) / 1e9 / hbm_peak,
+                              "traffic": None, "peak_kind": f"of {hbm_kind}",
+                              "algorithmic_bytes_per_launch": table_bytes},
+                    cpu_baseline={"value": n_ref / cpu_s, "unit": "models/s", "cores": 1, "kind": "oracle",
+                                  "sample": f"first {n_ref} models, {cpu_s:.2f} s (numpy lstsq per model)"},
+                    matches_oracle_on_sample=same, gpu_launches=args.steps)
+        print(json.dumps(line), flush=True)
+        return
+
+    if args.entry == "fallback":
+        wl = workloads.make_workload(3, args.instances)
+        res = 1000                                               # search points every 1 request/s
+        n_ref = min(wl.n_instances, 4096)
+        # the sample: the busiest seconds (where the last branch is taken) and a stride of quiet ones
+        hot = np.argsort(wl.lambda_mrps)[-n_ref // 2:]
+        pick = np.unique(np.concatenate([hot, np.arange(0, wl.n_instances, max(1, 2 * wl.n_instances // n_ref))]))
+        sub = dataclasses.replace(wl, n_instances=len(pick), profile_id=wl.profile_id[pick].copy(),
+                                  lambda_mrps=wl.lambda_mrps[pick].copy(), replicas=wl.replicas[pick].copy())
+        t = time.perf_counter()
+        ref = oracle.vertical_fallback_batch(sub, res)
+        cpu_s = time.perf_counter() - t
+        torch.cuda.set_device(0)
+        from paper_2407_14843_b200 import solver
+        prob = solver.Problem.of_workload(wl)
+        dev = solver.workload_to_device(wl)
+        ws = torch.empty(solver.themis_fallback_workspace_bytes(prob), dtype=torch.uint8, device="cuda")
+        out = solver.alloc_result(wl.n_instances, wl.n_stages)
+        lam_v = torch.empty(wl.n_instances, dtype=torch.uint32, device="cuda")
+        extra = torch.empty((wl.n_instances, wl.n_stages), dtype=torch.int32, device="cuda")
+        lam_max = int(wl.lambda_mrps.max())
+        call = lambda: solver.themis_vertical_fallback_batch(prob, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"],
+                                                             dev["replicas"], res, lam_max, out, lam_v, extra, ws)
+        ms = _timed(torch, call, args.steps, args.warmup)
+        ms_plain = _timed(torch, lambda: solver.themis_solve_vertical_batch(
+            prob, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"], dev["replicas"], out, ws), args.steps, 1)
+        call()
+        torch.cuda.synchronize()
+        st = out["status"].cpu().numpy()
+        same = all(np.array_equal(out[k].cpu().numpy()[pick], ref[k]) for k in out) \
+            and np.array_equal(lam_v.cpu().numpy()[pick], ref["lambda_vertical"]) \
+            and np.array_equal(extra.cpu().numpy()[pick], ref["extra_replicas"])
+        rounds = max(0, int(np.ceil(np.log2(max(1, (lam_max + res - 1) // res)))))
+        line = dict(base, metric="fallback_instances_per_s", value=wl.n_instances / (ms * 1e-3), unit=UNIT,
+                    ms_per_step=ms, dtype="u16", scaling="weak",
+                    config={"workload": f"config 3 ({wl.name}): every second of the day, Algorithm 1 with its last "
+                                        f"branch, search points every {res} mrps",
+                            "instances": wl.n_instances, "stages": wl.n_stages, "T": wl.T,
+                            "bisection_rounds": rounds, "split_instances": int((st == 2).sum()),
+                            "served_in_place": int((st == 0).sum())},
+                    ms_plain_vertical_solve=ms_plain, ms_search_and_second_solve=ms - ms_plain,
+                    cpu_baseline={"value": len(pick) / cpu_s, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                  "sample": f"{len(pick)} seconds of the trace (the busiest {len(hot)} and a stride of "
+                                            f"the rest), {cpu_s:.1f} s"},
+                    matches_oracle_on_sample=bool(same), gpu_launches=None)
+        print(json.dumps(line), flush=True)
+        return
+
+    # horizontal: Algorithm 2 at the current and at the predicted rate, then the stability test
+    full = workloads.make_workload(2, args.instances)
+    h_max = 256
+    wl = dataclasses.replace(full, c_max=1, h_max=h_max, lat_us=np.ascontiguousarray(full.lat_us[:, :, :1, :]))
+    growth = 1.0 + 0.3 * workloads.rand_uniform(7501, 1, np.arange(wl.n_instances, dtype=np.uint64))
+    pred = dataclasses.replace(wl, lambda_mrps=(wl.lambda_mrps * growth).astype(np.uint32))
+    t = time.perf_counter()
+    a, b = oracle.solve_batch(wl, horizontal=True), oracle.solve_batch(pred, horizontal=True)
+    cpu_s = time.perf_counter() - t
+    expect = (a["status"] == 0) & (b["status"] == 0) & np.all(a["h"] == b["h"], axis=1) \
+        & np.all(a["b"] == b["b"], axis=1) & np.all(a["c"] == b["c"], axis=1)
+    torch.cuda.set_device(0)
+    from paper_2407_14843_b200 import solver
+    prob = solver.Problem.of_workload(wl)
+    d_now, d_pred = solver.workload_to_device(wl), solver.workload_to_device(pred)
+    ws = solver.alloc_workspace(prob, False)
+    o_now, o_pred = (solver.alloc_result(wl.n_instances, wl.n_stages) for _ in range(2))
+    stable = torch.empty(wl.n_instances, dtype=torch.int32, device="cuda")
+
+    def call():
+        solver.themis_solve_horizontal_batch(prob, d_now["lat_us"], d_now["profile_id"], d_now["lambda_mrps"], o_now, ws)
+        solver.themis_solve_horizontal_batch(prob, d_pred["lat_us"], d_pred["profile_id"], d_pred["lambda_mrps"], o_pred, ws)
+        solver.themis_configs_equal_batch(o_now, o_pred, stable)
+
+    ms = _timed(torch, call, args.steps, args.warmup)
+    same = bool(np.array_equal(stable.cpu().numpy().astype(bool), expect)
+                and all(np.array_equal(o_now[k].cpu().numpy(), a[k]) for k in o_now))
+    line = dict(base, metric="stability_tests_per_s", value=wl.n_instances / (ms * 1e-3), unit=UNIT, ms_per_step=ms,
+                dtype="u16", scaling="weak",
+                config={"workload": f"config 2 shapes with one-core replicas (Algorithm 2, up to {h_max} replicas): two "
+                                    "solves (current rate, predicted rate up to 30 % higher) and the comparison",
+                        "instances": wl.n_instances, "stages": wl.n_stages, "T": wl.T,
+                        "batch_sizes": list(wl.batch_sizes), "stable_instances": int(expect.sum()),
+                        "infeasible_now": int((a["status"] == 1).sum())},
+                cpu_baseline={"value": wl.n_instances / cpu_s, "unit": UNIT, "cores": cores, "kind": "oracle",
+                              "sample": f"all {wl.n_instances} instances, both rates, {cpu_s:.1f} s"},
+                matches_oracle_on_sample=same, gpu_launches=5 * args.steps)
+    print(json.dumps(line), flush=True)
+
+
 def run_alu_probe():
     """Rates of themis_alu_probe in all its forms (updates per SM per clock at the boost
     clock, and TOP/s counting two operations per cell update).  Forms 0-4 keep their
@@ -489,6 +650,8 @@ def main():
         run_alu_probe()
     elif args.impl == "reference":
         run_reference(args)
+    elif args.entry != "solve":
+        run_entry(args)
     else:
         run_ours(args)
 

@@ -175,8 +175,11 @@ int themis_solve_vertical_batch(const themis_problem_t *problem, const int32_t *
  *   d_extra_replicas     [N][S] int32 out: 0 except for THEMIS_STATUS_SPLIT instances
  *   out                  the vertical part's configuration (for split instances: the
  *                        solve at lambda_vertical), status in {0, 1, 2, < 0}
- * Every round re-solves only the instances still searching.  Workspace:
- * themis_fallback_workspace_bytes.
+ * A search point only has to be classified as served or not, and a rate is served
+ * exactly when the fastest feasible candidates of all stages fit the budget
+ * together, so the search of an instance runs inside one kernel without the
+ * recurrence; the recurrence runs twice, at the full rate and at the rate found
+ * (for the searching instances only).  Workspace: themis_fallback_workspace_bytes.
  */
 int themis_fallback_workspace_bytes(const themis_problem_t *problem, size_t *out_bytes);
 int themis_vertical_fallback_batch(const themis_problem_t *problem, const int32_t *d_lat_us,

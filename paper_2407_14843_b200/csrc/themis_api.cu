@@ -178,7 +178,8 @@ int solve_impl(const themis_problem_t *pr, const int32_t *lat, const int32_t *pi
     return rc;
 }
 
-// Search state and trial results appended to the solver workspace by the fallback entry point.
+// Search state appended to the solver workspace by the fallback entry point (the result-shaped
+// arrays behind it are reserved).
 struct FallbackStage {
     size_t lo, hi, active, iter_active, trial_lambda, h, c, b, cost, latb, status, total;
 };
@@ -347,13 +348,6 @@ int themis_vertical_fallback_batch(const themis_problem_t *problem, const int32_
     int32_t *active = reinterpret_cast<int32_t *>(base + F.active);
     int32_t *iter_active = reinterpret_cast<int32_t *>(base + F.iter_active);
     uint32_t *trial_lambda = reinterpret_cast<uint32_t *>(base + F.trial_lambda);
-    themis_result_t trial;
-    trial.h = reinterpret_cast<int32_t *>(base + F.h);
-    trial.c = reinterpret_cast<int32_t *>(base + F.c);
-    trial.b = reinterpret_cast<int32_t *>(base + F.b);
-    trial.total_cost = reinterpret_cast<int32_t *>(base + F.cost);
-    trial.latency_buckets = reinterpret_cast<int32_t *>(base + F.latb);
-    trial.status = reinterpret_cast<int32_t *>(base + F.status);
 
     // 1. the whole load on the replicas in place
     rc = solve_impl(problem, d_lat_us, d_profile_id, d_lambda_mrps, d_replicas, SolveOpts{kVertical}, out, d_workspace,
@@ -361,19 +355,17 @@ int themis_vertical_fallback_batch(const themis_problem_t *problem, const int32_
     if (rc != THEMIS_OK) return rc;
     cudaError_t e = launch_fb_init(N, resolution_mrps, out.status, d_lambda_mrps, lo, hi, active, st);
     if (e != cudaSuccess) return fail_cuda(e);
-    // 2. bisection rounds: enough to close an interval of ceil(max / resolution) points
+    // 2. bisection: enough rounds to close an interval of ceil(max / resolution) points
     const unsigned long long points = ((unsigned long long)lambda_max_mrps + resolution_mrps - 1) / resolution_mrps;
     int rounds = 0;
     while ((1ull << rounds) < points) ++rounds;
-    for (int r = 0; r < rounds; ++r) {
-        e = launch_fb_trial(N, resolution_mrps, lo, hi, active, iter_active, trial_lambda, st);
-        if (e != cudaSuccess) return fail_cuda(e);
-        rc = solve_impl(problem, d_lat_us, d_profile_id, trial_lambda, d_replicas,
-                        SolveOpts{kVertical, iter_active}, trial, d_workspace, L.total_bytes, st);
-        if (rc != THEMIS_OK) return rc;
-        e = launch_fb_update(N, lo, hi, iter_active, trial.status, st);
-        if (e != cudaSuccess) return fail_cuda(e);
-    }
+    Params P;
+    rc = make_params(problem, SolveOpts{kVertical}, d_workspace, L.total_bytes, &P);
+    if (rc != THEMIS_OK) return rc;
+    P.lat_us = d_lat_us; P.profile_id = d_profile_id; P.lambda_mrps = d_lambda_mrps; P.replicas = d_replicas;
+    P.out = out;
+    e = launch_fb_bisect(P, rounds, resolution_mrps, active, lo, hi, st);
+    if (e != cudaSuccess) return fail_cuda(e);
     // 3. the vertical part at the rate found, straight into the caller's arrays
     e = launch_fb_final_trial(N, resolution_mrps, lo, active, iter_active, trial_lambda, st);
     if (e != cudaSuccess) return fail_cuda(e);
@@ -381,11 +373,6 @@ int themis_vertical_fallback_batch(const themis_problem_t *problem, const int32_
                     out, d_workspace, L.total_bytes, st);
     if (rc != THEMIS_OK) return rc;
     // 4. the rest of the load on extra replicas
-    Params P;
-    rc = make_params(problem, SolveOpts{kVertical}, d_workspace, L.total_bytes, &P);
-    if (rc != THEMIS_OK) return rc;
-    P.lat_us = d_lat_us; P.profile_id = d_profile_id; P.lambda_mrps = d_lambda_mrps; P.replicas = d_replicas;
-    P.out = out;
     e = launch_fb_finish(P, resolution_mrps, lo, hi, active, d_lambda_vertical, d_extra_replicas, st);
     return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
 }

@@ -89,10 +89,8 @@ inline size_t pruned_smem_bytes(int pitch) { return sizeof(uint32_t) * (5u * (si
 cudaError_t launch_configs_equal(int N, int S, themis_result_t a, themis_result_t b, int32_t *stable, cudaStream_t st);
 cudaError_t launch_fb_init(int N, uint32_t res, const int32_t *status, const uint32_t *lambda, uint32_t *lo,
                            uint32_t *hi, int32_t *active, cudaStream_t st);
-cudaError_t launch_fb_trial(int N, uint32_t res, const uint32_t *lo, const uint32_t *hi, const int32_t *active,
-                            int32_t *iter_active, uint32_t *trial_lambda, cudaStream_t st);
-cudaError_t launch_fb_update(int N, uint32_t *lo, uint32_t *hi, const int32_t *iter_active,
-                             const int32_t *trial_status, cudaStream_t st);
+cudaError_t launch_fb_bisect(const Params &p, int rounds, uint32_t res, const int32_t *active, uint32_t *lo,
+                             uint32_t *hi, cudaStream_t st);
 cudaError_t launch_fb_final_trial(int N, uint32_t res, const uint32_t *lo, const int32_t *active,
                                   int32_t *iter_active, uint32_t *trial_lambda, cudaStream_t st);
 cudaError_t launch_fb_finish(const Params &p, uint32_t res, const uint32_t *lo, const uint32_t *hi,
