@@ -204,6 +204,10 @@ score_kernel(const Params p)
                     // sustain lambda (feasibility is monotone in h) are the pair's one candidate.
                     if (live) {
                         int lo = 0, cnt = HN;
+                        if (HN == 1) {                       // vertical variant: the one replica count
+                            lo = smem[lmax_row] < l_us ? 1 : 0;
+                            cnt = 0;
+                        }
                         while (cnt > 0) {
                             const int half = cnt >> 1;
                             if (smem[lmax_row + lo + half] < l_us) { lo += half + 1; cnt -= half + 1; }
