@@ -280,10 +280,9 @@ def run_ours(args):
         dist.barrier()
     from paper_2407_14843_b200 import solver
 
-    solver.themis_set_minplus_mode(args.minplus_mode)
-    solver.themis_set_minplus_tile(args.minplus_tile)
     packed = args.minplus_mode == 0
-    prob = solver.Problem.of_workload(wl)
+    prob = solver.Problem.of_workload(wl, solver.KERNEL_PACKED16 if packed else solver.KERNEL_WIDE32, args.minplus_tile)
+    prob_sparse = solver.Problem.of_workload(wl, solver.KERNEL_SPARSE)
     dev = solver.workload_to_device(wl)
     ws = solver.alloc_workspace(prob, wl.vertical, host_variant=True)
     out = solver.alloc_result(wl.n_instances, wl.n_stages)
@@ -338,14 +337,13 @@ def run_ours(args):
     pruned = None
     if args.pruned_steps > 0:
         dense_out = {k: v.clone() for k, v in out.items()}
-        solver.themis_set_minplus_mode(3)
 
         def sparse_step():
             if wl.vertical:
-                solver.themis_solve_vertical_batch(prob, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"],
+                solver.themis_solve_vertical_batch(prob_sparse, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"],
                                                    dev["replicas"], out, ws)
             else:
-                solver.themis_solve_batch(prob, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"], out, ws)
+                solver.themis_solve_batch(prob_sparse, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"], out, ws)
 
         sparse_step()
         barrier()
@@ -355,17 +353,16 @@ def run_ours(args):
             sparse_step()
             pe[k + 1].record()
         barrier()
-        solver.themis_set_minplus_mode(args.minplus_mode)
         tp = torch.tensor([pe[0].elapsed_time(pe[-1])], dtype=torch.float64, device="cuda")
         if use_dist:
             dist.all_reduce(tp, op=dist.ReduceOp.MAX)
         p_total = float(tp.item())
         pruned = {"value": wl.n_instances * world * args.pruned_steps / (p_total * 1e-3), "unit": UNIT,
                   "ms_per_step": p_total / args.pruned_steps, "steps": args.pruned_steps,
-                  "kernel": "solve_sparse_kernel (1 launch per step)",
+                  "kernel": "solve_front_kernel + solve_sparse_kernel for listed instances (memset + 2 launches per step)",
                   "same_results_as_dense": all(bool((out[k] == dense_out[k]).all()) for k in out),
-                  "note": "themis_set_minplus_mode(3): scoring, fronts and recurrence on undominated "
-                          "entries in one kernel"}
+                  "note": "THEMIS_KERNEL_SPARSE: scoring, fronts and recurrence on undominated "
+                          "entries in one kernel, one warp per instance"}
 
     status = out["status"].cpu()
     n_infeasible = int((status == 1).sum())

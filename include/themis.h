@@ -54,9 +54,60 @@ extern "C" {
 #define THEMIS_MAX_CANDIDATES 65535 /* per stage (candidate index is uint16) */
 #define THEMIS_MAX_TOTAL_COST 131070 /* n_stages * h_max * c_max must not exceed it */
 
-/* themis_problem_t.flags */
+/* themis_problem_t.flags, bit 0: the queuing model */
 #define THEMIS_QUEUE_PER_REPLICA 1u /* q = (b-1) * h / lambda: every replica fills
                                        its own batch.  Clear: q = (b-1)/lambda, Eq. 4 */
+
+/* themis_problem_t.flags, bits 8..11: which kernels this call runs.  An implementation
+ * choice per call (the paper has no counterpart): returned configurations, costs,
+ * latencies and statuses never depend on it; what the rows of the workspace hold
+ * does (see themis_workspace_layout_t).  The choice travels with the call, so calls
+ * from different host threads on different streams may differ in it.
+ *   THEMIS_KERNEL_DEFAULT      same as THEMIS_KERNEL_PACKED16.
+ *   THEMIS_KERNEL_PACKED16     dense recurrence on packed 16-bit costs (two budget
+ *      cells per register), on costs relative to every stage's cheapest entry; the A
+ *      rows then hold the prefix tables themselves, uint16
+ *          F_s[t] - sum_{k<=s} min_l G_k[l]     (0x7FFF: unreachable or >= 32767),
+ *      and the backtrack recovers the argmin along the optimal path only.  Instances
+ *      whose optimum lies 32767 or more above the sum of the stages' cheapest entries
+ *      are redone by the 32-bit kernel in a second launch.
+ *   THEMIS_KERNEL_WIDE32       dense recurrence on 32-bit keys; the A rows hold the
+ *      argmin tables.
+ *   THEMIS_KERNEL_PRUNED       dense scoring, then the recurrence restricted to the
+ *      undominated entries of every G_s (an entry is dominated when a smaller l has
+ *      a cost at most as high; such entries never occur in the returned solution);
+ *      A and F are the tables of the restricted problem.  Budgets above about 11000
+ *      buckets run THEMIS_KERNEL_PACKED16 instead.
+ *   THEMIS_KERNEL_SPARSE       the solvers (themis_solve_*batch, host and static
+ *      variants, the fallback) run one kernel, one warp per instance, that scores only
+ *      the candidates that can matter (per cores and batch size the fewest replicas
+ *      that sustain lambda) and keeps only undominated stage entries and undominated
+ *      prefix states (budget, total) as short sorted lists; no dense table exists and
+ *      its cost does not grow with the budget length T.  The G rows of the workspace
+ *      then hold one backtrack record per prefix state.  Instances whose lists outgrow
+ *      the kernel's fixed capacities are redone by THEMIS_KERNEL_SPARSE_BLOCK's kernel
+ *      in a second launch.  The two-step entry points treat it as THEMIS_KERNEL_PRUNED.
+ *   THEMIS_KERNEL_SPARSE_BLOCK the same restriction with one thread block per instance
+ *      and dense shared-memory rows per budget cell (any list length); G, Garg and A
+ *      rows hold the stage fronts and the argmin of the front cells.  Falls back to
+ *      THEMIS_KERNEL_PRUNED when its shared memory (about 12 * row_pitch bytes plus
+ *      tables) does not fit. */
+#define THEMIS_KERNEL_DEFAULT      (0u << 8)
+#define THEMIS_KERNEL_PACKED16     (1u << 8)
+#define THEMIS_KERNEL_WIDE32       (2u << 8)
+#define THEMIS_KERNEL_PRUNED       (3u << 8)
+#define THEMIS_KERNEL_SPARSE       (4u << 8)
+#define THEMIS_KERNEL_SPARSE_BLOCK (5u << 8)
+#define THEMIS_KERNEL_MASK         (15u << 8)
+
+/* themis_problem_t.flags, bits 12..13: consecutive budget cells per thread of the
+ * dense recurrence kernels (a tuning knob, no counterpart in the paper; the 32-bit
+ * kernel treats 4 as its default).  Results do not depend on it. */
+#define THEMIS_TILE_DEFAULT (0u << 12)
+#define THEMIS_TILE_4       (1u << 12)
+#define THEMIS_TILE_8       (2u << 12)
+#define THEMIS_TILE_16      (3u << 12)
+#define THEMIS_TILE_MASK    (3u << 12)
 
 /* return codes */
 #define THEMIS_OK 0
@@ -89,7 +140,7 @@ typedef struct {
     int32_t h_max;         /* joint: replicas range over 1..h_max; vertical: ignored */
     int32_t slo_us;        /* SLO in microseconds */
     int32_t bucket_us;     /* bucket width w; T = slo_us / bucket_us, 1 <= T <= THEMIS_MAX_T */
-    uint32_t flags;        /* THEMIS_QUEUE_PER_REPLICA or 0 */
+    uint32_t flags;        /* THEMIS_QUEUE_PER_REPLICA | THEMIS_KERNEL_* | THEMIS_TILE_* */
 } themis_problem_t;
 
 /* Result arrays, caller-owned and caller-sized.  Device pointers for the d_
@@ -107,9 +158,10 @@ typedef struct {
  * start; rows are row_pitch entries long, entries beyond T are padding).
  *   G    int32  [N][S][row_pitch]  per-bucket minimum cost, THEMIS_G_INF if empty
  *   Garg uint16 [N][S][row_pitch]  lowest candidate index attaining G (0 if empty)
- *   A    uint16 [N][S][row_pitch]  mode 1: A[s][t] = lowest l attaining F_s[t] (row 0
- *                                  unused, 0 where F_s[t] is unreachable); mode 0: the
- *                                  prefix tables F_s[t] (see themis_set_minplus_mode)
+ *   A    uint16 [N][S][row_pitch]  THEMIS_KERNEL_WIDE32: A[s][t] = lowest l attaining
+ *                                  F_s[t] (row 0 unused, 0 where F_s[t] is unreachable);
+ *                                  THEMIS_KERNEL_PACKED16: the prefix tables F_s[t]
+ *                                  (see the THEMIS_KERNEL_* flags)
  *   F    int32  [N][row_pitch]     last prefix table F_{S-1}, THEMIS_G_INF if unreachable
  * Candidate index: idx = ((h-1)*c_max + (c-1))*n_batch + bi (joint),
  *                  idx = (c-1)*n_batch + bi (vertical). */
@@ -254,8 +306,9 @@ int themis_solve_batch_host(const themis_problem_t *problem, const int32_t *h_la
  * pool that hands out no scratch, a plug-in that is only given its input and
  * output buffers, a service that must not call cudaMalloc on its request path
  * because that call synchronises the device.  For them this entry point runs
- * the same two kernels as themis_solve_batch / themis_solve_vertical_batch
- * (d_replicas = NULL selects the joint problem) with the intermediate tables in
+ * the same kernels as themis_solve_batch / themis_solve_vertical_batch (whichever
+ * the problem's THEMIS_KERNEL_* flag selects; d_replicas = NULL selects the joint
+ * problem) with the intermediate tables in
  * a fixed buffer of THEMIS_STATIC_SCRATCH_BYTES that is part of the library
  * image: every GPU that loads the library holds that much memory until the
  * process exits.  It calls no allocation or free routine of any kind.
@@ -300,77 +353,6 @@ int themis_fit_profiles_batch(int32_t n_models, int32_t n_samples, const int32_t
                               const int32_t *d_sample_c, const double *d_latency_ms, int32_t c_max,
                               int32_t n_batch, const int32_t *d_batch_sizes, double *d_coeffs,
                               int32_t *d_lat_us, int32_t *d_status, void *cuda_stream);
-
-/*
- * Integer-ALU throughput probe (not part of the method, and the paper has no
- * counterpart): every thread keeps 16 independent chains in registers and runs
- * `iters` iterations of 4 rounds, each round one add-then-min update per chain (the
- * operation pair of the recurrence), every update reading two values produced one
- * round earlier.  Instruction form by mode:
- *   0: separate 32-bit add and unsigned min;
- *   1: fused 32-bit add-min (one instruction per update);
- *   2: two adds and one three-input min per two updates;
- *   3: fused add-min on packed 2 x 16-bit (two cell updates per instruction);
- *   4: single-precision add and min;
- *   5: the packed recurrence kernel's own inner step, operands loaded from shared
- *      memory as there but without stages, barriers or global traffic: every
- *      thread walks `iters` columns of 256 chunk steps of 8 x 8 cells (threads
- *      must be 256; 128 fused instructions per 4 steps as in mode 3).
- * Launches `blocks` x `threads` (32..1024) and writes one word per thread to d_sink
- * (blocks*threads uint32).  Updates performed = blocks * threads * iters * 64
- * (x 2 cells in mode 3; blocks * 256 * iters * 256 * 64 cells in mode 5).
- */
-int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_sink,
-                     void *cuda_stream);
-
-/*
- * Bounded-wait probe (not part of the method; the paper has no counterpart).  The
- * recurrence kernels stage every row G_s with an asynchronous bulk copy and wait for
- * it on a shared-memory barrier; that wait gives up after a fixed number of attempts
- * and the instance reports THEMIS_STATUS_TIMEOUT instead of hanging.  This entry point
- * runs the same wait routine in a one-warp kernel on two barriers: one whose 16-byte
- * copy from d_src16 (16-byte aligned) is issued (waited for with the kernels' own
- * limit), and one that expects 16 bytes which nothing delivers (waited for with
- * `max_polls` attempts, 1 .. 2^20).  Results:
- *   d_status[0] = THEMIS_STATUS_OK and d_dst16[0..3] = d_src16[0..3]  (the copy landed);
- *   d_status[1] = THEMIS_STATUS_TIMEOUT                               (the wait ran out);
- * the kernel returns normally in both cases and the context stays usable.
- * Returns THEMIS_E_INVALID_ARG for a NULL or misaligned pointer or max_polls out of range.
- */
-int themis_wait_probe(int32_t max_polls, const uint32_t *d_src16, uint32_t *d_dst16, int32_t *d_status,
-                      void *cuda_stream);
-
-/* Which min-plus kernel themis_minplus_batch and the solvers run (an implementation
- * choice; the paper has no counterpart).  Results do not depend on it; what the rows
- * of the workspace hold does.
- *   0 (default): packed 16-bit kernel (two budget cells per register).  It works
- *      on costs relative to every stage's cheapest entry, and the A rows then hold
- *      the prefix tables themselves, uint16
- *          F_s[t] - sum_{k<=s} min_l G_k[l]     (0x7FFF: unreachable or >= 32767),
- *      while the backtrack recovers the argmin along the optimal path only.
- *      Instances whose optimum lies 32767 or more above the sum of the stages'
- *      cheapest entries are redone by the 32-bit kernel in a second launch.
- *   1: 32-bit kernel only; the A rows hold the argmin tables described above.
- *   2: recurrence restricted to the undominated entries of every G_s (an entry is
- *      dominated when a smaller l has a cost at most as high; such entries never
- *      occur in the returned solution).  Returned configurations, costs, latencies
- *      and statuses are identical to modes 0 and 1 at a small fraction of the work;
- *      the A and F tables are those of the restricted problem.  Budgets above about
- *      11000 buckets run mode 0 instead.
- *   3: the solvers (themis_solve_*batch, host and static variants, the fallback) run
- *      ONE kernel that scores only the candidates that can matter (per cores and
- *      batch size the fewest replicas that sustain lambda), keeps only undominated
- *      stage entries and undominated prefix states (budget, total), and never writes
- *      a dense table: the G, Garg and A rows of the workspace then hold the stage
- *      fronts and the argmin of the front cells only.  Same results again.  The
- *      two-step entry points behave as in mode 2.  Falls back to mode 2 when its
- *      shared memory (about 12 * row_pitch bytes plus tables) does not fit. */
-int themis_set_minplus_mode(int mode);
-
-/* Tuning knob of the dense min-plus kernels (no counterpart in the paper): consecutive budget cells per thread
- * (4, 8 or 16; the 32-bit kernel treats 4 as its default); 0 restores the built-in
- * choice.  Results do not depend on it. */
-int themis_set_minplus_tile(int cells_per_thread);
 
 /* Library housekeeping (no counterpart in the paper).  Text for a return code; for THEMIS_E_CUDA includes the last CUDA error seen by
  * the calling thread.  The pointer stays valid until the thread's next call. */

@@ -174,12 +174,13 @@ def _per_instance(fn, wl, n: int) -> dict:
 
 
 def alg1_scatter(wl, n: int) -> dict:
-    """Instance ``n`` solved by Algorithm 1 in the paper's own loop order."""
+    """Instance ``n`` solved by forward relaxation over reachable (stage, budget) states in
+    Algorithm 1's visiting order (no per-bucket minimum, no (min,+) combine)."""
     return _per_instance(_load().oracle_alg1_scatter, wl, n)
 
 
 def alg2_scatter(wl, n: int) -> dict:
-    """Instance ``n`` solved by Algorithm 2 in the paper's own loop order (c_max = 1)."""
+    """Instance ``n`` of Algorithm 2's problem (c_max = 1) solved by the same forward relaxation."""
     return _per_instance(_load().oracle_alg2_scatter, wl, n)
 
 

@@ -24,14 +24,15 @@
  *   oracle_solve_batch      the stage-by-stage dynamic program of Algorithm 1,
  *                           with the candidate minimum hoisted out of the
  *                           budget loop (G_s) and a min-plus combine (F_s);
- *   oracle_alg1_scatter     Algorithm 1 in the paper's own loop order
- *                           (stage, budget descending, cores, batch), scattering
- *                           into best[s][i + l];
+ *   oracle_alg1_scatter     the same optimum by forward relaxation over reachable
+ *                           (stage, budget) states, extended option by option in
+ *                           Algorithm 1's visiting order, with no per-bucket
+ *                           minimum and no (min,+) combine;
  *   brute_force.c           Eq. 6 by exhaustive enumeration (separate file);
  * and, for the horizontal-only solver of Algorithm 2 (one-core replicas, replica
  * count computed as ceil(lambda / thr) per batch size):
  *   oracle_solve_horizontal_batch   the same program over batch sizes only;
- *   oracle_alg2_scatter             Algorithm 2 in the paper's loop order.
+ *   oracle_alg2_scatter             Algorithm 2's problem by the same forward relaxation.
  *
  * Readings of the paper taken here (each is pinned by a test):
  *   - a candidate is skipped iff its replicas cannot sustain lambda or it does
@@ -423,137 +424,148 @@ int oracle_vertical_fallback_batch(const oracle_problem *p, const int32_t *lat_u
 }
 
 /*
- * Algorithm 2 in the paper's loop order, one instance: as oracle_alg1_scatter, with
- * the candidate loop over batch sizes only and the replica count computed per
- * candidate.  lat_pipeline is [S][1][n_batch].
+ * Cross-check of the hoisted solver: the same optimum by forward relaxation over
+ * reachable states, without per-bucket minima and without a (min,+) combine.
+ *
+ * A state is "the first s+1 stages take exactly t buckets"; it remembers the
+ * cheapest total found so far, the state of the previous stage it was reached
+ * from and the option that led there.  The options of a stage (feasible
+ * candidates with their latency, cost and index) are listed once, in index
+ * order; then every reachable state of the previous stage, the one with the
+ * largest budget first, is extended by every option that still fits, and a
+ * state is replaced only by a strictly cheaper total.  Visiting order and the
+ * strict comparison are what Algorithm 1 / Algorithm 2 do (budget loop downwards,
+ * candidate loops upwards, '<'), so ties resolve as there: for a given state the
+ * extension with the shortest stage latency, and among those the lowest option
+ * index, is kept.  The final choice is the cheapest state of the last stage, the
+ * smallest budget among equals.
  */
+typedef struct { int32_t ell, cost, idx, h; } relax_option;
+typedef struct { int32_t total, from, option; } relax_state;    /* total < 0: not reached */
+
+static int relax_pipeline(int32_t S, int32_t T, relax_option *const *options, const int32_t *n_options,
+                          int32_t *opt_of_stage /* [S] out: chosen option per stage */,
+                          int32_t *cost_out, int32_t *lat_out)
+{
+    const int32_t W = T + 1;
+    relax_state *st = (relax_state *)malloc(sizeof(relax_state) * (size_t)S * W);
+    if (!st) return -1;
+    for (size_t k = 0; k < (size_t)S * W; ++k) st[k].total = -1;
+    for (int32_t s = 0; s < S; ++s) {
+        relax_state *here = st + (size_t)s * W;
+        const relax_state *before = s ? st + (size_t)(s - 1) * W : NULL;
+        for (int32_t spent = s ? T : 0; spent >= 0; --spent) {
+            int32_t base_total = 0;
+            if (before) {
+                if (before[spent].total < 0) continue;
+                base_total = before[spent].total;
+            }
+            for (int32_t o = 0; o < n_options[s]; ++o) {
+                const relax_option *opt = &options[s][o];
+                if ((int64_t)spent + opt->ell > T) continue;
+                relax_state *dst = &here[spent + opt->ell];
+                int32_t total = base_total + opt->cost;
+                if (dst->total < 0 || total < dst->total) {
+                    dst->total = total; dst->from = spent; dst->option = o;
+                }
+            }
+        }
+    }
+    int32_t end = -1;
+    const relax_state *last = st + (size_t)(S - 1) * W;
+    for (int32_t t = 0; t <= T; ++t)
+        if (last[t].total >= 0 && (end < 0 || last[t].total < last[end].total)) end = t;
+    int rc = 1;
+    *cost_out = -1; *lat_out = -1;
+    if (end >= 0) {
+        *cost_out = last[end].total; *lat_out = end;
+        int32_t t = end;
+        for (int32_t s = S - 1; s >= 0; --s) {
+            const relax_state *x = &st[(size_t)s * W + t];
+            opt_of_stage[s] = x->option;
+            t = x->from;
+        }
+        rc = 0;
+    }
+    free(st);
+    return rc;
+}
+
+/* Runs relax_pipeline on the options produced by fill(stage, list) and decodes the result. */
+static int relax_and_decode(const oracle_problem *p, const int32_t *lat_pipeline, uint32_t lambda_m,
+                            const int32_t *replicas, int horizontal, int32_t *h_out, int32_t *c_out,
+                            int32_t *b_out, int32_t *cost_out, int32_t *lat_out)
+{
+    const int32_t S = p->n_stages, T = p->slo_us / p->bucket_us;
+    const int32_t per_stage_max = horizontal ? p->n_batch : (replicas ? 1 : p->h_max) * p->c_max * p->n_batch;
+    relax_option **options = (relax_option **)calloc((size_t)S, sizeof(relax_option *));
+    int32_t *n_options = (int32_t *)calloc((size_t)S, sizeof(int32_t));
+    int32_t *chosen = (int32_t *)calloc((size_t)S, sizeof(int32_t));
+    int rc = -1;
+    if (!options || !n_options || !chosen) goto done;
+    for (int32_t s = 0; s < S; ++s) {
+        options[s] = (relax_option *)malloc(sizeof(relax_option) * (size_t)per_stage_max);
+        if (!options[s]) goto done;
+        relax_option *list = options[s];
+        int32_t n = 0;
+        if (horizontal) {
+            const int32_t *lat_stage = lat_pipeline + (size_t)s * p->n_batch;
+            for (int32_t bi = 0; bi < p->n_batch; ++bi) {
+                int64_t ell; int32_t h;
+                if (!horizontal_candidate(p, lat_stage[bi], p->batch_sizes[bi], lambda_m, &ell, &h)) continue;
+                if (ell > T) continue;
+                list[n].ell = (int32_t)ell; list[n].cost = h; list[n].idx = bi; list[n].h = h;
+                ++n;
+            }
+        } else {
+            const int32_t *lat_stage = lat_pipeline + (size_t)s * p->c_max * p->n_batch;
+            const int32_t h_first = replicas ? replicas[s] : 1, h_last = replicas ? replicas[s] : p->h_max;
+            int32_t idx = 0;
+            for (int32_t h = h_first; h <= h_last; ++h)
+                for (int32_t c = 1; c <= p->c_max; ++c)
+                    for (int32_t bi = 0; bi < p->n_batch; ++bi, ++idx) {
+                        int64_t ell; int32_t cost;
+                        if (!score_candidate(lat_stage[(c - 1) * p->n_batch + bi], h, c, p->batch_sizes[bi],
+                                             lambda_m, p->bucket_us, p->flags, &ell, &cost))
+                            continue;
+                        if (ell > T) continue;
+                        list[n].ell = (int32_t)ell; list[n].cost = cost; list[n].idx = idx; list[n].h = h;
+                        ++n;
+                    }
+        }
+        n_options[s] = n;
+    }
+    rc = relax_pipeline(S, T, options, n_options, chosen, cost_out, lat_out);
+    if (rc >= 0) {
+        for (int32_t s = 0; s < S; ++s) {
+            if (rc != 0) { h_out[s] = 0; c_out[s] = 0; b_out[s] = 0; continue; }
+            const relax_option *opt = &options[s][chosen[s]];
+            if (horizontal) { h_out[s] = opt->h; c_out[s] = 1; b_out[s] = p->batch_sizes[opt->idx]; }
+            else decode_idx(p, opt->idx, replicas ? replicas[s] : 0, &h_out[s], &c_out[s], &b_out[s]);
+        }
+    }
+done:
+    if (options) for (int32_t s = 0; s < S; ++s) free(options[s]);
+    free(options); free(n_options); free(chosen);
+    return rc;
+}
+
+/* Algorithm 2's problem (one-core replicas, replica count computed per batch size) by
+ * forward relaxation; lat_pipeline is [S][1][n_batch].  Returns 0 (solved) or 1 (infeasible). */
 int oracle_alg2_scatter(const oracle_problem *p, const int32_t *lat_pipeline, uint32_t lambda_m,
                         const int32_t *unused, int32_t *h_out, int32_t *c_out, int32_t *b_out,
                         int32_t *cost_out, int32_t *lat_out)
 {
     (void)unused;
-    const int32_t S = p->n_stages, T = p->slo_us / p->bucket_us, W = T + 1;
-    const size_t cells = (size_t)S * W;
-    uint8_t *dp = (uint8_t *)calloc(cells, 1);
-    int32_t *best_total = (int32_t *)malloc(sizeof(int32_t) * cells);
-    int32_t *best_ell = (int32_t *)malloc(sizeof(int32_t) * cells);
-    int32_t *best_ins = (int32_t *)malloc(sizeof(int32_t) * cells);
-    int32_t *best_bi = (int32_t *)malloc(sizeof(int32_t) * cells);
-    if (!dp || !best_total || !best_ell || !best_ins || !best_bi) {
-        free(dp); free(best_total); free(best_ell); free(best_ins); free(best_bi);
-        return -1;
-    }
-    for (int32_t s = 0; s < S; ++s) {
-        const int32_t *lat_stage = lat_pipeline + (size_t)s * p->n_batch;
-        for (int32_t i = T; i >= 0; --i) {
-            int reachable = (s == 0) ? (i == 0) : dp[(size_t)(s - 1) * W + i];
-            if (!reachable) continue;
-            for (int32_t bi = 0; bi < p->n_batch; ++bi) {
-                int64_t ell; int32_t ins;
-                if (!horizontal_candidate(p, lat_stage[bi], p->batch_sizes[bi], lambda_m, &ell, &ins)) continue;
-                if ((int64_t)i + ell > T) continue;
-                int32_t total = ins + (s == 0 ? 0 : best_total[(size_t)(s - 1) * W + i]);
-                size_t dst = (size_t)s * W + (size_t)(i + ell);
-                if (!dp[dst] || total < best_total[dst]) {
-                    dp[dst] = 1; best_total[dst] = total; best_ell[dst] = (int32_t)ell;
-                    best_ins[dst] = ins; best_bi[dst] = bi;
-                }
-            }
-        }
-    }
-    int32_t least = ORACLE_INF, ind = -1;
-    for (int32_t i = 0; i <= T; ++i) {
-        size_t k = (size_t)(S - 1) * W + i;
-        if (dp[k] && best_total[k] < least) { least = best_total[k]; ind = i; }
-    }
-    int rc = 1;
-    if (ind < 0) {
-        for (int32_t s = 0; s < S; ++s) { h_out[s] = 0; c_out[s] = 0; b_out[s] = 0; }
-        *cost_out = -1; *lat_out = -1;
-    } else {
-        int32_t t = ind;
-        for (int32_t s = S - 1; s >= 0; --s) {
-            size_t k = (size_t)s * W + t;
-            h_out[s] = best_ins[k]; c_out[s] = 1; b_out[s] = p->batch_sizes[best_bi[k]];
-            t -= best_ell[k];
-        }
-        *cost_out = least; *lat_out = ind;
-        rc = 0;
-    }
-    free(dp); free(best_total); free(best_ell); free(best_ins); free(best_bi);
-    return rc;
+    return relax_and_decode(p, lat_pipeline, lambda_m, NULL, 1, h_out, c_out, b_out, cost_out, lat_out);
 }
 
-/*
- * Algorithm 1 in the paper's loop order, one instance: for each stage, for the
- * budget already spent i from T down to 0, for each candidate (replicas,
- * cores, batch), extend the reachable state (s-1, i) to (s, i + l) when the
- * candidate sustains lambda and i + l <= T, keeping the cheaper total under a
- * strict '<'.  The first stage extends the empty prefix (i = 0 only).
- * best_* hold, per state, the running total, the stage latency used and the
- * candidate index, from which the configuration is read back recursively.
- * Returns 0 (solved) or 1 (infeasible); outputs as in oracle_solve_batch.
- */
+/* Algorithm 1's problem (replicas given) or the joint problem (replicas == NULL) by forward
+ * relaxation; lat_pipeline is [S][c_max][n_batch].  Returns 0 (solved) or 1 (infeasible);
+ * outputs as in oracle_solve_batch. */
 int oracle_alg1_scatter(const oracle_problem *p, const int32_t *lat_pipeline, uint32_t lambda_m,
                         const int32_t *replicas, int32_t *h_out, int32_t *c_out, int32_t *b_out,
                         int32_t *cost_out, int32_t *lat_out)
 {
-    const int32_t S = p->n_stages, T = p->slo_us / p->bucket_us, W = T + 1;
-    const size_t cells = (size_t)S * W;
-    uint8_t *dp = (uint8_t *)calloc(cells, 1);
-    int32_t *best_total = (int32_t *)malloc(sizeof(int32_t) * cells);
-    int32_t *best_ell = (int32_t *)malloc(sizeof(int32_t) * cells);
-    int32_t *best_idx = (int32_t *)malloc(sizeof(int32_t) * cells);
-    if (!dp || !best_total || !best_ell || !best_idx) {
-        free(dp); free(best_total); free(best_ell); free(best_idx);
-        return -1;
-    }
-    for (int32_t s = 0; s < S; ++s) {
-        const int32_t *lat_stage = lat_pipeline + (size_t)s * p->c_max * p->n_batch;
-        int32_t h_lo = replicas ? replicas[s] : 1, h_hi = replicas ? replicas[s] : p->h_max;
-        for (int32_t i = T; i >= 0; --i) {
-            int reachable = (s == 0) ? (i == 0) : dp[(size_t)(s - 1) * W + i];
-            if (!reachable) continue;
-            int32_t idx = 0;
-            for (int32_t h = h_lo; h <= h_hi; ++h)
-                for (int32_t c = 1; c <= p->c_max; ++c)
-                    for (int32_t bi = 0; bi < p->n_batch; ++bi, ++idx) {
-                        int64_t ell; int32_t cost;
-                        if (!score_candidate(lat_stage[(c - 1) * p->n_batch + bi], h, c,
-                                             p->batch_sizes[bi], lambda_m, p->bucket_us, p->flags,
-                                             &ell, &cost))
-                            continue;
-                        if ((int64_t)i + ell > T) continue;
-                        int32_t total = cost + (s == 0 ? 0 : best_total[(size_t)(s - 1) * W + i]);
-                        size_t dst = (size_t)s * W + (size_t)(i + ell);
-                        if (!dp[dst] || total < best_total[dst]) {
-                            dp[dst] = 1;
-                            best_total[dst] = total;
-                            best_ell[dst] = (int32_t)ell;
-                            best_idx[dst] = idx;
-                        }
-                    }
-        }
-    }
-    int32_t least = ORACLE_INF, ind = -1;
-    for (int32_t i = 0; i <= T; ++i) {
-        size_t k = (size_t)(S - 1) * W + i;
-        if (dp[k] && best_total[k] < least) { least = best_total[k]; ind = i; }
-    }
-    int rc = 1;
-    if (ind < 0) {
-        for (int32_t s = 0; s < S; ++s) { h_out[s] = 0; c_out[s] = 0; b_out[s] = 0; }
-        *cost_out = -1; *lat_out = -1;
-    } else {
-        int32_t t = ind;
-        for (int32_t s = S - 1; s >= 0; --s) {
-            size_t k = (size_t)s * W + t;
-            decode_idx(p, best_idx[k], replicas ? replicas[s] : 0, &h_out[s], &c_out[s], &b_out[s]);
-            t -= best_ell[k];
-        }
-        *cost_out = least; *lat_out = ind;
-        rc = 0;
-    }
-    free(dp); free(best_total); free(best_ell); free(best_idx);
-    return rc;
+    return relax_and_decode(p, lat_pipeline, lambda_m, replicas, 0, h_out, c_out, b_out, cost_out, lat_out);
 }

@@ -5,22 +5,35 @@
 #include <mutex>
 
 #include "themis_internal.h"
+#include "themis_probe.h"
 
 namespace themis {
 namespace {
 
 thread_local cudaError_t t_last_cuda = cudaSuccess;
 thread_local char t_msg[256];
-int g_tile = 0;   // min-plus cells per thread; 0 = built-in choice
 // Which problem a launch solves and for which instances.
 enum Mode { kJoint = 0, kVertical = 1, kHorizontal = 2 };
 struct SolveOpts {
     Mode mode = kJoint;
     const int32_t *active = nullptr;   // [N] device mask, or nullptr: every instance
 };
-int g_mode = 0;   // 0: packed 16-bit dense kernel with 32-bit second pass; 1: 32-bit dense kernel;
-                  // 2: recurrence over undominated entries only (dense packed kernel above 11000 buckets);
-                  // 3: scoring and recurrence on undominated entries in one kernel
+
+// Kernel choice and tile of a call, from the flags of its problem description.
+inline uint32_t kernel_of(const themis_problem_t *pr)
+{
+    const uint32_t k = pr->flags & THEMIS_KERNEL_MASK;
+    return k == THEMIS_KERNEL_DEFAULT ? THEMIS_KERNEL_PACKED16 : k;
+}
+inline int tile_of(const themis_problem_t *pr)
+{
+    switch (pr->flags & THEMIS_TILE_MASK) {
+        case THEMIS_TILE_4: return 4;
+        case THEMIS_TILE_8: return 8;
+        case THEMIS_TILE_16: return 16;
+        default: return 0;
+    }
+}
 
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
@@ -38,7 +51,8 @@ int validate(const themis_problem_t *pr, int vertical, int32_t *T_out, int32_t *
     if (pr->n_instances < 1 || pr->n_stages < 1 || pr->n_profiles < 1 || pr->c_max < 1 || pr->n_batch < 1)
         return THEMIS_E_INVALID_ARG;
     if (pr->slo_us < 1 || pr->bucket_us < 1) return THEMIS_E_INVALID_ARG;
-    if (pr->flags & ~THEMIS_QUEUE_PER_REPLICA) return THEMIS_E_INVALID_ARG;
+    if (pr->flags & ~(THEMIS_QUEUE_PER_REPLICA | THEMIS_KERNEL_MASK | THEMIS_TILE_MASK)) return THEMIS_E_INVALID_ARG;
+    if ((pr->flags & THEMIS_KERNEL_MASK) > THEMIS_KERNEL_SPARSE_BLOCK) return THEMIS_E_INVALID_ARG;
     if (!vertical && pr->h_max < 1) return THEMIS_E_INVALID_ARG;
     if (pr->n_batch > THEMIS_MAX_BATCH_SIZES) return THEMIS_E_UNSUPPORTED_SIZE;
     for (int i = 0; i < pr->n_batch; ++i) {
@@ -77,6 +91,8 @@ int layout_of(const themis_problem_t *pr, int vertical, themis_workspace_layout_
     L->a_offset = off;    off = align_up(off + rows * pitch * sizeof(uint16_t));
     L->f_offset = off;    off = align_up(off + (size_t)pr->n_instances * pitch * sizeof(int32_t));
     L->flag_offset = off; off = align_up(off + (size_t)pr->n_instances * sizeof(int32_t));
+    // behind the tables: instances the sparse warp kernel hands to the block kernel (count, then ids)
+    off = align_up(off + ((size_t)pr->n_instances + 1) * sizeof(int32_t));
     L->total_bytes = off;
     L->row_pitch = (int32_t)pitch;
     L->T = T;
@@ -104,6 +120,8 @@ int make_params(const themis_problem_t *pr, const SolveOpts &opts, void *ws, siz
     P->A = reinterpret_cast<uint16_t *>(base + L.a_offset);
     P->F = reinterpret_cast<int32_t *>(base + L.f_offset);
     P->inst_flag = reinterpret_cast<int32_t *>(base + L.flag_offset);
+    P->redo_count = reinterpret_cast<int32_t *>(base + align_up(L.flag_offset + (size_t)pr->n_instances * sizeof(int32_t)));
+    P->redo_list = P->redo_count + 1;
     return THEMIS_OK;
 }
 
@@ -135,19 +153,21 @@ int minplus_impl(const themis_problem_t *pr, const int32_t *rep, const SolveOpts
     if (!result_ok(out) || (vertical && !rep)) return THEMIS_E_INVALID_ARG;
     P.replicas = rep; P.out = out;
     cudaError_t e;
-    if (g_mode == 1) {
-        e = launch_minplus(P, g_tile, st);
-    } else if (g_mode >= 2 && pruned_smem_bytes(P.pitch) <= kMaxDynamicSmem) {
+    const uint32_t kernel = kernel_of(pr);
+    const int tile = tile_of(pr);
+    if (kernel == THEMIS_KERNEL_WIDE32) {
+        e = launch_minplus(P, tile, st);
+    } else if (kernel >= THEMIS_KERNEL_PRUNED && pruned_smem_bytes(P.pitch) <= kMaxDynamicSmem) {
         e = launch_minplus_pruned(P, st);
     } else {
-        e = launch_minplus16(P, g_tile, st);
+        e = launch_minplus16(P, tile, st);
         // A total can only reach the 16-bit saturation value if the static bound allows it
         // (vertical: the bound depends on replicas[], which lives on the device).
         const bool may_saturate =
             vertical || (int64_t)pr->n_stages * pr->h_max * pr->c_max >= (int64_t)kInf16;
         if (e == cudaSuccess && may_saturate) {
             P.only_flagged = 1;
-            e = launch_minplus(P, g_tile, st);
+            e = launch_minplus(P, tile, st);
         }
     }
     return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
@@ -162,14 +182,25 @@ int solve_impl(const themis_problem_t *pr, const int32_t *lat, const int32_t *pi
     int rc = validate(pr, vertical, &T, &K);
     if (rc != THEMIS_OK) return rc;
     if (!result_ok(out)) return THEMIS_E_INVALID_ARG;
-    if (g_mode == 3) {          // one kernel on undominated entries, when its shared memory fits
+    const uint32_t kernel = kernel_of(pr);
+    if (kernel == THEMIS_KERNEL_SPARSE || kernel == THEMIS_KERNEL_SPARSE_BLOCK) {
+        // one kernel on undominated entries, when its shared memory fits
         Params P;
         rc = make_params(pr, opts, ws, ws_bytes, &P);
         if (rc != THEMIS_OK) return rc;
         if (!lat || !lam || (vertical && !rep)) return THEMIS_E_INVALID_ARG;
         P.lat_us = lat; P.profile_id = pid; P.lambda_mrps = lam; P.replicas = rep; P.out = out;
-        if (sparse_smem_bytes(P) <= kMaxDynamicSmem) {
-            cudaError_t e = launch_solve_sparse(P, st);
+        const bool block_fits = sparse_smem_bytes(P) <= kMaxDynamicSmem;
+        if (kernel == THEMIS_KERNEL_SPARSE && block_fits && front_kernel_fits(P)) {
+            // one warp per instance on short sorted lists; what outgrows them is listed and
+            // redone by the block kernel
+            cudaError_t e = cudaMemsetAsync(P.redo_count, 0, sizeof(int32_t), st);
+            if (e == cudaSuccess) e = launch_solve_front(P, st);
+            if (e == cudaSuccess) e = launch_solve_sparse(P, /*only_listed=*/true, st);
+            return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
+        }
+        if (block_fits) {
+            cudaError_t e = launch_solve_sparse(P, /*only_listed=*/false, st);
             return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
         }
     }
@@ -526,21 +557,6 @@ int themis_wait_probe(int32_t max_polls, const uint32_t *d_src16, uint32_t *d_ds
     cudaError_t e = launch_wait_probe((uint32_t)max_polls, d_src16, d_dst16, d_status,
                                       static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
-}
-
-int themis_set_minplus_mode(int mode)
-{
-    if (mode < 0 || mode > 3) return THEMIS_E_INVALID_ARG;
-    g_mode = mode;
-    return THEMIS_OK;
-}
-
-int themis_set_minplus_tile(int cells_per_thread)
-{
-    if (cells_per_thread != 0 && cells_per_thread != 4 && cells_per_thread != 8 && cells_per_thread != 16)
-        return THEMIS_E_INVALID_ARG;
-    g_tile = cells_per_thread;
-    return THEMIS_OK;
 }
 
 }  // extern "C"

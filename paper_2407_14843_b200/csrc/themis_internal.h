@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "themis.h"
 
 namespace themis {
@@ -54,7 +56,9 @@ struct Params {
     uint16_t *Garg;
     uint16_t *A;
     int32_t *F;
-    int32_t *inst_flag;  // [N] nonzero = bad input seen by the scoring kernel
+    int32_t *redo_count; // sparse warp kernel: number of instances handed to the block kernel ...
+    int32_t *redo_list;  // ... and their indices [N]
+    int32_t *inst_flag;  // [N] kFlagBadInput: bad input seen by the scoring kernel; kFlagNeedsWide: see above
     themis_result_t out;
 };
 
@@ -76,14 +80,35 @@ inline void assign_warp_groups(int n_warps, uint8_t *warp_group)
     }
 }
 
+constexpr size_t kMaxDynamicSmem = 226u * 1024u;   // 227 KB per block less room for static variables
+
+// Raises a kernel's dynamic shared-memory limit to kMaxDynamicSmem, once per device and
+// kernel (`done` has one bit per device ordinal and belongs to the launch site), so that a
+// launch costs no attribute call.
+inline cudaError_t allow_max_smem(const void *kernel, std::atomic<uint64_t> &done)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const uint64_t bit = 1ull << (dev & 63);
+    if (done.load(std::memory_order_acquire) & bit) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynamicSmem);
+    if (e == cudaSuccess) done.fetch_or(bit, std::memory_order_release);
+    return e;
+}
+
 cudaError_t launch_score(const Params &p, cudaStream_t stream);
 cudaError_t launch_minplus(const Params &p, int tile, cudaStream_t stream);
 cudaError_t launch_minplus16(const Params &p, int tile, cudaStream_t stream);
 cudaError_t launch_minplus_pruned(const Params &p, cudaStream_t stream);
-// Scoring and recurrence on undominated entries in one kernel (needs lat_us, lambda, out set).
+// Scoring and recurrence on undominated entries in one kernel (needs lat_us, lambda, out set),
+// one block per instance; only_listed: a fixed grid works through redo_list instead.
 size_t sparse_smem_bytes(const Params &p);
-cudaError_t launch_solve_sparse(const Params &p, cudaStream_t stream);
-constexpr size_t kMaxDynamicSmem = 227u * 1024u;
+cudaError_t launch_solve_sparse(const Params &p, bool only_listed, cudaStream_t stream);
+// The same on short sorted lists, one warp per instance; instances that outgrow the lists are
+// appended to redo_list (redo_count must be zero before the launch).
+bool front_kernel_fits(const Params &p);
+cudaError_t launch_solve_front(const Params &p, cudaStream_t stream);
 // Dynamic shared memory of the pruned kernel for a row pitch; it cannot run above 227 KB.
 inline size_t pruned_smem_bytes(int pitch) { return sizeof(uint32_t) * (5u * (size_t)pitch + 4 + 32); }
 cudaError_t launch_configs_equal(int N, int S, themis_result_t a, themis_result_t b, int32_t *stable, cudaStream_t st);

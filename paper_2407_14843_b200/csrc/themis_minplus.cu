@@ -98,7 +98,7 @@ minplus_kernel(const Params p)
     };
     if (p.only_flagged) {                               // second pass: only what the packed kernel left over
         if (p.inst_flag[n] != kFlagNeedsWide) return;
-    } else if (p.inst_flag[n] != 0) {                   // bad input seen while scoring
+    } else if (p.inst_flag[n] == kFlagBadInput) {       // bad input seen while scoring
         if (tid == 0) write_unsolved(THEMIS_STATUS_BAD_INPUT);
         return;
     }
@@ -253,8 +253,8 @@ cudaError_t launch_variant(const Params &p_in, int threads, size_t smem, cudaStr
 {
     Params p = p_in;
     assign_warp_groups(threads / 32, p.warp_group);
-    cudaError_t e = cudaFuncSetAttribute(minplus_kernel<R, MAXT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+    static std::atomic<uint64_t> ready{0};
+    cudaError_t e = allow_max_smem(reinterpret_cast<const void *>(minplus_kernel<R, MAXT>), ready);
     if (e != cudaSuccess) return e;
     minplus_kernel<R, MAXT><<<p.prob.n_instances, threads, smem, stream>>>(p);
     return cudaGetLastError();

@@ -131,7 +131,8 @@ minplus16_kernel(const Params p)
         p.out.latency_buckets[n] = -1;
         p.out.status[n] = status;
     };
-    if (p.inst_flag[n] != 0) {                            // bad input seen while scoring
+    if (p.inst_flag[n] == kFlagBadInput) {                // bad input seen while scoring (a leftover
+                                                          // kFlagNeedsWide of an earlier pass is re-decided below)
         if (tid == 0) write_unsolved(THEMIS_STATUS_BAD_INPUT);
         return;
     }
@@ -549,7 +550,9 @@ cudaError_t launch_variant16x(const Params &p, int threads, size_t smem, cudaStr
 {
     auto kernel = (p.n_half_groups & 3) == 0 ? minplus16_kernel<R, MAXT, EXTRA, true>
                                              : minplus16_kernel<R, MAXT, EXTRA, false>;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static std::atomic<uint64_t> pairs_ready{0}, general_ready{0};
+    cudaError_t e = allow_max_smem(reinterpret_cast<const void *>(kernel),
+                                   (p.n_half_groups & 3) == 0 ? pairs_ready : general_ready);
     if (e != cudaSuccess) return e;
     kernel<<<p.prob.n_instances, threads, smem, stream>>>(p);
     return cudaGetLastError();

@@ -102,7 +102,7 @@ minplus_pruned_kernel(const Params p)
         p.out.latency_buckets[n] = -1;
         p.out.status[n] = status;
     };
-    if (p.inst_flag[n] != 0) {                 // bad input seen while scoring
+    if (p.inst_flag[n] == kFlagBadInput) {     // bad input seen while scoring
         if (tid == 0) write_unsolved(THEMIS_STATUS_BAD_INPUT);
         return;
     }
@@ -241,8 +241,8 @@ minplus_pruned_kernel(const Params p)
 cudaError_t launch_minplus_pruned(const Params &p, cudaStream_t stream)
 {
     const size_t smem = pruned_smem_bytes(p.pitch);
-    cudaError_t e = cudaFuncSetAttribute(minplus_pruned_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+    static std::atomic<uint64_t> ready{0};
+    cudaError_t e = allow_max_smem(reinterpret_cast<const void *>(minplus_pruned_kernel), ready);
     if (e != cudaSuccess) return e;
     minplus_pruned_kernel<<<p.prob.n_instances, kPrunedThreads, smem, stream>>>(p);
     return cudaGetLastError();

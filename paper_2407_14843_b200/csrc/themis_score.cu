@@ -292,10 +292,9 @@ cudaError_t launch_score(const Params &p, cudaStream_t stream)
     const int threads = p.pitch <= 1024 ? 128 : 256;
     const size_t smem = sizeof(uint32_t) * (2u * (size_t)p.pitch + 2u * table + 4u + (threads / 32) * kListWords + 32u);
     auto kernel = threads == 128 ? score_kernel<128> : score_kernel<256>;
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-    }
+    static std::atomic<uint64_t> ready128{0}, ready256{0};
+    cudaError_t e = allow_max_smem(reinterpret_cast<const void *>(kernel), threads == 128 ? ready128 : ready256);
+    if (e != cudaSuccess) return e;
     kernel<<<p.prob.n_instances, threads, smem, stream>>>(p);
     return cudaGetLastError();
 }

@@ -87,14 +87,11 @@ __device__ __forceinline__ int front_of_row(uint32_t *row, int n_entries, int se
     return (int)*s_total;
 }
 
-// kThreads: 128 for short budgets (fewer, cheaper barriers per stage), else 256.
+// One instance, solved by the whole block.
 template <int kThreads>
-__global__ void __launch_bounds__(kThreads)
-solve_sparse_kernel(const Params p)
+__device__ __forceinline__ void solve_instance_sparse(const Params &p, const int n, uint32_t *smem)
 {
     constexpr int kWarps = kThreads / 32;
-    extern __shared__ __align__(16) uint32_t smem[];
-    const int n = blockIdx.x;
     if (p.active && !p.active[n]) return;
     const int tid = threadIdx.x;
     const int T = p.T, pitch = p.pitch;
@@ -270,6 +267,25 @@ solve_sparse_kernel(const Params p)
     p.out.status[n] = THEMIS_STATUS_OK;
 }
 
+// kThreads: 128 for short budgets (fewer, cheaper barriers per stage), else 256.
+// LISTED: the grid works through the instances in redo_list (those the warp kernel handed
+// over) instead of taking one instance per block.
+template <int kThreads, bool LISTED>
+__global__ void __launch_bounds__(kThreads)
+solve_sparse_kernel(const Params p)
+{
+    extern __shared__ __align__(16) uint32_t smem[];
+    if (!LISTED) {
+        solve_instance_sparse<kThreads>(p, blockIdx.x, smem);
+        return;
+    }
+    const int count = min(*p.redo_count, p.prob.n_instances);
+    for (int i = blockIdx.x; i < count; i += gridDim.x) {
+        solve_instance_sparse<kThreads>(p, p.redo_list[i], smem);
+        __syncthreads();                 // the last reader of this instance's shared memory is done
+    }
+}
+
 }  // namespace
 
 size_t sparse_smem_bytes(const Params &p)
@@ -280,21 +296,26 @@ size_t sparse_smem_bytes(const Params &p)
     return sizeof(uint32_t) * (3u * (size_t)p.pitch + 2u * cap_g + 2u * table + 32u);
 }
 
-cudaError_t launch_solve_sparse(const Params &p, cudaStream_t stream)
+template <int kThreads, bool LISTED>
+cudaError_t launch_sparse_variant(const Params &p, size_t smem, cudaStream_t stream)
+{
+    static std::atomic<uint64_t> ready{0};
+    cudaError_t e = allow_max_smem(reinterpret_cast<const void *>(solve_sparse_kernel<kThreads, LISTED>), ready);
+    if (e != cudaSuccess) return e;
+    // listed: a fixed grid of a few blocks per SM; an empty list costs one short launch
+    const int blocks = LISTED ? min(p.prob.n_instances, 4 * 148) : p.prob.n_instances;
+    solve_sparse_kernel<kThreads, LISTED><<<blocks, kThreads, smem, stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_solve_sparse(const Params &p, bool only_listed, cudaStream_t stream)
 {
     const size_t smem = sparse_smem_bytes(p);
-    if (p.pitch <= 1024) {
-        cudaError_t e = cudaFuncSetAttribute(solve_sparse_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)smem);
-        if (e != cudaSuccess) return e;
-        solve_sparse_kernel<128><<<p.prob.n_instances, 128, smem, stream>>>(p);
-    } else {
-        cudaError_t e = cudaFuncSetAttribute(solve_sparse_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)smem);
-        if (e != cudaSuccess) return e;
-        solve_sparse_kernel<256><<<p.prob.n_instances, 256, smem, stream>>>(p);
-    }
-    return cudaGetLastError();
+    if (p.pitch <= 1024)
+        return only_listed ? launch_sparse_variant<128, true>(p, smem, stream)
+                           : launch_sparse_variant<128, false>(p, smem, stream);
+    return only_listed ? launch_sparse_variant<256, true>(p, smem, stream)
+                       : launch_sparse_variant<256, false>(p, smem, stream);
 }
 
 }  // namespace themis

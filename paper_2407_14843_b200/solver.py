@@ -19,6 +19,11 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libthemis.so")
 
 QUEUE_PER_REPLICA = 1
+# themis_problem_t.flags: kernel choice of a call (bits 8..11) and cells per thread (bits 12..13)
+KERNEL_DEFAULT, KERNEL_PACKED16, KERNEL_WIDE32, KERNEL_PRUNED, KERNEL_SPARSE, KERNEL_SPARSE_BLOCK = (
+    k << 8 for k in range(6))
+KERNEL_MASK = 15 << 8
+TILE_FLAGS = {0: 0 << 12, 4: 1 << 12, 8: 2 << 12, 16: 3 << 12}
 OK, E_INVALID_ARG, E_UNSUPPORTED_SIZE, E_WORKSPACE_TOO_SMALL, E_CUDA = 0, -1, -2, -3, -4
 E_STATIC_SCRATCH_EXCEEDED = -5
 STATIC_SCRATCH_BYTES = 32 << 20
@@ -31,11 +36,12 @@ INF16 = 0x7FFF
 EXPORTS = (
     "themis_version", "themis_strerror", "themis_workspace_bytes", "themis_workspace_layout",
     "themis_solve_batch", "themis_solve_vertical_batch", "themis_score_batch", "themis_minplus_batch",
-    "themis_host_workspace_bytes", "themis_solve_batch_host", "themis_alu_probe", "themis_wait_probe",
-    "themis_set_minplus_tile", "themis_solve_batch_static", "themis_set_minplus_mode",
+    "themis_host_workspace_bytes", "themis_solve_batch_host", "themis_solve_batch_static",
     "themis_solve_horizontal_batch", "themis_fallback_workspace_bytes", "themis_vertical_fallback_batch",
     "themis_fit_profiles_batch", "themis_configs_equal_batch",
 )
+# include/themis_probe.h: measurement probes, not part of the solver
+PROBE_EXPORTS = ("themis_alu_probe", "themis_wait_probe")
 
 
 class ThemisError(RuntimeError):
@@ -64,9 +70,10 @@ class Problem(ctypes.Structure):
         return p
 
     @classmethod
-    def of_workload(cls, wl) -> "Problem":
+    def of_workload(cls, wl, kernel: int = KERNEL_DEFAULT, tile: int = 0) -> "Problem":
+        """``kernel``: one of the ``KERNEL_*`` flag values; ``tile``: 0, 4, 8 or 16 cells per thread."""
         return cls.make(wl.n_instances, wl.n_stages, wl.n_profiles, wl.c_max, wl.batch_sizes,
-                        wl.h_max, wl.slo_us, wl.bucket_us, wl.flags)
+                        wl.h_max, wl.slo_us, wl.bucket_us, wl.flags | kernel | TILE_FLAGS[tile])
 
 
 class Result(ctypes.Structure):
@@ -111,9 +118,7 @@ def _load() -> ctypes.CDLL:
                                               ctypes.c_int32, vp, vp, vp, vp, vp]
     lib.themis_alu_probe.argtypes = [ctypes.c_int] * 4 + [vp, vp]
     lib.themis_wait_probe.argtypes = [ctypes.c_int32, vp, vp, vp, vp]
-    lib.themis_set_minplus_tile.argtypes = [ctypes.c_int]
-    lib.themis_set_minplus_mode.argtypes = [ctypes.c_int]
-    for name in EXPORTS:
+    for name in EXPORTS + PROBE_EXPORTS:
         if name != "themis_strerror":
             getattr(lib, name).restype = ctypes.c_int
     return lib
@@ -284,14 +289,6 @@ def themis_wait_probe(max_polls: int, src16, dst16, status) -> None:
                                   _dptr(status, torch.int32, "status"), _stream()), "themis_wait_probe")
 
 
-def themis_set_minplus_mode(mode: int) -> None:
-    _check(_lib.themis_set_minplus_mode(mode), "themis_set_minplus_mode")
-
-
-def themis_set_minplus_tile(cells_per_thread: int) -> None:
-    _check(_lib.themis_set_minplus_tile(cells_per_thread), "themis_set_minplus_tile")
-
-
 # --- plumbing helpers (allocation and copies only) ---------------------------
 
 def alloc_result(n_instances: int, n_stages: int, device="cuda", pin: bool = False) -> dict:
@@ -336,11 +333,12 @@ def workspace_tables(problem: Problem, vertical: bool, workspace: torch.Tensor) 
 
 
 def solve(wl, dev: Optional[dict] = None, workspace: Optional[torch.Tensor] = None,
-          out: Optional[dict] = None, horizontal: bool = False):
+          out: Optional[dict] = None, horizontal: bool = False, kernel: int = KERNEL_DEFAULT, tile: int = 0):
     """Solve a workload on the current device: allocates what is not given,
     then calls ``themis_solve_batch`` / ``themis_solve_vertical_batch`` (or
-    ``themis_solve_horizontal_batch`` when ``horizontal``)."""
-    problem = Problem.of_workload(wl)
+    ``themis_solve_horizontal_batch`` when ``horizontal``).  ``kernel`` and ``tile``
+    go into the problem's flags (``KERNEL_*``; 0, 4, 8 or 16 cells per thread)."""
+    problem = Problem.of_workload(wl, kernel, tile)
     dev = dev if dev is not None else workload_to_device(wl)
     workspace = workspace if workspace is not None else alloc_workspace(problem, wl.vertical)
     out = out if out is not None else alloc_result(wl.n_instances, wl.n_stages)

@@ -25,13 +25,18 @@ def _good(S, **kw):
     return S.Problem.make(**args)
 
 
-def test_every_declared_function_is_exported(S):
-    header = open(os.path.join(ROOT, "include", "themis.h")).read()
+def _declared(header_name):
+    header = open(os.path.join(ROOT, "include", header_name)).read()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = set(re.findall(r"\b(themis_[a-z0-9_]+)\s*\(", header))
-    assert declared == set(S.EXPORTS)
+    return set(re.findall(r"\b(themis_[a-z0-9_]+)\s*\(", header))
+
+
+def test_every_declared_function_is_exported(S):
+    """Both headers: the solver's (themis.h) and the measurement probes' (themis_probe.h)."""
+    assert _declared("themis.h") == set(S.EXPORTS)
+    assert _declared("themis_probe.h") == set(S.PROBE_EXPORTS)
     lib = ctypes.CDLL(S.LIB_PATH)
-    for name in declared:
+    for name in S.EXPORTS + S.PROBE_EXPORTS:
         assert hasattr(lib, name), name
     assert S.themis_version() == 100
 
@@ -102,9 +107,19 @@ def test_pointer_and_workspace_checks(S):
     assert lib.themis_wait_probe(0, one, one, one, None) == S.E_INVALID_ARG
     assert lib.themis_wait_probe(100, ctypes.c_void_p(260), one, one, None) == S.E_INVALID_ARG
     assert lib.themis_wait_probe(100, one, None, one, None) == S.E_INVALID_ARG
-    assert lib.themis_set_minplus_tile(12) == S.E_INVALID_ARG
-    assert lib.themis_set_minplus_tile(0) == S.OK
-    assert lib.themis_set_minplus_mode(4) == S.E_INVALID_ARG and lib.themis_set_minplus_mode(0) == S.OK
+
+
+def test_kernel_choice_is_part_of_the_problem_flags(S):
+    """Kernel and tile are bits of themis_problem_t.flags; unknown values are refused and the
+    choice does not change the workspace a problem needs."""
+    n = ctypes.c_size_t()
+    base = S.themis_workspace_bytes(_good(S), False)
+    for kernel in (S.KERNEL_DEFAULT, S.KERNEL_PACKED16, S.KERNEL_WIDE32, S.KERNEL_PRUNED, S.KERNEL_SPARSE,
+                   S.KERNEL_SPARSE_BLOCK):
+        for tile in (0, 4, 8, 16):
+            assert S.themis_workspace_bytes(_good(S, flags=1 | kernel | S.TILE_FLAGS[tile]), False) == base
+    for flags in (6 << 8, 15 << 8, 1 << 14, 2, 1 << 31):
+        assert S._lib.themis_workspace_bytes(ctypes.byref(_good(S, flags=flags)), 0, ctypes.byref(n)) == S.E_INVALID_ARG
 
 
 def test_strerror(S):
@@ -123,6 +138,7 @@ def test_header_is_plain_c_and_links_from_c(S, tmp_path):
 #include <stdio.h>
 #include <string.h>
 #include "themis.h"
+#include "themis_probe.h"
 int main(void) {
     themis_problem_t p;
     themis_workspace_layout_t lay;
@@ -130,7 +146,7 @@ int main(void) {
     memset(&p, 0, sizeof p);
     p.n_instances = 10; p.n_stages = 5; p.n_profiles = 1; p.c_max = 16; p.n_batch = 3;
     p.batch_sizes[0] = 1; p.batch_sizes[1] = 2; p.batch_sizes[2] = 4;
-    p.h_max = 8; p.slo_us = 1000000; p.bucket_us = 1000; p.flags = THEMIS_QUEUE_PER_REPLICA;
+    p.h_max = 8; p.slo_us = 1000000; p.bucket_us = 1000; p.flags = THEMIS_QUEUE_PER_REPLICA | THEMIS_KERNEL_SPARSE | THEMIS_TILE_8;
     if (themis_version() != THEMIS_VERSION) return 1;
     if (themis_workspace_bytes(&p, 0, &bytes) != THEMIS_OK || bytes == 0) return 2;
     if (themis_workspace_layout(&p, 0, &lay) != THEMIS_OK || lay.T != 1000 || lay.row_pitch != 1024) return 3;

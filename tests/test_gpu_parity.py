@@ -21,9 +21,13 @@ def S():
     return solver
 
 
-def _gpu_solve(S, wl, tables=False, horizontal=False):
+def _gpu_solve(S, wl, tables=False, horizontal=False, mode=None, tile=None):
+    """Solves through the C ABI with the kernel (0 packed16, 1 wide32, 2 pruned, 3 sparse,
+    4 sparse-block) and tile under test, both passed per call in the problem's flags."""
     import torch
-    out, ws = S.solve(wl, horizontal=horizontal)
+    mode = MODE["mode"] if mode is None else mode
+    tile = MODE["tile"] if tile is None else tile
+    out, ws = S.solve(wl, horizontal=horizontal, kernel=(mode + 1) << 8, tile=tile)
     torch.cuda.synchronize()
     res = {k: v.cpu().numpy() for k, v in out.items()}
     if tables:
@@ -59,15 +63,15 @@ def _assert_results_equal(gpu, ref, idx=None):
                                            + _diagnose(gpu, ref, idx))
 
 
-MODE = {"mode": 0}   # min-plus kernel under test: 0 packed 16-bit (default), 1 32-bit, 2 pruned
+# kernel under test: 0 packed 16-bit (the default), 1 32-bit, 2 pruned, 3 sparse (one warp per
+# instance, block kernel for what outgrows its lists), 4 sparse block kernel; tile: cells per thread
+MODE = {"mode": 0, "tile": 0}
 
 
-@pytest.fixture(params=[0, 1, 2, 3], ids=["packed16", "wide32", "pruned", "sparse"])
+@pytest.fixture(params=[0, 1, 2, 3, 4], ids=["packed16", "wide32", "pruned", "sparse", "sparse_block"])
 def mode(request, S):
-    S.themis_set_minplus_mode(request.param)
     MODE["mode"] = request.param
     yield request.param
-    S.themis_set_minplus_mode(0)
     MODE["mode"] = 0
 
 
@@ -75,7 +79,7 @@ def _assert_tables_equal(S, gpu, ref):
     """G, Garg everywhere; F (last prefix) where the instance is solved; then
     32-bit kernel: A where F_s[t] is reachable (0 elsewhere);
     packed kernel: every prefix table F_s[t], saturated at 0x7FFF."""
-    if MODE["mode"] == 3:      # one fused kernel: the workspace holds fronts, not the dense tables
+    if MODE["mode"] >= 3:      # one fused kernel: the workspace holds fronts, not the dense tables
         return
     assert np.array_equal(gpu["G"], ref["G"])
     assert np.array_equal(gpu["Garg"], ref["Garg"])
@@ -107,7 +111,7 @@ def _assert_tables_equal(S, gpu, ref):
 @pytest.mark.parametrize("tile", [4, 8, 16])
 def test_config1_every_table(S, oracle_mod, tile, mode):
     """Smallest benchmark configuration: every intermediate table and result."""
-    S.themis_set_minplus_tile(tile)
+    MODE["tile"] = tile
     try:
         wl = W.make_workload(1)
         ref = oracle_mod.solve_batch(wl, dumps=True)
@@ -115,7 +119,7 @@ def test_config1_every_table(S, oracle_mod, tile, mode):
         _assert_tables_equal(S, gpu, ref)
         _assert_results_equal(gpu, ref)
     finally:
-        S.themis_set_minplus_tile(0)
+        MODE["tile"] = 0
 
 
 @pytest.mark.parametrize("cfg,n", [(2, 96), (3, 160), (4, 12), (5, 3)])
@@ -125,7 +129,7 @@ def test_config_subsets_every_table(S, oracle_mod, cfg, n, tile, mode):
     never a multiple of the tile): every table and result."""
     if tile == 8 and cfg == 5:
         pytest.skip("8 cells per thread would need more than 1024 threads at T = 8192")
-    S.themis_set_minplus_tile(tile)
+    MODE["tile"] = tile
     try:
         wl = W.make_workload(cfg, n)
         if cfg == 3:   # seconds spread over the day so that spikes are included
@@ -138,7 +142,7 @@ def test_config_subsets_every_table(S, oracle_mod, cfg, n, tile, mode):
         _assert_tables_equal(S, gpu, ref)
         _assert_results_equal(gpu, ref)
     finally:
-        S.themis_set_minplus_tile(0)
+        MODE["tile"] = 0
 
 
 @pytest.mark.parametrize("flags", [0, W.QUEUE_PER_REPLICA])
@@ -217,7 +221,7 @@ def test_vertical_fallback(S, oracle_mod, res, mode):
     wl = _spiky_vertical_workload(40)
     ref = oracle_mod.vertical_fallback_batch(wl, res)
     assert (ref["status"] == 2).any() and (ref["status"] == 0).any()
-    prob = S.Problem.of_workload(wl)
+    prob = S.Problem.of_workload(wl, kernel=(mode + 1) << 8)
     dev = S.workload_to_device(wl)
     ws = torch.empty(S.themis_fallback_workspace_bytes(prob), dtype=torch.uint8, device="cuda")
     out = S.alloc_result(wl.n_instances, wl.n_stages)
@@ -392,28 +396,24 @@ def test_repeatable_and_tile_independent(S, mode):
     wl = W.make_workload(4, 24)
     runs = []
     for tile in (16, 16, 8, 4):
-        S.themis_set_minplus_tile(tile)
-        runs.append(_gpu_solve(S, wl, tables=True))
-    S.themis_set_minplus_tile(0)
+        runs.append(_gpu_solve(S, wl, tables=True, tile=tile))
     for r in runs[1:]:
         for k in RESULT_KEYS + ("G", "Garg", "A", "F"):
             assert np.array_equal(runs[0][k], r[k]), k
 
 
 def test_all_kernels_agree(S):
-    """Packed 16-bit, 32-bit, pruned and fused sparse kernels: the same results, word for word."""
+    """Packed 16-bit, 32-bit, pruned and the two sparse kernels: the same results, word for word."""
     for wl in (W.make_workload(3, 300), W.make_workload(4, 96), W.make_workload(2, 512)):
         runs = []
-        for m in (1, 0, 2, 3):
-            S.themis_set_minplus_mode(m)
-            runs.append(_gpu_solve(S, wl))
-        S.themis_set_minplus_mode(0)
+        for m in (1, 0, 2, 3, 4):
+            runs.append(_gpu_solve(S, wl, mode=m))
         for r in runs[1:]:
             for k in RESULT_KEYS:
                 assert np.array_equal(runs[0][k], r[k]), k
 
 
-def test_totals_beyond_16_bits_fall_back_to_the_wide_kernel(S, oracle_mod):
+def _beyond_16_bits_workload():
     """Vertical problem with thousands of replicas per stage.  The packed kernel holds, in 15
     bits, what an instance pays beyond the sum of its stages' cheapest entries.  One group of
     instances has totals of 36000 and more but pays little beyond those entries (solved by the
@@ -430,7 +430,11 @@ def test_totals_beyond_16_bits_fall_back_to_the_wide_kernel(S, oracle_mod):
     lat[3::4, :, 0, :] = 130_000            # one core: 130 buckets; two cores: 65; budget 420, so
     lat[3::4, :, 1, :] = 65_000             # six stages only fit with two cores everywhere
     lat[3::4, :, :, 1:] = 900_000           # larger batches never fit
-    wl = dataclasses.replace(base, replicas=rep, lambda_mrps=lam, lat_us=lat)
+    return dataclasses.replace(base, replicas=rep, lambda_mrps=lam, lat_us=lat)
+
+
+def test_totals_beyond_16_bits_fall_back_to_the_wide_kernel(S, oracle_mod):
+    wl = _beyond_16_bits_workload()
     ref = oracle_mod.solve_batch(wl, dumps=True)
     assert (ref["status"] == 1).any()
     assert ((ref["total_cost"] > 0) & (ref["total_cost"] < S.INF16)).any()
@@ -438,8 +442,111 @@ def test_totals_beyond_16_bits_fall_back_to_the_wide_kernel(S, oracle_mod):
     solved = ref["status"] == 0
     assert (solved & (ref["total_cost"] >= S.INF16) & (beyond < S.INF16)).any()
     assert (solved[3::4] & (beyond[3::4] >= S.INF16)).all()
-    S.themis_set_minplus_mode(0)
-    _assert_results_equal(_gpu_solve(S, wl), ref)
+    _assert_results_equal(_gpu_solve(S, wl, mode=0), ref)
+
+
+def test_recurrence_step_repeats_on_a_scored_workspace(S, oracle_mod):
+    """themis_minplus_batch only consumes G and Garg: called again on the same scored
+    workspace, with the same or another kernel, it returns the same results.  On the
+    workload whose dear instances the packed kernel hands to the 32-bit kernel (they stay
+    marked in the workspace between the calls)."""
+    import torch
+    wl = _beyond_16_bits_workload()
+    ref = oracle_mod.solve_batch(wl)
+    dev = S.workload_to_device(wl)
+    ws = S.alloc_workspace(S.Problem.of_workload(wl), True)
+    S.themis_score_batch(S.Problem.of_workload(wl), dev["lat_us"], dev["profile_id"], dev["lambda_mrps"],
+                         dev["replicas"], ws)
+    for kernel in (S.KERNEL_PACKED16, S.KERNEL_PACKED16, S.KERNEL_WIDE32, S.KERNEL_PRUNED, S.KERNEL_PACKED16):
+        out = S.alloc_result(wl.n_instances, wl.n_stages)
+        for v in out.values():
+            v.fill_(-9)
+        S.themis_minplus_batch(S.Problem.of_workload(wl, kernel), dev["replicas"], out, ws)
+        torch.cuda.synchronize()
+        _assert_results_equal({k: v.cpu().numpy() for k, v in out.items()}, ref)
+
+
+def _long_front_workload():
+    """Instances whose undominated lists are long.  Two stages, one batch size, replicas fixed:
+    latencies fall by a whole number of buckets per core, so every core count is an undominated
+    stage entry.  Instances 0 and 3: stage 0 costs 61 per core, stage 1 costs 1 per core, and
+    stage 0 gains 60 buckets per core against 1 in stage 1, so all 3600 pairs of core counts
+    up to 60 are undominated prefix states.  Instances 1 and 4: 100 undominated entries in a
+    stage.  Instances 2 and 5: two core counts matter."""
+    N, S_, C, w = 6, 2, 100, 100
+    lat = np.empty((N, S_, C, 1), np.int32)
+    rep = np.ones((N, S_), np.int32)
+    c = np.arange(1, C + 1)
+    for n in range(N):
+        kind = n % 3
+        if kind == 0:
+            lat[n, 0, :, 0] = (4000 - 60 * np.minimum(c, 60)) * w
+            lat[n, 1, :, 0] = (100 - np.minimum(c, 60)) * w
+            rep[n] = (61, 1)
+        elif kind == 1:
+            lat[n, 0, :, 0] = (3000 - 7 * c) * w + 13          # not a whole number of buckets
+            lat[n, 1, :, 0] = (900 - 3 * c) * w
+        else:
+            lat[n, 0, :, 0] = np.where(c < 40, 700, 300) * w
+            lat[n, 1, :, 0] = np.where(c < 7, 900, 500) * w
+    return W.Workload(name="long_fronts", n_instances=N, n_stages=S_, n_profiles=N, c_max=C, batch_sizes=(1,),
+                      h_max=1, slo_us=4200 * w, bucket_us=w, flags=W.QUEUE_PER_REPLICA, vertical=True,
+                      lat_us=lat, profile_id=np.arange(N, dtype=np.int32),
+                      lambda_mrps=np.full(N, 2000, np.uint32), replicas=rep)
+
+
+def test_sparse_kernel_hands_long_lists_to_the_block_kernel(S, oracle_mod):
+    """The warp-per-instance kernel keeps fixed-size lists; instances that outgrow them (here:
+    3600 prefix states against 256 slots, 100 stage entries against 64) are listed in the
+    workspace and redone by the block kernel.  Results equal the oracle's either way."""
+    import torch
+    wl = _long_front_workload()
+    ref = oracle_mod.solve_batch(wl, dumps=True)
+    assert (ref["status"] == 0).all()
+    front = lambda X: (X < np.concatenate([np.full(X.shape[:2] + (1,), S.G_INF, X.dtype),
+                                           np.minimum.accumulate(X, axis=2)[:, :, :-1]], axis=2)).sum(axis=2)
+    g, f = front(ref["G"]), front(ref["F"])
+    assert (f[[0, 3], 1] == 3600).all() and (g[[1, 4]] == 100).all() and (g[[2, 5]] <= 2).all()
+    prob = S.Problem.of_workload(wl, S.KERNEL_SPARSE)
+    out, ws = S.solve(wl, kernel=S.KERNEL_SPARSE)
+    torch.cuda.synchronize()
+    _assert_results_equal({k: v.cpu().numpy() for k, v in out.items()}, ref)
+    lay = S.themis_workspace_layout(prob, True)
+    redo_at = (lay.flag_offset + 4 * wl.n_instances + 255) // 256 * 256
+    redo = ws[redo_at:redo_at + 4 * (1 + wl.n_instances)].view(torch.int32).cpu().numpy()
+    assert redo[0] == 4 and sorted(redo[1:5].tolist()) == [0, 1, 3, 4]
+
+
+def test_two_host_threads_with_different_kernels(S, oracle_mod):
+    """The kernel choice travels with the call: two host threads, each on its own stream,
+    solve different batches with different kernels at the same time, repeatedly; every
+    result equals the oracle's."""
+    import threading
+    import torch
+    jobs = [(W.make_workload(2, 192), S.KERNEL_PACKED16), (W.make_workload(3, 256), S.KERNEL_SPARSE),
+            (W.make_workload(4, 24), S.KERNEL_WIDE32), (W.make_workload(2, 160), S.KERNEL_SPARSE_BLOCK)]
+    refs = [oracle_mod.solve_batch(wl) for wl, _ in jobs]
+    errors = []
+
+    def work(k):
+        try:
+            wl, kernel = jobs[k]
+            torch.cuda.set_device(0)
+            with torch.cuda.stream(torch.cuda.Stream()):
+                dev = S.workload_to_device(wl)
+                for _ in range(12):
+                    out, _ws = S.solve(wl, dev=dev, kernel=kernel)
+                    torch.cuda.current_stream().synchronize()
+                    _assert_results_equal({key: v.cpu().numpy() for key, v in out.items()}, refs[k])
+        except BaseException as e:          # reported by the main thread
+            errors.append((k, e))
+
+    threads = [threading.Thread(target=work, args=(k,)) for k in range(len(jobs))]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
 
 
 def test_two_step_entry_points_equal_the_solver(S, oracle_mod):
@@ -523,20 +630,14 @@ def test_full_size_configs_every_instance(S, oracle_mod, cfg, mode):
     _assert_results_equal(gpu, _oracle_cached(oracle_mod, ("full", cfg), wl))
 
 
-def test_full_size_config5_sampled(S, oracle_mod, mode):
+def test_full_size_config5_every_instance(S, oracle_mod, mode):
     """Configuration 5 (4096 instances, 20 stages, T = 8192) in the benchmark's launch
-    configuration: every instance is checked against the size-independent properties,
-    a seeded sample of 48 instances against the oracle one by one (the oracle needs
-    about a second per instance and core)."""
+    configuration: every instance against the oracle (one oracle run per session, a few
+    minutes of host time, shared by all kernel modes)."""
     wl = W.make_workload(5)
     gpu = _gpu_solve(S, wl)
     _check_properties(wl, gpu)
-    pick = np.unique(np.concatenate([
-        W.rand_int(77, 5, np.arange(46, dtype=np.uint64), 0, wl.n_instances - 1), [0, wl.n_instances - 1],
-        np.flatnonzero(gpu["status"] == 1)[:8]]))
-    sub = dataclasses.replace(wl, n_instances=len(pick), profile_id=wl.profile_id[pick].copy(),
-                              lambda_mrps=wl.lambda_mrps[pick].copy())
-    _assert_results_equal(gpu, _oracle_cached(oracle_mod, ("cfg5", tuple(pick.tolist())), sub), idx=pick)
+    _assert_results_equal(gpu, _oracle_cached(oracle_mod, ("full", 5), wl))
 
 
 def test_bounded_wait_gives_up_and_reports(S, oracle_mod):

@@ -14,7 +14,10 @@ GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "hand_cases.json")
 
 
 def _hand_workload(case):
-    lat = (np.asarray(case["lat_ms"], dtype=np.int64) * 1000).astype(np.int32)[None]  # [1][S][C][B]
+    if "lat_us" in case:
+        lat = np.asarray(case["lat_us"], dtype=np.int32)[None]                        # [1][S][C][B]
+    else:
+        lat = (np.asarray(case["lat_ms"], dtype=np.int64) * 1000).astype(np.int32)[None]
     S = lat.shape[1]
     rep = case["replicas"]
     return W.Workload(
