@@ -23,6 +23,9 @@ constexpr uint32_t kInfKey = kInfCost << kIdxBits;
 // instance has to be redone by the 32-bit kernel.
 constexpr int32_t kFlagBadInput = 1;
 constexpr int32_t kFlagNeedsWide = 2;
+// 3: set by the sparse warp kernels for an instance whose lists outgrew their capacities; it
+// is on the redo list and the block kernel solves it.
+constexpr int32_t kFlagRedo = 3;
 
 // Packed 16-bit path: costs are exact below kInf16 and saturate there; two of
 // them add without carrying into the neighbouring half-word.

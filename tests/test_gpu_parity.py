@@ -467,13 +467,15 @@ def test_recurrence_step_repeats_on_a_scored_workspace(S, oracle_mod):
 
 
 def _long_front_workload():
-    """Instances whose undominated lists are long.  Two stages, one batch size, replicas fixed:
+    """Instances whose undominated lists are long.  Three stages, one batch size, replicas fixed:
     latencies fall by a whole number of buckets per core, so every core count is an undominated
     stage entry.  Instances 0 and 3: stage 0 costs 61 per core, stage 1 costs 1 per core, and
     stage 0 gains 60 buckets per core against 1 in stage 1, so all 3600 pairs of core counts
-    up to 60 are undominated prefix states.  Instances 1 and 4: 100 undominated entries in a
-    stage.  Instances 2 and 5: two core counts matter."""
-    N, S_, C, w = 6, 2, 100, 100
+    up to 60 are undominated states of the first two stages (the third stage has 150 entries,
+    which also keeps the stage fronts out of the scratch of the upper-bound search, so nothing
+    is pruned).  Instances 1 and 4: 160 undominated entries in every stage.  Instances 2 and 5:
+    two core counts matter."""
+    N, S_, C, w = 6, 3, 160, 100
     lat = np.empty((N, S_, C, 1), np.int32)
     rep = np.ones((N, S_), np.int32)
     c = np.arange(1, C + 1)
@@ -482,22 +484,25 @@ def _long_front_workload():
         if kind == 0:
             lat[n, 0, :, 0] = (4000 - 60 * np.minimum(c, 60)) * w
             lat[n, 1, :, 0] = (100 - np.minimum(c, 60)) * w
-            rep[n] = (61, 1)
+            lat[n, 2, :, 0] = (600 - 2 * np.minimum(c, 150)) * w
+            rep[n] = (61, 1, 1)
         elif kind == 1:
             lat[n, 0, :, 0] = (3000 - 7 * c) * w + 13          # not a whole number of buckets
             lat[n, 1, :, 0] = (900 - 3 * c) * w
+            lat[n, 2, :, 0] = (500 - c) * w
         else:
             lat[n, 0, :, 0] = np.where(c < 40, 700, 300) * w
             lat[n, 1, :, 0] = np.where(c < 7, 900, 500) * w
+            lat[n, 2, :, 0] = np.where(c < 90, 400, 350) * w
     return W.Workload(name="long_fronts", n_instances=N, n_stages=S_, n_profiles=N, c_max=C, batch_sizes=(1,),
-                      h_max=1, slo_us=4200 * w, bucket_us=w, flags=W.QUEUE_PER_REPLICA, vertical=True,
+                      h_max=1, slo_us=4700 * w, bucket_us=w, flags=W.QUEUE_PER_REPLICA, vertical=True,
                       lat_us=lat, profile_id=np.arange(N, dtype=np.int32),
-                      lambda_mrps=np.full(N, 2000, np.uint32), replicas=rep)
+                      lambda_mrps=np.full(N, 1000, np.uint32), replicas=rep)
 
 
 def test_sparse_kernel_hands_long_lists_to_the_block_kernel(S, oracle_mod):
-    """The warp-per-instance kernel keeps fixed-size lists; instances that outgrow them (here:
-    3600 prefix states against 256 slots, 100 stage entries against 64) are listed in the
+    """The warp-per-instance kernels keep fixed-size lists; instances that outgrow them (here:
+    3600 prefix states against 256 slots, 160 stage entries against 128) are listed in the
     workspace and redone by the block kernel.  Results equal the oracle's either way."""
     import torch
     wl = _long_front_workload()
@@ -506,7 +511,8 @@ def test_sparse_kernel_hands_long_lists_to_the_block_kernel(S, oracle_mod):
     front = lambda X: (X < np.concatenate([np.full(X.shape[:2] + (1,), S.G_INF, X.dtype),
                                            np.minimum.accumulate(X, axis=2)[:, :, :-1]], axis=2)).sum(axis=2)
     g, f = front(ref["G"]), front(ref["F"])
-    assert (f[[0, 3], 1] == 3600).all() and (g[[1, 4]] == 100).all() and (g[[2, 5]] <= 2).all()
+    assert (f[[0, 3], 1] == 3600).all() and (g[[0, 3], 2] == 150).all()
+    assert (g[[1, 4]] == 160).all() and (g[[2, 5]] <= 2).all()
     prob = S.Problem.of_workload(wl, S.KERNEL_SPARSE)
     out, ws = S.solve(wl, kernel=S.KERNEL_SPARSE)
     torch.cuda.synchronize()
