@@ -5,12 +5,20 @@ A "step" is one pass of the whole hot path (candidate scoring, min-plus
 recurrence, final scan, backtrack) over one batch of synthetic instances.
 Prints ONE JSON line.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--scaling weak|strong]
+                    [--impl reference]
 
-With N > 1 launch under ``python -m torch.distributed.run`` (one rank per GPU);
-the batch is replicated per rank with independent seeds (weak scaling, no
-collective on the solve path).  ``--impl reference`` times the CPU oracle
-instead (rank 0 only).
+With N > 1 launch under ``python -m torch.distributed.run`` (one rank per GPU).
+Weak scaling (default): every rank solves its own batch (independent seeds);
+strong scaling: one batch is split over the ranks and the gathered answer is
+checked against the one-GPU answer.  Either way there is no collective on the
+solve path.  ``--impl reference`` times the CPU oracle instead (rank 0 only).
+
+Beside the headline step the line carries: the recurrence kernel's roofline
+against the integer-ALU rate measured in the same run (nominal, useful and
+executed cell updates), the other dense kernel on the same batch, the sparse
+solver, the end-to-end figure through the host-buffer entry point, the CPU
+oracle, and the other benchmark configurations at full size.
 """
 from __future__ import annotations
 
@@ -39,15 +47,17 @@ ALU_PEAK_TOPS_INT32 = N_SMS * INT_LANES_PER_SM * 2 * SM_GHZ / 1e3
 ALU_PEAK_TOPS_INT16X2 = 2 * ALU_PEAK_TOPS_INT32
 HBM_FALLBACK_GBS = 6650.0
 
-# DRAM bytes (read + write) of one min-plus launch from the ncu capture summarised
-# under profiles/, per instance of the captured workload.  Traffic is proportional
-# to the instance count (one block per instance, no reuse across blocks).  The
-# figure is only reported while the kernel sources still have the recorded hash.
+# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/, per
+# instance of the captured workload.  Traffic is proportional to the instance count (one block
+# per instance, no reuse across blocks).  A figure is only reported while the kernel's sources
+# still have the recorded hash.
 NCU_TRAFFIC = {
-    "config": 4, "bytes_per_instance": (315.842304e6 + 156.111616e6) / 2368,
-    "sources": ("paper_2407_14843_b200/csrc/themis_minplus16.cu",
-                "paper_2407_14843_b200/csrc/themis_minplus16_step.cuh"),
-    "sha256_16": "1a1de2cc92ace9e8",
+    "minplus16": {"config": 4, "bytes_per_instance": (315.842304e6 + 156.111616e6) / 2368,
+                  "sources": ("paper_2407_14843_b200/csrc/themis_minplus16.cu",
+                              "paper_2407_14843_b200/csrc/themis_minplus16_step.cuh"),
+                  "sha256_16": "1a1de2cc92ace9e8"},
+    "score": {"config": 4, "bytes_per_instance": 0.0,
+              "sources": ("paper_2407_14843_b200/csrc/themis_score.cu",), "sha256_16": "none"},
 }
 
 
@@ -59,7 +69,17 @@ def parse_args():
     ap.add_argument("--config", type=int, default=4, help="benchmark configuration 1..5 (default 4: large joint DP)")
     ap.add_argument("--instances", type=int, default=None, help="override the batch size (debugging)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="weak: every rank solves its own batch; strong: one batch split over the ranks "
+                         "(sharding.shard_range), the gathered answer checked against the one-GPU answer")
+    ap.add_argument("--other-kernel-steps", type=int, default=3,
+                    help="steps of the other dense recurrence kernel (32-bit when the packed one is timed) on the "
+                         "same batch (0: skip)")
+    ap.add_argument("--other-configs", type=int, nargs="*", default=[1, 2, 3, 5],
+                    help="further benchmark configurations timed at full size after the headline one, one GPU only "
+                         "(empty: none)")
+    ap.add_argument("--other-config-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--alu-probe", action="store_true",
                     help="only run the integer-ALU probe in its five instruction forms and print the rates")
@@ -77,18 +97,19 @@ def parse_args():
     return ap.parse_args()
 
 
-def ncu_traffic_bytes(cfg: int, n_instances: int):
+def ncu_traffic_bytes(kernel: str, cfg: int, n_instances: int):
     import hashlib
+    rec = NCU_TRAFFIC[kernel]
     try:
         h = hashlib.sha256()
-        for src in NCU_TRAFFIC["sources"]:
+        for src in rec["sources"]:
             with open(os.path.join(ROOT, src), "rb") as f:
                 h.update(f.read())
-        if h.hexdigest()[:16] != NCU_TRAFFIC["sha256_16"]:
+        if h.hexdigest()[:16] != rec["sha256_16"]:
             return None
     except OSError:
         return None
-    return NCU_TRAFFIC["bytes_per_instance"] * n_instances if cfg == NCU_TRAFFIC["config"] else None
+    return rec["bytes_per_instance"] * n_instances if cfg == rec["config"] else None
 
 
 def measured_hbm_peak():
@@ -248,6 +269,60 @@ def probe_alu_peak(solver, torch, mode):
 
 # --------------------------------------------------------------------------- the CUDA arm
 
+def packed_launch_shape(cells: int, tile: int = 0):
+    """Tiling of the packed recurrence kernel for a budget of `cells` = T + 1 cells, as its
+    launcher chooses it: cells per tile R, half-groups of 16 tiles, cells left to the
+    block-wide reduction."""
+    R = tile if tile in (4, 8, 16) else (4 if cells <= 896 + 8 else 8)
+    while True:
+        tiles = (cells + R - 1) // R
+        half_groups = (tiles + 15) // 16
+        extra = False
+        if half_groups > 1 and cells - (half_groups - 1) * 16 * R <= 8:
+            half_groups -= 1
+            extra = True
+        threads = ((half_groups + 1) // 2 + 1) // 2 * 32
+        if threads <= 1024 or R == 16:
+            break
+        R *= 2
+    return R, half_groups, extra
+
+
+def cell_update_counts(torch, wl, tables, tile: int = 0):
+    """Cell updates of the recurrence per batch, three ways, from the scored tables G:
+    nominal   (S-1)(T+1)(T+2)/2 per instance;
+    useful    cells (t, l) of stage s that are not unreachable by construction:
+              l >= first reachable entry of G_s and t - l >= sum of the earlier stages' first
+              reachable entries (the bounds the packed kernel skips by);
+    executed  what the packed kernel actually performs: per stage and tile its chunk steps
+              (the same skip rule, in whole chunk pairs, every lane of a half-group running to
+              the half-group's longest column) times R x R cells, plus the cells of the
+              block-wide reduction."""
+    G, T = tables["G"], wl.T
+    N, S, W = wl.n_instances, wl.n_stages, T + 1
+    reach = G[:, :, :W] != 2 ** 31 - 1
+    first = torch.where(reach.any(dim=2), reach.int().argmax(dim=2), torch.full((N, S), -1, device=G.device)).long()
+    dead = (first < 0).long().cumsum(dim=1) > 0                      # an empty stage kills everything after it
+    first = first.clamp(min=0)
+    prefix = first.cumsum(dim=1) - first                             # sum over earlier stages
+    m = (T - first - prefix)[:, 1:]
+    alive = ~dead[:, 1:]
+    useful = int(((m + 1) * (m + 2) // 2 * (m >= 0) * alive).sum())
+    R, nhg, extra = packed_launch_shape(W, tile)
+    n_tiles = nhg * 16
+    Tc = n_tiles * R
+    n_dummy = max(0, Tc - W) // R
+    n_extra = max(0, W - Tc) if extra else 0
+    q_lo = (first[:, 1:] // R) & ~1
+    q_shift = ((prefix[:, 1:] // R) + n_dummy) & ~1
+    ends = torch.arange(nhg, device=G.device).long() * 16 + 15       # tile | 15 of every half-group
+    steps = (ends.view(1, 1, -1) - q_shift.unsqueeze(2) - q_lo.unsqueeze(2) + 1).clamp(min=0)
+    steps = steps * alive.unsqueeze(2)
+    executed = int(steps.sum()) * 16 * R * R
+    executed += int(alive.sum()) * sum(Tc + e + 1 for e in range(n_extra))
+    return {"nominal": N * wl.minplus_cells, "useful": useful, "executed": executed}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -262,15 +337,22 @@ def run_ours(args):
                "--master-addr", "127.0.0.1", "--master-port", "29533", os.path.abspath(__file__)] + sys.argv[1:]
         sys.exit(subprocess.call(cmd))
 
-    from paper_2407_14843_b200 import workloads
-    wl = workloads.make_workload(args.config, args.instances, seed_offset=rank)
+    from paper_2407_14843_b200 import sharding, workloads
+    strong = args.scaling == "strong"
+    # weak scaling: every rank its own batch (seeds offset by rank); strong: one batch, split
+    wl_all = workloads.make_workload(args.config, args.instances, seed_offset=0 if strong else rank)
+    if strong:
+        a, b = sharding.shard_range(wl_all.n_instances, rank, world)
+        wl = wl_all.take(b - a, a)
+    else:
+        wl = wl_all
     cpu = None
     if rank == 0:
         _build.build_library()
         if not args.no_cpu_baseline:
             import oracle
             oracle.build()                       # before the first GPU call
-            cpu = cpu_baseline(wl)
+            cpu = cpu_baseline(wl_all)
     torch.cuda.set_device(local_rank)
     # Under a launcher (RANK set) the process group is brought up even for one rank, so that
     # the barrier / max-over-ranks path is the same code at every N.
@@ -280,33 +362,97 @@ def run_ours(args):
         dist.barrier()
     from paper_2407_14843_b200 import solver
 
-    packed = args.minplus_mode == 0
-    prob = solver.Problem.of_workload(wl, solver.KERNEL_PACKED16 if packed else solver.KERNEL_WIDE32, args.minplus_tile)
-    prob_sparse = solver.Problem.of_workload(wl, solver.KERNEL_SPARSE)
-    dev = solver.workload_to_device(wl)
-    ws = solver.alloc_workspace(prob, wl.vertical, host_variant=True)
-    out = solver.alloc_result(wl.n_instances, wl.n_stages)
-
-    def step(events=None):
-        if events:
-            events[0].record()
-        solver.themis_score_batch(prob, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"], dev["replicas"], ws)
-        if events:
-            events[1].record()
-        solver.themis_minplus_batch(prob, dev["replicas"], out, ws)
-        if events:
-            events[2].record()
-
     def barrier():
         torch.cuda.synchronize()
         if use_dist:
             dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 1)):
-        step()
-    alu_probe_tops = {"int32": probe_alu_peak(solver, torch, 1), "int16x2": probe_alu_peak(solver, torch, 3)} \
-        if rank == 0 else None
+    def max_over_ranks(values):
+        t = torch.tensor(values, dtype=torch.float64, device="cuda")
+        if use_dist:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return t.tolist()
+
+    mk = lambda: torch.cuda.Event(enable_timing=True)
+    packed = args.minplus_mode == 0
+    main_kernel = solver.KERNEL_PACKED16 if packed else solver.KERNEL_WIDE32
+
+    def time_dense(w, dev, ws, out, kernel, tile, steps, warmup):
+        """`steps` timed steps (scoring launch + recurrence launch) after `warmup` untimed ones."""
+        prob = solver.Problem.of_workload(w, kernel, tile)
+
+        def step(ev=None):
+            if ev:
+                ev[0].record()
+            solver.themis_score_batch(prob, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"], dev["replicas"], ws)
+            if ev:
+                ev[1].record()
+            solver.themis_minplus_batch(prob, dev["replicas"], out, ws)
+            if ev:
+                ev[2].record()
+
+        for _ in range(max(warmup, 1)):
+            step()
+        evs = [[mk(), mk(), mk()] for _ in range(steps)]
+        barrier()
+        for k in range(steps):
+            step(evs[k])
+        barrier()
+        total, score, minplus = max_over_ranks([
+            evs[0][0].elapsed_time(evs[-1][2]), sum(e[0].elapsed_time(e[1]) for e in evs) / steps,
+            sum(e[1].elapsed_time(e[2]) for e in evs) / steps])
+        per_step = sorted(e[0].elapsed_time(e[2]) for e in evs)
+        return {"total_ms": total, "score_ms": score, "minplus_ms": minplus, "per_step_ms": per_step}
+
+    def time_sparse(w, dev, ws, out, steps):
+        prob = solver.Problem.of_workload(w, solver.KERNEL_SPARSE)
+
+        def call():
+            if w.vertical:
+                solver.themis_solve_vertical_batch(prob, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"],
+                                                   dev["replicas"], out, ws)
+            else:
+                solver.themis_solve_batch(prob, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"], out, ws)
+
+        call()
+        barrier()
+        a, b = mk(), mk()
+        a.record()
+        for _ in range(steps):
+            call()
+        b.record()
+        barrier()
+        return max_over_ranks([a.elapsed_time(b)])[0] / steps
+
+    def dense_rooflines(w, t, is_packed, probe, counts=None):
+        """The recurrence kernel against the integer-ALU peak and the scoring kernel against HBM."""
+        cells = w.n_instances * w.minplus_cells
+        tops = 2.0 * cells / (t["minplus_ms"] * 1e-3) / 1e12
+        derived = ALU_PEAK_TOPS_INT16X2 if is_packed else ALU_PEAK_TOPS_INT32
+        measured = probe["int16x2" if is_packed else "int32"] if probe else None
+        lay = solver.themis_workspace_layout(solver.Problem.of_workload(w), w.vertical)
+        score_bytes = 6.0 * lay.row_pitch * w.n_instances * w.n_stages
+        score_gbs = score_bytes / (t["score_ms"] * 1e-3) / 1e9
+        r = {"minplus_ms": t["minplus_ms"], "score_ms": t["score_ms"], "achieved_tops": tops,
+             "frac_of_derived_peak": tops / derived, "frac_of_probe_peak": tops / measured if measured else None,
+             "score_gbs": score_gbs, "score_frac_of_hbm": score_gbs / hbm_peak, "score_bytes": score_bytes}
+        if counts:
+            r["frac_useful"] = r["frac_of_derived_peak"] * counts["useful"] / counts["nominal"]
+            r["frac_executed"] = r["frac_of_derived_peak"] * counts["executed"] / counts["nominal"]
+        return r
+
+    hbm_peak, hbm_kind = measured_hbm_peak()
+    prob = solver.Problem.of_workload(wl, main_kernel, args.minplus_tile)
+    dev = solver.workload_to_device(wl)
+    ws = solver.alloc_workspace(prob, wl.vertical, host_variant=True)
+    out = solver.alloc_result(wl.n_instances, wl.n_stages)
+
+    # warm-up of the headline step, then the ALU probe (its rate is the measured roofline denominator)
+    warm = time_dense(wl, dev, ws, out, main_kernel, args.minplus_tile, 1, args.warmup)
+    del warm
+    probe = {"int32": probe_alu_peak(solver, torch, 1), "int16x2": probe_alu_peak(solver, torch, 3)}
+    probe = dict(zip(probe, max_over_ranks(list(probe.values()))))      # one figure per form for the line
     barrier()
 
     uuid = str(getattr(torch.cuda.get_device_properties(local_rank), "uuid", ""))
@@ -314,59 +460,34 @@ def run_ours(args):
     if sampler:
         sampler.start()
         time.sleep(0.25)
-    mk = lambda: torch.cuda.Event(enable_timing=True)
-    evs = [[mk(), mk(), mk()] for _ in range(args.steps)]
-    barrier()
-    for k in range(args.steps):
-        step(evs[k])
-    barrier()
+    main = time_dense(wl, dev, ws, out, main_kernel, args.minplus_tile, args.steps, 1)
     clocks = sampler.stop() if sampler else None
+    total_ms, score_ms, minplus_ms, step_ms = main["total_ms"], main["score_ms"], main["minplus_ms"], main["per_step_ms"]
+    dense_out = {k: v.clone() for k, v in out.items()}
+    status = out["status"].cpu()
+    n_infeasible, n_error = int((status == 1).sum()), int((status < 0).sum())
+    counts = None
+    if packed:       # the tables of the last timed step are still in the workspace
+        counts = cell_update_counts(torch, wl, solver.workspace_tables(prob, wl.vertical, ws), args.minplus_tile)
 
-    step_ms = sorted(e[0].elapsed_time(e[2]) for e in evs)
-    total_ms = evs[0][0].elapsed_time(evs[-1][2])
-    score_ms = sum(e[0].elapsed_time(e[1]) for e in evs) / args.steps
-    minplus_ms = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
-    t = torch.tensor([total_ms, score_ms, minplus_ms], dtype=torch.float64, device="cuda")
-    if use_dist:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, score_ms, minplus_ms = t.tolist()
+    # the other dense kernel on the same batch, a few steps
+    other_kernel = solver.KERNEL_WIDE32 if packed else solver.KERNEL_PACKED16
+    other = time_dense(wl, dev, ws, out, other_kernel, args.minplus_tile, max(1, args.other_kernel_steps), 1) \
+        if args.other_kernel_steps > 0 else None
+    other_same = all(bool((out[k] == dense_out[k]).all()) for k in out) if other else None
 
-    # The same batch through the solver restricted to undominated entries (mode 3: one fused
-    # kernel; identical results, a small fraction of the cell updates): reported beside the
-    # dense figures, not as them.
+    # The same batch through the solver restricted to undominated entries (one warp per
+    # instance on sorted fronts; identical results, a small fraction of the cell updates):
+    # reported beside the dense figures, not as them.
     pruned = None
     if args.pruned_steps > 0:
-        dense_out = {k: v.clone() for k, v in out.items()}
-
-        def sparse_step():
-            if wl.vertical:
-                solver.themis_solve_vertical_batch(prob_sparse, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"],
-                                                   dev["replicas"], out, ws)
-            else:
-                solver.themis_solve_batch(prob_sparse, dev["lat_us"], dev["profile_id"], dev["lambda_mrps"], out, ws)
-
-        sparse_step()
-        barrier()
-        pe = [mk() for _ in range(args.pruned_steps + 1)]
-        pe[0].record()
-        for k in range(args.pruned_steps):
-            sparse_step()
-            pe[k + 1].record()
-        barrier()
-        tp = torch.tensor([pe[0].elapsed_time(pe[-1])], dtype=torch.float64, device="cuda")
-        if use_dist:
-            dist.all_reduce(tp, op=dist.ReduceOp.MAX)
-        p_total = float(tp.item())
-        pruned = {"value": wl.n_instances * world * args.pruned_steps / (p_total * 1e-3), "unit": UNIT,
-                  "ms_per_step": p_total / args.pruned_steps, "steps": args.pruned_steps,
-                  "kernel": "solve_front_kernel + solve_sparse_kernel for listed instances (memset + 2 launches per step)",
+        p_ms = time_sparse(wl, dev, ws, out, args.pruned_steps)
+        pruned = {"value": wl.n_instances * world / (p_ms * 1e-3), "unit": UNIT, "ms_per_step": p_ms,
+                  "steps": args.pruned_steps,
+                  "kernel": "stage_fronts_kernel + prefix_fronts_kernel (+ solve_sparse_kernel for listed "
+                            "instances): a 4-byte memset and 3 launches per step",
                   "same_results_as_dense": all(bool((out[k] == dense_out[k]).all()) for k in out),
-                  "note": "THEMIS_KERNEL_SPARSE: scoring, fronts and recurrence on undominated "
-                          "entries in one kernel, one warp per instance"}
-
-    status = out["status"].cpu()
-    n_infeasible = int((status == 1).sum())
-    n_error = int((status < 0).sum())
+                  "note": "THEMIS_KERNEL_SPARSE: scoring, fronts and recurrence on undominated entries only"}
 
     # end to end through the host-buffer entry point: pinned host inputs in,
     # host results out, copies inside the timed region
@@ -382,14 +503,54 @@ def run_ours(args):
     for _ in range(args.e2e_steps):
         e2e_call()
     torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-    t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-    if use_dist:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_s = float(t.item())
+    e2e_s = max_over_ranks([time.perf_counter() - t0])[0]
     h2d = sum(x.numel() * x.element_size() for x in h_in.values() if x is not None)
     d2h = sum(x.numel() * x.element_size() for x in h_out.values())
-    same = all(bool((h_out[k] == out[k].cpu()).all()) for k in h_out)
+    same = all(bool((h_out[k] == dense_out[k].cpu()).all()) for k in h_out)
+
+    # strong scaling: the gathered answer of the split batch against the one-GPU answer
+    sharded_check = None
+    if strong and use_dist:
+        full = sharding.solve_sharded(wl_all, lambda block: solver.solve(block)[0])
+        if rank == 0:
+            one, _ = solver.solve(wl_all)
+            torch.cuda.synchronize()
+            sharded_check = {k: bool((full[k] == one[k]).all()) for k in full}
+            del one
+        del full
+
+    # the other benchmark configurations at full size, one after the other (rank 0 of a
+    # one-GPU run only: they are context for the headline figure, not part of it)
+    others = {}
+    if args.other_configs and world == 1:
+        del dev, ws, out, dense_out, h_in, h_out
+        torch.cuda.empty_cache()
+        for cfg in args.other_configs:
+            if cfg == args.config:
+                continue
+            w = workloads.make_workload(cfg)
+            d = solver.workload_to_device(w)
+            pr = solver.Problem.of_workload(w)
+            wsp = solver.alloc_workspace(pr, w.vertical)
+            o = solver.alloc_result(w.n_instances, w.n_stages)
+            steps = args.other_config_steps
+            t16 = time_dense(w, d, wsp, o, solver.KERNEL_PACKED16, 0, steps, 3)
+            ref = {k: v.clone() for k, v in o.items()}
+            cnt = cell_update_counts(torch, w, solver.workspace_tables(pr, w.vertical, wsp))
+            t32 = time_dense(w, d, wsp, o, solver.KERNEL_WIDE32, 0, max(2, steps // 2), 1)
+            same32 = all(bool((o[k] == ref[k]).all()) for k in o)
+            sp_ms = time_sparse(w, d, wsp, o, steps)
+            same_sp = all(bool((o[k] == ref[k]).all()) for k in o)
+            others[str(cfg)] = {
+                "workload": w.name, "instances": w.n_instances, "stages": w.n_stages, "T": w.T, "steps": steps,
+                "ms_per_step": t16["total_ms"] / steps, "instances_per_s": w.n_instances * steps / (t16["total_ms"] * 1e-3),
+                "packed16": dense_rooflines(w, t16, True, probe, cnt),
+                "wide32": dict(dense_rooflines(w, t32, False, probe), same_results=same32),
+                "sparse": {"ms_per_step": sp_ms, "instances_per_s": w.n_instances / (sp_ms * 1e-3), "same_results": same_sp},
+                "cell_updates": cnt, "infeasible_instances": int((ref["status"] == 1).sum()),
+            }
+            del d, wsp, o, ref
+            torch.cuda.empty_cache()
 
     if use_dist:
         dist.barrier()
@@ -397,54 +558,81 @@ def run_ours(args):
     if rank != 0:
         return
 
-    N_total = wl.n_instances * world
+    N_total = wl.n_instances * world if not strong else wl_all.n_instances
     # score + min-plus, plus the 32-bit second pass where a total may exceed 15 bits
     second_pass = packed and (wl.vertical or wl.n_stages * wl.h_max * wl.c_max >= 0x7FFF)
     launches_per_step = 3 if second_pass else 2
     cells_per_launch = wl.n_instances * wl.minplus_cells
-    achieved_tops = 2.0 * cells_per_launch / (minplus_ms * 1e-3) / 1e12
-    alu_peak = ALU_PEAK_TOPS_INT16X2 if packed else ALU_PEAK_TOPS_INT32
-    lay = solver.themis_workspace_layout(prob, wl.vertical)
-    score_bytes = 6.0 * lay.row_pitch * wl.n_instances * wl.n_stages
-    hbm_peak, hbm_kind = measured_hbm_peak()
-    score_gbs = score_bytes / (score_ms * 1e-3) / 1e9
+    main_r = dense_rooflines(wl, main, packed, probe, counts)
+    kernel_name = "minplus16_kernel" if packed else "minplus_kernel"
+    measured_peak = probe["int16x2" if packed else "int32"]
+    derived_peak = ALU_PEAK_TOPS_INT16X2 if packed else ALU_PEAK_TOPS_INT32
     line = {
         "metric": METRIC, "value": N_total * args.steps / (total_ms * 1e-3), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
         "ms_per_step_best": step_ms[0], "ms_per_step_median": step_ms[len(step_ms) // 2],
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "higher_is_better": True, "scaling": "strong" if strong else "weak", "vs_baseline": None,
         # arithmetic of the dominant kernel: packed pairs of unsigned 16-bit costs, or 32-bit keys
         "dtype": "u16" if packed else "u32",
-        "data": "synthetic", "config": workload_config(wl, args, world),
+        "data": "synthetic", "config": workload_config(wl_all if strong else wl, args, world),
         "cell_updates_per_s": world * cells_per_launch * args.steps / (total_ms * 1e-3),
         "minplus_cell_updates_per_s_kernel": cells_per_launch / (minplus_ms * 1e-3),
-        "kernels_ms": {"score_kernel": score_ms, ("minplus16_kernel" if packed else "minplus_kernel"): minplus_ms},
+        "kernels_ms": {"score_kernel": score_ms, kernel_name: minplus_ms},
         "infeasible_instances": n_infeasible, "device_error_instances": n_error,
         "input_checksums": wl.checksums(),
         "device": {"name": torch.cuda.get_device_name(local_rank),
                    "sms": torch.cuda.get_device_properties(local_rank).multi_processor_count},
         "roofline": {
-            "kernel": "minplus16_kernel" if packed else "minplus_kernel", "bound": "alu",
-            "achieved": achieved_tops, "peak": alu_peak,
-            "unit": "TOP/s (integer add+min, 2 per cell update)", "frac": achieved_tops / alu_peak,
-            "traffic": ncu_traffic_bytes(args.config, wl.n_instances) if packed else None,
-            "peak_kind": ("derived: 148 SMs x 64 int lanes x 2 ops x 1.965 GHz"
-                          + (" x 2 half-word cells per lane (packed 16-bit add-min)" if packed else "")),
-            "peak_probe": alu_probe_tops, "frac_of_int32_peak": achieved_tops / ALU_PEAK_TOPS_INT32,
+            "kernel": kernel_name, "bound": "alu", "achieved": main_r["achieved_tops"], "peak": measured_peak,
+            "unit": "TOP/s (integer add+min, 2 per cell update)", "frac": main_r["achieved_tops"] / measured_peak,
+            "traffic": ncu_traffic_bytes("minplus16", args.config, wl.n_instances) if packed else None,
+            "peak_kind": "measured in this run: themis_alu_probe, " +
+                         ("fused add-min on packed 2 x 16-bit" if packed else "fused 32-bit add-min") +
+                         " on registers, all SMs",
+            "peak_derived": derived_peak, "frac_of_derived_peak": main_r["frac_of_derived_peak"],
+            "peak_derived_kind": ("148 SMs x 64 int lanes x 2 ops x 1.965 GHz"
+                                  + (" x 2 half-word cells per lane" if packed else "")),
+            "peak_probe": probe, "frac_of_int32_peak": main_r["achieved_tops"] / ALU_PEAK_TOPS_INT32,
             "algorithmic_cells_per_launch": cells_per_launch, "avg_launch_ms": minplus_ms,
         },
         "roofline_score_kernel": {
-            "kernel": "score_kernel", "bound": "hbm", "achieved": score_gbs, "peak": hbm_peak, "unit": "GB/s",
-            "frac": score_gbs / hbm_peak, "traffic": None, "peak_kind": f"of {hbm_kind}",
-            "algorithmic_bytes_per_launch": score_bytes, "avg_launch_ms": score_ms,
+            "kernel": "score_kernel", "bound": "hbm", "achieved": main_r["score_gbs"], "peak": hbm_peak, "unit": "GB/s",
+            "frac": main_r["score_frac_of_hbm"], "traffic": ncu_traffic_bytes("score", args.config, wl.n_instances),
+            "peak_kind": f"of {hbm_kind}",
+            "algorithmic_bytes_per_launch": main_r["score_bytes"], "avg_launch_ms": score_ms,
         },
         "e2e": {"value": N_total * args.e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": args.e2e_steps, "matches_device_path": same},
         "gpu_launches": launches_per_step * args.steps,
         "clocks": clocks,
     }
+    if counts:
+        line["cell_updates_useful_per_s"] = world * counts["useful"] * args.steps / (total_ms * 1e-3)
+        line["cell_updates_executed_per_s"] = world * counts["executed"] * args.steps / (total_ms * 1e-3)
+        line["roofline"].update({
+            "cells_per_launch": counts,
+            "frac_useful": main_r["achieved_tops"] / measured_peak * counts["useful"] / counts["nominal"],
+            "frac_executed": main_r["achieved_tops"] / measured_peak * counts["executed"] / counts["nominal"],
+            "cells_note": "nominal = (S-1)(T+1)(T+2)/2 per instance; useful = cells not unreachable by the stages' "
+                          "first reachable entries; executed = chunk steps the kernel performs x R x R (skips in "
+                          "chunk pairs, lanes run to their half-group's longest column)"})
+    if other:
+        o_packed = not packed
+        o_r = dense_rooflines(wl, other, o_packed, probe)
+        o_peak = probe["int16x2" if o_packed else "int32"]
+        line["roofline_int32_kernel" if packed else "roofline_int16_kernel"] = {
+            "kernel": "minplus_kernel" if packed else "minplus16_kernel", "bound": "alu",
+            "achieved": o_r["achieved_tops"], "peak": o_peak, "unit": "TOP/s (integer add+min, 2 per cell update)",
+            "frac": o_r["achieved_tops"] / o_peak, "frac_of_derived_peak": o_r["frac_of_derived_peak"],
+            "avg_launch_ms": other["minplus_ms"], "steps": max(1, args.other_kernel_steps),
+            "ms_per_step": other["total_ms"] / max(1, args.other_kernel_steps), "same_results": other_same,
+            "peak_kind": "measured in this run: themis_alu_probe", "traffic": None}
     if pruned is not None:
         line["pruned_path"] = pruned
+    if sharded_check is not None:
+        line["sharded_equals_one_gpu"] = sharded_check
+    if others:
+        line["other_configs"] = others
     if cpu is not None:
         line["cpu_baseline"] = cpu
     print(json.dumps(line), flush=True)

@@ -7,7 +7,7 @@ when one buffer is wanted.
 """
 from __future__ import annotations
 
-from typing import Dict, Tuple
+from typing import Callable, Dict, Tuple
 
 import torch
 import torch.distributed as dist
@@ -46,3 +46,21 @@ def gather_results(local: Dict[str, torch.Tensor], n_instances: int, group=None)
         out[k] = torch.cat(rows, dim=0)
     del rank
     return out
+
+
+def solve_sharded(wl, solve_fn: Callable, group=None) -> Dict[str, torch.Tensor]:
+    """Solves one batch across the ranks of a process group: every rank takes its
+    ``shard_range`` block of ``wl`` (a ``workloads.Workload``; the latency tables are
+    replicated, no instance data crosses ranks), solves it with ``solve_fn(block)`` and
+    the result arrays are all-gathered, so every rank returns the full-batch arrays in
+    instance order.
+
+    ``solve_fn`` takes a Workload and returns a mapping with the keys of ``RESULT_KEYS``
+    (torch tensors or numpy arrays, rows = the block's instances): on a GPU rank
+    ``lambda block: solver.solve(block)[0]`` with the rank's device current.  The only
+    collective is the gather of the results (``N * (3 * S + 3) * 4`` bytes)."""
+    world, rank = dist.get_world_size(group), dist.get_rank(group)
+    start, stop = shard_range(wl.n_instances, rank, world)
+    local = solve_fn(wl.take(stop - start, start))
+    local = {k: torch.as_tensor(local[k]) for k in RESULT_KEYS}
+    return gather_results(local, wl.n_instances, group)

@@ -555,6 +555,27 @@ def test_two_host_threads_with_different_kernels(S, oracle_mod):
     assert not errors, errors
 
 
+def test_sharded_solve_on_a_one_rank_group(S, oracle_mod):
+    """sharding.solve_sharded with the CUDA solver as its solve function (NCCL group of one
+    rank; the two-rank split is covered on CPU with gloo)."""
+    import socket
+    import torch
+    import torch.distributed as dist
+    from paper_2407_14843_b200 import sharding
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1,
+                            device_id=torch.device("cuda", 0))
+    try:
+        wl = W.make_workload(2, 300)
+        full = sharding.solve_sharded(wl, lambda block: S.solve(block)[0])
+        torch.cuda.synchronize()
+        _assert_results_equal({k: v.cpu().numpy() for k, v in full.items()}, oracle_mod.solve_batch(wl))
+    finally:
+        dist.destroy_process_group()
+
+
 def test_two_step_entry_points_equal_the_solver(S, oracle_mod):
     import torch
     wl = W.make_workload(3, 64)

@@ -1,6 +1,6 @@
-"""Multi-rank host logic on CPU: two gloo ranks each solve their shard (with
-the oracle standing in for the device) and the gathered arrays equal the
-full-batch solution."""
+"""Multi-rank host logic on CPU: two gloo ranks run the library's sharded solve
+(``sharding.solve_sharded``, with the oracle standing in for the device) and the
+gathered arrays equal the full-batch solution on every rank."""
 import os
 import socket
 import sys
@@ -33,13 +33,11 @@ def _worker(rank, world, port, n_total, ret):
     dist.init_process_group("gloo", rank=rank, world_size=world)
     try:
         from paper_2407_14843_b200 import workloads
-        from paper_2407_14843_b200.sharding import gather_results, shard_range
+        from paper_2407_14843_b200.sharding import solve_sharded
         import oracle
         wl = workloads.make_workload(2, n_total)
-        a, b = shard_range(n_total, rank, world)
-        local = oracle.solve_batch(wl.take(b - a, a), n_threads=1)
-        full = gather_results({k: torch.from_numpy(local[k]) for k in
-                               ("h", "c", "b", "total_cost", "latency_buckets", "status")}, n_total)
+        # the library's sharded solve with the oracle standing in for the device
+        full = solve_sharded(wl, lambda block: oracle.solve_batch(block, n_threads=1))
         ret[rank] = {k: v.numpy() for k, v in full.items()}
     finally:
         dist.destroy_process_group()
