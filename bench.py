@@ -294,10 +294,13 @@ def cell_update_counts(torch, wl, tables, tile: int = 0):
     useful    cells (t, l) of stage s that are not unreachable by construction:
               l >= first reachable entry of G_s and t - l >= sum of the earlier stages' first
               reachable entries (the bounds the packed kernel skips by);
-    executed  what the packed kernel actually performs: per stage and tile its chunk steps
-              (the same skip rule, in whole chunk pairs, every lane of a half-group running to
-              the half-group's longest column) times R x R cells, plus the cells of the
-              block-wide reduction."""
+    needed    useful cells whose budget t the later stages can still complete:
+              t <= T - sum of the later stages' first reachable entries (the packed kernel
+              computes no budget above that limit);
+    executed  what the packed kernel actually performs: per stage and tile in use its chunk
+              steps (the same skip rules, in whole chunk pairs and half-groups of 16 tiles, every
+              lane of a half-group running to the half-group's longest column) times R x R cells,
+              plus the cells of the block-wide reduction."""
     G, T = tables["G"], wl.T
     N, S, W = wl.n_instances, wl.n_stages, T + 1
     reach = G[:, :, :W] != 2 ** 31 - 1
@@ -305,9 +308,13 @@ def cell_update_counts(torch, wl, tables, tile: int = 0):
     dead = (first < 0).long().cumsum(dim=1) > 0                      # an empty stage kills everything after it
     first = first.clamp(min=0)
     prefix = first.cumsum(dim=1) - first                             # sum over earlier stages
+    later = (first.sum(dim=1, keepdim=True) - first.cumsum(dim=1)).clamp(max=W)   # sum over later stages
+    t_max = (T - later)[:, 1:]                                       # budget limit of stages 1..S-1
     m = (T - first - prefix)[:, 1:]
-    alive = ~dead[:, 1:]
-    useful = int(((m + 1) * (m + 2) // 2 * (m >= 0) * alive).sum())
+    alive = ~dead[:, 1:] & ~dead[:, -1:]                             # an empty later stage: nothing to complete
+    useful = int(((m + 1) * (m + 2) // 2 * (m >= 0) * ~dead[:, 1:]).sum())
+    m2 = (t_max - first[:, 1:] - prefix[:, 1:])
+    needed = int(((m2 + 1) * (m2 + 2) // 2 * (m2 >= 0) * alive).sum())
     R, nhg, extra = packed_launch_shape(W, tile)
     n_tiles = nhg * 16
     Tc = n_tiles * R
@@ -316,11 +323,13 @@ def cell_update_counts(torch, wl, tables, tile: int = 0):
     q_lo = (first[:, 1:] // R) & ~1
     q_shift = ((prefix[:, 1:] // R) + n_dummy) & ~1
     ends = torch.arange(nhg, device=G.device).long() * 16 + 15       # tile | 15 of every half-group
+    used = torch.where(t_max < 0, torch.zeros_like(t_max), ((n_dummy + t_max.clamp(min=0) // R) // 16 + 1).clamp(max=nhg))
+    in_use = torch.arange(nhg, device=G.device).view(1, 1, -1) < used.unsqueeze(2)
     steps = (ends.view(1, 1, -1) - q_shift.unsqueeze(2) - q_lo.unsqueeze(2) + 1).clamp(min=0)
-    steps = steps * alive.unsqueeze(2)
+    steps = steps * in_use * (~dead[:, 1:]).unsqueeze(2)
     executed = int(steps.sum()) * 16 * R * R
-    executed += int(alive.sum()) * sum(Tc + e + 1 for e in range(n_extra))
-    return {"nominal": N * wl.minplus_cells, "useful": useful, "executed": executed}
+    executed += int((alive & (t_max >= Tc)).sum()) * sum(Tc + e + 1 for e in range(n_extra))
+    return {"nominal": N * wl.minplus_cells, "useful": useful, "needed": needed, "executed": executed}
 
 
 def run_ours(args):
@@ -614,8 +623,9 @@ def run_ours(args):
             "frac_useful": main_r["achieved_tops"] / measured_peak * counts["useful"] / counts["nominal"],
             "frac_executed": main_r["achieved_tops"] / measured_peak * counts["executed"] / counts["nominal"],
             "cells_note": "nominal = (S-1)(T+1)(T+2)/2 per instance; useful = cells not unreachable by the stages' "
-                          "first reachable entries; executed = chunk steps the kernel performs x R x R (skips in "
-                          "chunk pairs, lanes run to their half-group's longest column)"})
+                          "first reachable entries; needed = useful cells at budgets the later stages can still "
+                          "complete; executed = chunk steps the kernel performs x R x R (skips in chunk pairs and "
+                          "half-groups, lanes run to their half-group's longest column)"})
     if other:
         o_packed = not packed
         o_r = dense_rooflines(wl, other, o_packed, probe)

@@ -68,7 +68,9 @@ extern "C" {
  *      cells per register), on costs relative to every stage's cheapest entry; the A
  *      rows then hold the prefix tables themselves, uint16
  *          F_s[t] - sum_{k<=s} min_l G_k[l]     (0x7FFF: unreachable or >= 32767),
- *      and the backtrack recovers the argmin along the optimal path only.  Instances
+ *      computed only for budgets that can still be completed, t <= T - (sum over the later
+ *      stages of their first non-empty bucket), and 0x7FFF above (such a state is part of
+ *      no solution); the backtrack recovers the argmin along the optimal path only.  Instances
  *      whose optimum lies 32767 or more above the sum of the stages' cheapest entries
  *      are redone by the 32-bit kernel in a second launch.
  *   THEMIS_KERNEL_WIDE32       dense recurrence on 32-bit keys; the A rows hold the

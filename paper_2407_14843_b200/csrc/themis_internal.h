@@ -46,10 +46,6 @@ struct Params {
     int32_t only_flagged;  // wide min-plus kernel: solve only instances flagged kFlagNeedsWide
     uint8_t warp_group[32];  // 32-bit min-plus kernel: tile group (32 tiles) owned by each warp
     int32_t n_half_groups;   // packed min-plus kernel: half-groups of 16 tiles
-    // packed min-plus kernel, half-groups of the block's half-warp slots: slot s < fold_pairs walks
-    // half-group fold_hi - s and then fold_lo + s; slots fold_pairs and fold_pairs + 1 walk the
-    // single half-groups fold_single[0], fold_single[1] (-1 = none); later slots are idle
-    int32_t fold_pairs, fold_lo, fold_hi, fold_single[2];
     const int32_t *lat_us;
     const int32_t *profile_id;
     const uint32_t *lambda_mrps;

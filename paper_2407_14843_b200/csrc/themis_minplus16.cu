@@ -33,10 +33,15 @@
 // and then a short one, paired so that the two half-warps of every warp carry equal sums
 // (a warp runs as long as its longer half): (last, first), (last-1, second), ... when the
 // number of half-groups is a multiple of four; otherwise the one or two shortest, or the
-// longest, stand alone and the rest is paired the same way (assign_half_groups).  The two
+// longest, stand alone and the rest is paired the same way (deal_half_groups).  The two
 // halves of a warp may stand at different l (two broadcast addresses instead of one).  A
 // finished tile's result waits in registers for the stage's barrier; only the word that
 // spills into the next tile goes through shared memory.
+//
+// Budget limit.  A state of stages 0..s can only be completed if the fastest candidates of
+// the later stages still fit, so stage s computes budgets up to T minus the sum of the
+// later stages' first non-empty buckets only; the half-groups above that limit are not
+// walked (they are the longest columns) and the remaining ones are dealt anew every stage.
 //
 // Saturation.  If the best total is 0x7FFF the instance is either infeasible
 // (decided exactly: the fastest configurations of all stages do not fit the
@@ -69,9 +74,7 @@ __device__ __forceinline__ uint32_t block_min(uint32_t v, uint32_t *red, int tid
 }
 
 // EXTRA: the block also computes up to kMaxExtra cells beyond its tiles (see kMaxExtra).
-// PAIRS_ONLY: the number of half-groups is a multiple of four, every half-warp slot walks the pair
-// (last - slot, slot); otherwise the slots are described by the fold_* fields of Params.
-template <int R, int MAXT, bool EXTRA, bool PAIRS_ONLY>
+template <int R, int MAXT, bool EXTRA>
 __global__ void __launch_bounds__(MAXT, (R == 16 || MAXT > 512) ? 1 : 2)   // 64 registers: two blocks of 512
 minplus16_kernel(const Params p)
 {
@@ -103,22 +106,35 @@ minplus16_kernel(const Params p)
     uint32_t *fx_prev = stage_lmin + THEMIS_MAX_STAGES;       // kMaxExtra words: F_{s-1} at the extra cells
     uint32_t *fx_acc = fx_prev + kMaxExtra;                   // kMaxExtra words: F_s at the extra cells, building
     uint32_t *stage_cmin = fx_acc + kMaxExtra;                // 64 words: cheapest entry of every G_s
+    uint32_t *later_first = stage_cmin + THEMIS_MAX_STAGES;   // 64 words: sum over the later stages of their
+                                                              // first non-empty bucket (T + 1 if a stage is empty)
 
-    // The two tiles of this thread: its half-warp takes one half-group (long columns) and then
-    // another (short columns), as dealt by the host (assign_half_groups); either may be absent.
+    // The two tiles of this thread in the stage in hand: its half-warp takes one half-group
+    // (long columns) and then another (short columns); either may be absent.  Only the budgets
+    // a stage can still complete are computed (see budget_limit below), so the half-groups in
+    // use, and with them the pairing, change from stage to stage (deal_half_groups).
     const int slot = tid >> 4, lane16 = tid & 15;
-    int hg_a, hg_b;
-    bool has_a, has_b;
-    if (PAIRS_ONLY) {
-        hg_a = NHG - 1 - slot; hg_b = slot;
-        has_a = hg_a >= hg_b; has_b = hg_b < hg_a;
-    } else {
-        has_b = slot < p.fold_pairs;
-        hg_a = has_b ? p.fold_hi - slot : slot - p.fold_pairs < 2 ? p.fold_single[slot - p.fold_pairs] : -1;
-        hg_b = p.fold_lo + slot;
+    bool has_a = false, has_b = false;
+    int tile_a = 0, tile_b = 0;
+    // Deals the first `nhg` half-groups (half-group g costs g + 1 units) to the block's half-warp
+    // slots, at most two each, so that the sum over warps of the longer of a warp's two halves is
+    // smallest: pair longest with shortest, after setting aside the shortest (count = 1 mod 4),
+    // the two shortest (2 mod 4) or the longest (3 mod 4) as slots of their own behind the pairs
+    // (their sums are equal to the pairs' or below), so that the two halves of a warp are equal or
+    // nearly so.  Found optimal by exhaustive search for up to 13 half-groups and within half a
+    // unit of the ideal (half the total) beyond.
+    auto deal_half_groups = [&](int nhg) {
+        int lo = 0, hi = nhg - 1, single0 = -1, single1 = -1;
+        if ((nhg & 3) == 1) single0 = lo++;
+        if ((nhg & 3) == 2) { single1 = lo++; single0 = lo++; }   // the longer of the two first
+        if ((nhg & 3) == 3) single0 = hi--;
+        const int pairs = (hi - lo + 1) / 2;
+        has_b = slot < pairs;
+        const int hg_a = has_b ? hi - slot : slot == pairs ? single0 : slot == pairs + 1 ? single1 : -1;
         has_a = hg_a >= 0;
-    }
-    const int tile_a = hg_a * 16 + lane16, tile_b = hg_b * 16 + lane16;
+        tile_a = hg_a * 16 + lane16;
+        tile_b = (lo + slot) * 16 + lane16;
+    };
     const uint32_t row_bytes = (uint32_t)pitch * 4u;
     const int32_t *G_inst = p.G + (size_t)n * S * pitch;
     uint16_t *F16_inst = p.A + (size_t)n * S * pitch;     // prefix tables F_s as uint16 rows
@@ -142,11 +158,10 @@ minplus16_kernel(const Params p)
         mbar_init(&mbar[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int i = tid; i < kPadChunks * CS; i += NT) Fw[i] = kInf16x2;
-    for (int i = tid; i < THEMIS_MAX_STAGES; i += NT) {
-        stage_lmin[i] = 0xFFFFFFFFu;
-        stage_cmin[i] = 0xFFFFFFFFu;
-    }
+    // every half-word of F stays at or below kInf16 from here on (tiles a stage does not use keep
+    // an older, equally harmless value), so sums with an "unreachable" G never wrap
+    for (int i = tid; i < (kPadChunks + n_tiles) * CS; i += NT) Fw[i] = kInf16x2;
+    for (int i = tid; i < THEMIS_MAX_STAGES; i += NT) stage_cmin[i] = 0xFFFFFFFFu;
     for (int l = pitch + tid; l < Tp; l += NT) {
         Gbuf0[l] = kInf16x2;
         Gbuf1[l] = kInf16x2;
@@ -163,6 +178,55 @@ minplus16_kernel(const Params p)
     }
     int failed = 0;                                       // a bounded wait ran out
     int pend0 = 0, pend1 = S > 1 ? 0 : -1;                // phase parity of a copy in flight, or -1
+
+    // Budget limit.  A state of stages 0..s with budget t can only be completed if the fastest
+    // candidates of the later stages still fit: t <= T - sum over later stages of their first
+    // non-empty bucket.  Budgets above that limit are never part of a solution and are not
+    // computed: the uint16 table holds kInf16 there.  The first non-empty buckets are read from
+    // the table in global memory (the rows reach shared memory one at a time), a warp per row,
+    // while the first two rows are on their way.
+    for (int s = tid >> 5; s < S; s += n_warps) {
+        const int32_t *row = G_inst + (size_t)s * pitch;
+        uint32_t first = (uint32_t)T + 1u;
+        for (int base = 0; base <= T; base += 32) {
+            const int l = base + (tid & 31);
+            const unsigned hit = __ballot_sync(0xFFFFFFFFu, l <= T && row[l] != THEMIS_G_INF);
+            if (hit) { first = (uint32_t)(base + __ffs((int)hit) - 1); break; }
+        }
+        if ((tid & 31) == 0) {
+            later_first[s] = first;
+            stage_lmin[s] = first > (uint32_t)T ? 0xFFFFFFFFu : first;   // also the bound the stage skips by
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        uint32_t later = 0;
+        for (int s = S - 1; s >= 0; --s) {
+            const uint32_t own = later_first[s];
+            later_first[s] = later;
+            later = min(later + own, (uint32_t)T + 1u);
+        }
+    }
+    __syncthreads();
+    auto budget_limit = [&](int s) -> int { return T - (int)later_first[s]; };          // -1: nothing
+    auto half_groups_in_use = [&](int t_max) -> int { return t_max < 0 ? 0 : min(NHG, (n_dummy + t_max / R) / 16 + 1); };
+    // "unreachable" for the cells of row s of the uint16 table that no tile in use covers
+    auto blank_unused = [&](int s, int nhg_used) {
+        const int t_first = max(0, (nhg_used * 16 - n_dummy) * R);
+        uint32_t *row = reinterpret_cast<uint32_t *>(F16_inst + (size_t)s * pitch);
+        for (int w = t_first / 2 + tid; w < pitch / 2; w += NT) row[w] = kInf16x2;
+    };
+    // "unreachable" for the cells of a tile above the budget limit (only the last tiles in use reach it)
+    auto mask_above = [&](uint32_t (&w)[H], int tile, int t_max) {
+        const int t0 = (tile - n_dummy) * R;
+        if (t0 + R - 1 > t_max) {
+#pragma unroll
+            for (int r = 0; r < H; ++r) {
+                if (t0 + 2 * r > t_max) w[r] = kInf16x2;
+                else if (t0 + 2 * r + 1 > t_max) w[r] = (w[r] & 0xFFFFu) | (kInf16 << 16);
+            }
+        }
+    };
 
     // Stores a tile's H words of F_s to shared memory and to the uint16 table.
     auto store_chunk = [&](int tile, const uint32_t (&w)[H], int s) {
@@ -201,13 +265,11 @@ minplus16_kernel(const Params p)
     __syncthreads();
     const uint32_t c_off0 = row_cmin(0);
     cost_offset += c_off0;
-    // Records the lowest reachable index among this thread's R entries of row s.
-    auto note_first_reachable = [&](uint32_t first, int s) {
-        first = __reduce_min_sync(0xFFFFFFFFu, first);
-        if ((tid & 31) == 0 && first != 0xFFFFFFFFu) atomicMin(&stage_lmin[s], first);
-    };
     {
-        uint32_t first = 0xFFFFFFFFu;
+        const int t_max = budget_limit(0);
+        const int nhg_used = half_groups_in_use(t_max);
+        deal_half_groups(nhg_used);
+        blank_unused(0, nhg_used);
         auto init_tile = [&](int tile) {
             const int t0 = (tile - n_dummy) * R;
             uint32_t w[H];
@@ -217,16 +279,14 @@ minplus16_kernel(const Params p)
                 const uint32_t lo = t0 < 0 ? kInf16 : min(Gbuf0[t0 + 2 * r] - c_off0, kInf16);
                 const uint32_t hi = t0 < 0 ? kInf16 : min(Gbuf0[t0 + 2 * r + 1] - c_off0, kInf16);
                 w[r] = lo | (hi << 16);
-                if (hi < kInf16) first = min(first, (uint32_t)(t0 + 2 * r + 1));
-                if (lo < kInf16) first = min(first, (uint32_t)(t0 + 2 * r));
             }
+            mask_above(w, tile, t_max);
             store_chunk(tile, w, 0);
         };
         if (has_a) init_tile(tile_a);
         if (has_b) init_tile(tile_b);
-        note_first_reachable(first, 0);
         if (tid < n_extra) {
-            const uint32_t v = min(Gbuf0[Tc + tid] - c_off0, kInf16);
+            const uint32_t v = Tc + tid <= t_max ? min(Gbuf0[Tc + tid] - c_off0, kInf16) : kInf16;
             fx_prev[tid] = v;
             F16_inst[Tc + tid] = (uint16_t)v;
         }
@@ -237,8 +297,9 @@ minplus16_kernel(const Params p)
         const uint32_t w = Fw[(kPadChunks + n_dummy + i / R) * CS + ((i % R) >> 1)];
         return (i & 1) ? (w >> 16) : (w & 0xFFFFu);
     };
-    // Lowest reachable budget of the prefix F_{s-1} (0xFFFFFFFF: nothing reachable).  Everything
-    // below it, and every G_s[l] below that row's first reachable l, can only give "unreachable".
+    // Lowest budget the prefix F_{s-1} can reach: the sum of the earlier rows' first non-empty
+    // buckets (0xFFFFFFFF: nothing reachable).  Everything below it, and every G_s[l] below that
+    // row's first non-empty bucket, can only give "unreachable".
     uint32_t prefix_min = stage_lmin[0];
 
     // `failed` is block-uniform here and after every __syncthreads_or below; between those it is
@@ -252,19 +313,16 @@ minplus16_kernel(const Params p)
         const uint32_t c_off = row_cmin(s);
         cost_offset += c_off;
         {
-            uint32_t first = 0xFFFFFFFFu;
             for (int l4 = tid * 4; l4 < pitch; l4 += NT * 4) {
                 uint4 v4 = *reinterpret_cast<const uint4 *>(Gk + l4);
                 uint32_t *v = reinterpret_cast<uint32_t *>(&v4);
 #pragma unroll
-                for (int i = 3; i >= 0; --i) {
+                for (int i = 0; i < 4; ++i) {
                     const uint32_t c = min(v[i] - c_off, kInf16);
-                    v[i] = c | (c << 16);
-                    if (c < kInf16) first = min(first, (uint32_t)(l4 + i));
+                    v[i] = c * 0x10001u;
                 }
                 *reinterpret_cast<uint4 *>(Gk + l4) = v4;
             }
-            note_first_reachable(first, s);
             if (EXTRA && tid < kMaxExtra) fx_acc[tid] = 0xFFFFFFFFu;
         }
         failed = __syncthreads_or(failed);                // G_s and F_{s-1} visible to all
@@ -279,6 +337,11 @@ minplus16_kernel(const Params p)
             if (nxt) pend1 = ((s + 1) >> 1) & 1; else pend0 = ((s + 1) >> 1) & 1;
         }
 
+        const int t_max = budget_limit(s);
+        const int nhg_used = half_groups_in_use(t_max);
+        deal_half_groups(nhg_used);                       // this stage's tiles: budgets up to the limit only
+        blank_unused(s, nhg_used);
+        const bool extra_in_use = EXTRA && n_extra > 0 && Tc <= t_max;
         uint32_t acc[H], accp[H], wa[H], wb[H];
         // All lanes of a half-warp walk the same l so that G is a broadcast; lanes that run
         // past their own range read the "unreachable" chunks in front of F[0].  Chunks of
@@ -347,8 +410,8 @@ minplus16_kernel(const Params p)
             }
         }
         prefix_min = dead ? 0xFFFFFFFFu : prefix_min + g_min;
-        if (EXTRA && n_extra > 0) {
-            // Extra cells t = Tc + e: this thread's share of min_l F_{s-1}[t-l] + G_s[l] is its own
+        if (extra_in_use) {
+            // Extra cells t = Tc + e (every tile is in use then): this thread's share of min_l F_{s-1}[t-l] + G_s[l] is its own
             // tile's l range; thread 0 adds l >= Tc.
             uint32_t ex[kMaxExtra];
 #pragma unroll
@@ -393,12 +456,13 @@ minplus16_kernel(const Params p)
             w[0] = __vminu2(w[0], __byte_perm(left, 0xFFFFFFFFu, 0x5432));
 #pragma unroll
             for (int r = 0; r < H; ++r) w[r] = __vminu2(w[r], kInf16x2);
+            mask_above(w, tile, t_max);
             store_chunk(tile, w, s);
         };
         if (has_a) finish_tile(res_a, tile_a);
         if (has_b) finish_tile(res_b, tile_b);
         if (tid < n_extra) {                              // every share arrived before the barrier above
-            const uint32_t v = min(fx_acc[tid], kInf16);
+            const uint32_t v = extra_in_use && Tc + tid <= t_max ? min(fx_acc[tid], kInf16) : kInf16;
             fx_prev[tid] = v;
             F16_inst[(size_t)s * pitch + Tc + tid] = (uint16_t)v;
         }
@@ -548,13 +612,10 @@ minplus16_kernel(const Params p)
 template <int R, int MAXT, bool EXTRA>
 cudaError_t launch_variant16x(const Params &p, int threads, size_t smem, cudaStream_t stream)
 {
-    auto kernel = (p.n_half_groups & 3) == 0 ? minplus16_kernel<R, MAXT, EXTRA, true>
-                                             : minplus16_kernel<R, MAXT, EXTRA, false>;
-    static std::atomic<uint64_t> pairs_ready{0}, general_ready{0};
-    cudaError_t e = allow_max_smem(reinterpret_cast<const void *>(kernel),
-                                   (p.n_half_groups & 3) == 0 ? pairs_ready : general_ready);
+    static std::atomic<uint64_t> ready{0};
+    cudaError_t e = allow_max_smem(reinterpret_cast<const void *>(minplus16_kernel<R, MAXT, EXTRA>), ready);
     if (e != cudaSuccess) return e;
-    kernel<<<p.prob.n_instances, threads, smem, stream>>>(p);
+    minplus16_kernel<R, MAXT, EXTRA><<<p.prob.n_instances, threads, smem, stream>>>(p);
     return cudaGetLastError();
 }
 
@@ -587,28 +648,9 @@ Shape16 shape_of(int cells, int pitch, int tile)
     const int CS = sh.R == 16 ? 12 : sh.R / 2;
     const size_t g_words = (size_t)(n_tiles * sh.R > pitch ? n_tiles * sh.R : pitch);
     const size_t words = (size_t)(kPadChunks + n_tiles) * CS + 2u * g_words + (size_t)n_tiles + 4 + 32 +
-                         2 * THEMIS_MAX_STAGES + 2 * kMaxExtra;
+                         3 * THEMIS_MAX_STAGES + 2 * kMaxExtra;
     sh.smem = words * sizeof(uint32_t);
     return sh;
-}
-
-// Deals the half-groups (half-group g costs g + 1 units) to the block's half-warp slots, at most
-// two each, so that the sum over warps of the longer of a warp's two halves is smallest: pair
-// longest with shortest, after setting aside the shortest (count = 1 mod 4), the two shortest
-// (2 mod 4) or the longest (3 mod 4) as slots of their own behind the pairs (their sums are equal
-// to the pairs' or below), so that the two halves of a warp are equal or nearly so.  Found optimal
-// by exhaustive search for up to 13 half-groups and within half a unit of the ideal (half the
-// total) beyond.
-void assign_half_groups(int nhg, Params *p)
-{
-    int lo = 0, hi = nhg - 1;
-    p->fold_single[0] = p->fold_single[1] = -1;
-    if ((nhg & 3) == 1) p->fold_single[0] = lo++;
-    if ((nhg & 3) == 2) { p->fold_single[1] = lo++; p->fold_single[0] = lo++; }   // the longer of the two first
-    if ((nhg & 3) == 3) p->fold_single[0] = hi--;
-    p->fold_lo = lo;
-    p->fold_hi = hi;
-    p->fold_pairs = (hi - lo + 1) / 2;
 }
 
 template <int R, int MAXT>
@@ -616,7 +658,6 @@ cudaError_t launch_variant16(const Params &p_in, const Shape16 &sh, cudaStream_t
 {
     Params p = p_in;
     p.n_half_groups = sh.half_groups;
-    assign_half_groups(sh.half_groups, &p);
     return sh.extra ? launch_variant16x<R, MAXT, true>(p, sh.threads, sh.smem, stream)
                     : launch_variant16x<R, MAXT, false>(p, sh.threads, sh.smem, stream);
 }

@@ -78,7 +78,8 @@ def mode(request, S):
 def _assert_tables_equal(S, gpu, ref):
     """G, Garg everywhere; F (last prefix) where the instance is solved; then
     32-bit kernel: A where F_s[t] is reachable (0 elsewhere);
-    packed kernel: every prefix table F_s[t], saturated at 0x7FFF."""
+    packed kernel: every prefix table F_s[t], saturated at 0x7FFF, up to the budget the
+    later stages can still complete."""
     if MODE["mode"] >= 3:      # one fused kernel: the workspace holds fronts, not the dense tables
         return
     assert np.array_equal(gpu["G"], ref["G"])
@@ -95,6 +96,15 @@ def _assert_tables_equal(S, gpu, ref):
         cheapest[cheapest == S.G_INF] = 0
         rel = ref["F"].astype(np.int64) - np.cumsum(cheapest, axis=1)[:, :, None]
         rel[ref["F"] == S.G_INF] = S.INF16
+        # budgets the later stages cannot complete any more (their fastest candidates do not
+        # fit) are not computed: "unreachable" above T - sum of their first non-empty buckets
+        N_, S_, W1 = ref["G"].shape
+        nonempty = ref["G"] != S.G_INF
+        first = np.where(nonempty.any(axis=2), nonempty.argmax(axis=2), W1)
+        later = np.zeros((N_, S_), np.int64)
+        for s in range(S_ - 2, -1, -1):
+            later[:, s] = np.minimum(later[:, s + 1] + first[:, s + 1], W1)
+        rel[np.arange(W1)[None, None, :] > (W1 - 1 - later)[:, :, None]] = S.INF16
         assert np.array_equal(gpu["A"], rel.astype(np.uint16))
         return
     assert np.array_equal(gpu["F"], ref["F"][:, -1, :])
