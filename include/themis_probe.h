@@ -55,6 +55,24 @@ int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_s
 int themis_wait_probe(int32_t max_polls, const uint32_t *d_src16, uint32_t *d_dst16, int32_t *d_status,
                       void *cuda_stream);
 
+/*
+ * Report of the bounds-checked build (not part of the method; the paper has no
+ * counterpart).  Built with -DTHEMIS_CHECK_BOUNDS (python -m paper_2407_14843_b200.build
+ * --check-bounds writes libthemis_check.so), the solver kernels pass every index into
+ * shared or global memory that they compute through a range check; the first index found
+ * outside its range is recorded in the workspace (and clamped, so that nothing faults and
+ * the kernels run to their end), and every solve starts with a clear record.  This call
+ * waits for the stream and copies the record of the last solve on `d_workspace` to the
+ * host:
+ *   h_report[0]  site number of the first violation, 0 if there was none
+ *   h_report[1]  the offending index        h_report[2]  the limit it had to stay below
+ *   h_report[3]  1 if the library was built with the checks, else 0 (then the rest is 0)
+ * The normal build checks nothing and pays nothing.  Results of a checked solve equal
+ * those of the normal build as long as no violation is reported.
+ */
+int themis_bounds_check_report(const themis_problem_t *problem, int vertical, const void *d_workspace,
+                               size_t workspace_bytes, int32_t *h_report, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -2,6 +2,9 @@
 
 Run as ``python -m paper_2407_14843_b200.build`` or call ``build_library()``.
 The library is written next to this file; nvcc cross-compiles without a GPU.
+``--check-bounds`` (``build_library(check_bounds=True)``) writes a second library,
+``libthemis_check.so``, in which the solver kernels range-check every index they
+compute (see ``themis_bounds_check_report`` in ``include/themis_probe.h``).
 """
 from __future__ import annotations
 
@@ -13,6 +16,7 @@ import sys
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 LIB_PATH = os.path.join(_PKG, "libthemis.so")
+CHECK_LIB_PATH = os.path.join(_PKG, "libthemis_check.so")
 SOURCES = sorted(glob.glob(os.path.join(_PKG, "csrc", "*.cu")))
 HEADERS = sorted(glob.glob(os.path.join(_PKG, "csrc", "*.h")) + glob.glob(os.path.join(_PKG, "csrc", "*.cuh"))) + [os.path.join(_ROOT, "include", "themis.h")]
 
@@ -22,31 +26,32 @@ def _nvcc() -> str:
     return cand if os.path.exists(cand) else "nvcc"
 
 
-def is_stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+def is_stale(path: str = LIB_PATH) -> bool:
+    if not os.path.exists(path):
         return True
-    built = os.path.getmtime(LIB_PATH)
+    built = os.path.getmtime(path)
     return any(os.path.getmtime(f) > built for f in SOURCES + HEADERS)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    """Compile the library if a source is newer than it; returns its path."""
-    if not force and not is_stale():
-        return LIB_PATH
-    tmp = LIB_PATH + f".tmp{os.getpid()}"
+def build_library(force: bool = False, verbose: bool = False, check_bounds: bool = False) -> str:
+    """Compile the library (or its bounds-checked variant) if a source is newer than it;
+    returns its path."""
+    path = CHECK_LIB_PATH if check_bounds else LIB_PATH
+    if not force and not is_stale(path):
+        return path
+    tmp = path + f".tmp{os.getpid()}"
     cmd = [_nvcc(), "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-           "-Xcompiler", "-fPIC", "-shared", "-Xptxas", "-v",
+           "-Xcompiler", "-fPIC", "-Xcompiler", "-fno-gnu-unique", "-shared", "-Xptxas", "-v"] + (["-DTHEMIS_CHECK_BOUNDS", "-diag-suppress", "177"] if check_bounds else []) + [
            "-I", os.path.join(_ROOT, "include"), "-I", os.path.join(_PKG, "csrc"), "-o", tmp] + SOURCES
     proc = subprocess.run(cmd, capture_output=True, text=True)
     log = proc.stdout + proc.stderr
     if proc.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + log)
-    os.replace(tmp, LIB_PATH)
+    os.replace(tmp, path)
     if verbose:
         print(log)
-    return LIB_PATH
+    return path
 
 
 if __name__ == "__main__":
-    build_library(force="--force" in sys.argv, verbose=True)
-    print(LIB_PATH)
+    print(build_library(force="--force" in sys.argv, verbose=True, check_bounds="--check-bounds" in sys.argv))

@@ -93,6 +93,8 @@ int layout_of(const themis_problem_t *pr, int vertical, themis_workspace_layout_
     L->flag_offset = off; off = align_up(off + (size_t)pr->n_instances * sizeof(int32_t));
     // behind the tables: instances the sparse warp kernel hands to the block kernel (count, then ids)
     off = align_up(off + ((size_t)pr->n_instances + 1) * sizeof(int32_t));
+    // record of the bounds-checked build (four words)
+    off = align_up(off + 4 * sizeof(int32_t));
     L->total_bytes = off;
     L->row_pitch = (int32_t)pitch;
     L->T = T;
@@ -122,7 +124,14 @@ int make_params(const themis_problem_t *pr, const SolveOpts &opts, void *ws, siz
     P->inst_flag = reinterpret_cast<int32_t *>(base + L.flag_offset);
     P->redo_count = reinterpret_cast<int32_t *>(base + align_up(L.flag_offset + (size_t)pr->n_instances * sizeof(int32_t)));
     P->redo_list = P->redo_count + 1;
+    P->check = reinterpret_cast<int32_t *>(base + L.total_bytes - kAlign);
     return THEMIS_OK;
+}
+
+// Bounds-checked build: clears the violation record at the start of a solve.
+cudaError_t reset_check(const Params &P, cudaStream_t st)
+{
+    return kBoundsChecked ? cudaMemsetAsync(P.check, 0, 4 * sizeof(int32_t), st) : cudaSuccess;
 }
 
 bool result_ok(const themis_result_t &o)
@@ -139,7 +148,8 @@ int score_impl(const themis_problem_t *pr, const int32_t *lat, const int32_t *pi
     if (rc != THEMIS_OK) return rc;
     if (!lat || !lam || (vertical && !rep)) return THEMIS_E_INVALID_ARG;
     P.lat_us = lat; P.profile_id = pid; P.lambda_mrps = lam; P.replicas = rep;
-    cudaError_t e = launch_score(P, st);
+    cudaError_t e = reset_check(P, st);
+    if (e == cudaSuccess) e = launch_score(P, st);
     return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
 }
 
@@ -195,12 +205,14 @@ int solve_impl(const themis_problem_t *pr, const int32_t *lat, const int32_t *pi
             // one warp per instance on short sorted lists; what outgrows them is listed and
             // redone by the block kernel
             cudaError_t e = cudaMemsetAsync(P.redo_count, 0, sizeof(int32_t), st);
+            if (e == cudaSuccess) e = reset_check(P, st);
             if (e == cudaSuccess) e = launch_solve_front(P, st);
             if (e == cudaSuccess) e = launch_solve_sparse(P, /*only_listed=*/true, st);
             return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
         }
         if (block_fits) {
-            cudaError_t e = launch_solve_sparse(P, /*only_listed=*/false, st);
+            cudaError_t e = reset_check(P, st);
+            if (e == cudaSuccess) e = launch_solve_sparse(P, /*only_listed=*/false, st);
             return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
         }
     }
@@ -545,6 +557,24 @@ int themis_alu_probe(int mode, int blocks, int threads, int iters, uint32_t *d_s
     if (mode < 0 || mode > 5 || (mode == 5 && threads != 256) || blocks < 1 || threads < 32 || threads > 1024 || iters < 1 || !d_sink)
         return THEMIS_E_INVALID_ARG;
     cudaError_t e = launch_alu_probe(mode, blocks, threads, iters, d_sink, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
+}
+
+int themis_bounds_check_report(const themis_problem_t *problem, int vertical, const void *d_workspace,
+                               size_t workspace_bytes, int32_t *h_report, void *cuda_stream)
+{
+    themis_workspace_layout_t L;
+    int rc = layout_of(problem, vertical, &L);
+    if (rc != THEMIS_OK) return rc;
+    if (!d_workspace || !h_report) return THEMIS_E_INVALID_ARG;
+    if (workspace_bytes < L.total_bytes) return THEMIS_E_WORKSPACE_TOO_SMALL;
+    h_report[0] = h_report[1] = h_report[2] = 0;
+    h_report[3] = kBoundsChecked;
+    if (!kBoundsChecked) return THEMIS_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaMemcpyAsync(h_report, static_cast<const char *>(d_workspace) + L.total_bytes - kAlign,
+                                    3 * sizeof(int32_t), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     return e == cudaSuccess ? THEMIS_OK : fail_cuda(e);
 }
 

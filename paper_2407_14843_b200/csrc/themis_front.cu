@@ -176,8 +176,8 @@ stage_fronts_kernel(const Params p)
             const unsigned long long b = (unsigned long long)p.prob.batch_sizes[bi];
             const unsigned long long m = (p.prob.flags & THEMIS_QUEUE_PER_REPLICA) ? h : 1ull;
             const unsigned long long q_num = (b - 1ull) * m * 1000000000ull;
-            Q[e] = sat_u32((q_num + q_den - 1ull) / q_den, (uint32_t)T + 1u);
-            Lmax[e] = sat_u32(h * b * 1000000000ull / lambda_m, 0x7FFFFFFFu);
+            Q[TH_IDX(601, e, L.tab)] = sat_u32((q_num + q_den - 1ull) / q_den, (uint32_t)T + 1u);
+            Lmax[TH_IDX(602, e, L.tab)] = sat_u32(h * b * 1000000000ull / lambda_m, 0x7FFFFFFFu);
         }
         if (lane < NB) rate_b[lane] = (float)lambda_m / ((float)p.prob.batch_sizes[lane] * 1.0e9f);
     }
@@ -205,8 +205,8 @@ stage_fronts_kernel(const Params p)
             if (e < CB) {
                 const int c1 = NB > 1 ? (int)__umulhi((uint32_t)e, nb_magic) : e;
                 const int bi = e - c1 * NB;
-                const int32_t l_us = (int32_t)latb[e];
-                const int32_t l_prev = e >= NB ? (int32_t)latb[e - NB] : 0;   // one core fewer
+                const int32_t l_us = (int32_t)latb[TH_IDX(603, e, L.cb)];
+                const int32_t l_prev = e >= NB ? (int32_t)latb[TH_IDX(604, e - NB, L.cb)] : 0;   // one core fewer
                 if (l_us <= 0) saw_bad_latency = 1;
                 // ceil(l / w): the reciprocal's quotient is the true one or one below it
                 // (l < 2^31, so the error of l * floor((2^32 - 1) / w) / 2^32 stays below 1/2)
@@ -221,20 +221,20 @@ stage_fronts_kernel(const Params p)
                     if (HN > 1) {
                         // fewest replicas: about l * lambda / (b * 1e9); the estimate is taken one
                         // low and settled on the exact table, two steps up at most as a rule
-                        const float need = (float)l_us * rate_b[bi] - (float)h_lo;
+                        const float need = (float)l_us * rate_b[TH_IDX(605, bi, THEMIS_MAX_BATCH_SIZES)] - (float)h_lo;
                         k = min(max(__float2int_rz(need) - 1, 0), HN - 1);   // the conversion saturates
-                        k += (uint32_t)l_us > lmax_row[k];
+                        k += (uint32_t)l_us > lmax_row[TH_IDX(606, k, HN)];
                         k = min(k, HN - 1);
-                        k += (uint32_t)l_us > lmax_row[k];
-                        if (k > 0 && k < HN && (uint32_t)l_us <= lmax_row[k - 1]) k = 0;   // estimate too high
+                        k += (uint32_t)l_us > lmax_row[TH_IDX(607, k, HN)];
+                        if (k > 0 && k < HN && (uint32_t)l_us <= lmax_row[TH_IDX(608, k - 1, HN)]) k = 0;   // estimate too high
                     }
-                    while (k < HN && (uint32_t)l_us > lmax_row[k]) ++k;
+                    while (k < HN && (uint32_t)l_us > lmax_row[TH_IDX(609, k, HN)]) ++k;
                     if (k < HN) {                          // else no replica count sustains lambda
-                        const uint32_t ell = l_b + Q_s[bi * HN + k];
+                        const uint32_t ell = l_b + Q_s[TH_IDX(610, bi * HN + k, NB * HN)];
                         if (ell <= (uint32_t)T) {
                             key = (((uint32_t)(h_lo + k) * (uint32_t)(c1 + 1)) << kIdxBits) | ell;
                             idx = (uint32_t)(k * CB + e);
-                            atomicMin(&bins[(ell * bin_scale) >> 16], key);
+                            atomicMin(&bins[TH_IDX(611, (ell * bin_scale) >> 16, kBins)], key);
                         }
                     }
                 }
@@ -242,8 +242,8 @@ stage_fronts_kernel(const Params p)
             const unsigned live = __ballot_sync(0xFFFFFFFFu, key != kNone);
             if (key != kNone) {
                 const int at = n_live + __popc(live & lanemask_lt);
-                ckey[at] = key;
-                cidx[at] = (uint16_t)idx;
+                ckey[TH_IDX(612, at, L.cb)] = key;
+                cidx[TH_IDX(613, at, L.cb)] = (uint16_t)idx;
             }
             n_live += __popc(live);
         }
@@ -287,14 +287,14 @@ stage_fronts_kernel(const Params p)
         int n_sv = 0;
         for (int i0 = 0; i0 < n_live; i0 += 32) {
             const int i = i0 + lane;
-            const uint32_t key = i < n_live ? ckey[i] : kNone;
+            const uint32_t key = i < n_live ? ckey[TH_IDX(615, i, L.cb)] : kNone;
             const bool keep = key != kNone &&
-                              (key >> kIdxBits) < (bins[((key & kLowMask) * bin_scale) >> 16] >> kIdxBits);
+                              (key >> kIdxBits) < (bins[TH_IDX(614, ((key & kLowMask) * bin_scale) >> 16, kBins)] >> kIdxBits);
             const unsigned kept = __ballot_sync(0xFFFFFFFFu, keep);
             const int at = n_sv + __popc(kept & lanemask_lt);
             if (keep && at < kMaxSurvivors) {
-                skey[at] = key;
-                sidx[at] = cidx[i];
+                skey[TH_IDX(616, at, kMaxSurvivors)] = key;
+                sidx[TH_IDX(617, at, kMaxSurvivors)] = cidx[TH_IDX(618, i, L.cb)];
             }
             n_sv += __popc(kept);
         }
@@ -317,8 +317,8 @@ stage_fronts_kernel(const Params p)
                 const uint32_t idx = warp_min(min(k0 == m ? i0 : kNone, k1 == m ? i1 : kNone));
                 ++n_g;                                     // at most 64 survivors: the front fits its slots
                 if (lane == 0) {
-                    gf[kMaxStageFront - n_g] = m;
-                    gidx[kMaxStageFront - n_g] = idx;
+                    gf[TH_IDX(619, kMaxStageFront - n_g, kMaxStageFront)] = m;
+                    gidx[TH_IDX(620, kMaxStageFront - n_g, kMaxStageFront)] = idx;
                 }
                 bound = m & kLowMask;
             }
@@ -327,7 +327,7 @@ stage_fronts_kernel(const Params p)
             for (;;) {
                 uint32_t mine = kNone;
                 for (int i = lane; i < n_sv; i += 32) {
-                    const uint32_t key = skey[i];
+                    const uint32_t key = skey[TH_IDX(621, i, kMaxSurvivors)];
                     if ((key & kLowMask) < bound) mine = min(mine, key);
                 }
                 const uint32_t m = warp_min(mine);
@@ -339,8 +339,8 @@ stage_fronts_kernel(const Params p)
                 idx = warp_min(idx);
                 ++n_g;
                 if (lane == 0) {
-                    gf[kMaxStageFront - n_g] = m;
-                    gidx[kMaxStageFront - n_g] = idx;
+                    gf[TH_IDX(622, kMaxStageFront - n_g, kMaxStageFront)] = m;
+                    gidx[TH_IDX(623, kMaxStageFront - n_g, kMaxStageFront)] = idx;
                 }
                 bound = m & kLowMask;
             }
@@ -350,10 +350,11 @@ stage_fronts_kernel(const Params p)
         // 5. to the workspace, ascending latency
         const size_t row = ((size_t)n * S + s) * pitch;
         for (int k = lane; k < n_g; k += 32) {
-            reinterpret_cast<uint32_t *>(p.G)[row + k] = gf[kMaxStageFront - n_g + k];
-            p.Garg[row + k] = (uint16_t)gidx[kMaxStageFront - n_g + k];
+            reinterpret_cast<uint32_t *>(p.G)[TH_IDX(624, row + k, (size_t)p.prob.n_instances * S * pitch)] =
+                gf[TH_IDX(625, kMaxStageFront - n_g + k, kMaxStageFront)];
+            p.Garg[TH_IDX(626, row + k, (size_t)p.prob.n_instances * S * pitch)] = (uint16_t)gidx[kMaxStageFront - n_g + k];
         }
-        if (lane == 0) p.A[row] = (uint16_t)n_g;
+        if (lane == 0) p.A[TH_IDX(627, row, (size_t)p.prob.n_instances * S * pitch)] = (uint16_t)n_g;
         __syncwarp();
     }
     asm volatile("cp.async.wait_all;" ::: "memory");       // nothing of ours in flight when the warp leaves
@@ -361,7 +362,7 @@ stage_fronts_kernel(const Params p)
     if (redo) {                                            // lists outgrown: the block kernel solves it
         if (lane == 0) {
             p.inst_flag[n] = kFlagRedo;
-            p.redo_list[atomicAdd(p.redo_count, 1)] = n;
+            p.redo_list[TH_IDX(628, atomicAdd(p.redo_count, 1), p.prob.n_instances)] = n;
         }
         return;
     }
@@ -400,10 +401,16 @@ __host__ __device__ inline PrefixLayout prefix_layout(int T, int S)
 // empty, so budgets below zero need no test.
 struct BudgetRank {
     const uint2 *pairs;     // points at pair 0
+    int wb;                 // pairs 0 .. wb - 1 (and pair -1)
+    int32_t *check;         // violation record of the bounds-checked build
     // number of front entries with budget <= x, for any x >= -32
     __device__ __forceinline__ int upto(int x) const
     {
+#ifdef THEMIS_CHECK_BOUNDS
+        const uint2 pr = pairs[th_checked_index(701, (long long)(x >> 5) + 1, (long long)wb + 1, check) - 1];
+#else
         const uint2 pr = pairs[x >> 5];
+#endif
         return (int)pr.y + __popc(pr.x & (0xFFFFFFFFu >> (31 - (x & 31))));
     }
 };
@@ -416,18 +423,19 @@ struct BudgetRank {
 // candidate index), to rec (= g_row) from 0 up.  Returns the number of entries; *more is
 // set when the limit cut the front short.
 template <int NL>
-__device__ __forceinline__ int merge_fronts(const uint32_t *Fprev, const BudgetRank &rank, uint32_t *g_row,
-                                            const uint16_t *gidx_row, int n_g, uint32_t *Ftop, int bound,
-                                            uint32_t stop, int limit, int lane, bool *more)
+__device__ __forceinline__ int merge_fronts(const Params &p, const uint32_t *Fprev, int n_prev, const BudgetRank &rank,
+                                            uint32_t *g_row, const uint16_t *gidx_row, int n_g, uint32_t *Ftop,
+                                            int bound, uint32_t stop, int limit, int lane, bool *more)
 {
+    (void)p; (void)n_prev;
     uint32_t gk[NL], gix[NL], cur[NL];
     int lk[NL], pp[NL];                      // list q: its latency + 1; prefix entries it may still use
 #pragma unroll
     for (int q = 0; q < NL; ++q) {
         const int k = lane + 32 * q;
         const bool valid = k < n_g;
-        gk[q] = valid ? g_row[k] : 0u;
-        gix[q] = valid ? (uint32_t)gidx_row[k] : 0u;
+        gk[q] = valid ? g_row[TH_IDX(702, k, p.pitch)] : 0u;
+        gix[q] = valid ? (uint32_t)gidx_row[TH_IDX(703, k, p.pitch)] : 0u;
         lk[q] = valid ? (int)(gk[q] & kLowMask) + 1 : 0x20000000;   // no budget reaches an absent list
     }
     __syncwarp();                            // the stage front is in registers: its row may take records
@@ -438,7 +446,7 @@ __device__ __forceinline__ int merge_fronts(const uint32_t *Fprev, const BudgetR
     // bound reads the absent word in front of the prefix front.
     auto settle = [&](int q, int below) {
         pp[q] = rank.upto(max(below - lk[q], -1));
-        cur[q] = Fprev[pp[q] - 1] + gk[q];
+        cur[q] = Fprev[TH_IDX(704, pp[q], n_prev + 1) - 1] + gk[q];
     };
 #pragma unroll
     for (int q = 0; q < NL; ++q) settle(q, bound);
@@ -457,8 +465,8 @@ __device__ __forceinline__ int merge_fronts(const uint32_t *Fprev, const BudgetR
             const bool offer = cur[q] == m;
             const unsigned offers = __ballot_sync(0xFFFFFFFFu, offer);
             if (!found && offer && (offers & lanemask_lt) == 0u) {
-                Ftop[-1 - count] = m;
-                rec[count] = ((uint32_t)pp[q] << 16) | gix[q];
+                Ftop[-1 - TH_IDX(705, count, limit)] = m;
+                rec[TH_IDX(706, count, p.pitch)] = ((uint32_t)pp[q] << 16) | gix[q];
             }
             found = found || offers != 0u;
         }
@@ -538,7 +546,7 @@ prefix_fronts_kernel(const Params p)
     uint32_t *rec_inst = reinterpret_cast<uint32_t *>(p.G + (size_t)n * S * pitch);
     const uint16_t *gidx_inst = p.Garg + (size_t)n * S * pitch;
     const uint16_t *count_inst = p.A + (size_t)n * S * pitch;
-    const BudgetRank rank{pairs};
+    const BudgetRank rank{pairs, L.wb, p.check};
     int32_t *h_o = p.out.h + (size_t)n * S, *c_o = p.out.c + (size_t)n * S, *b_o = p.out.b + (size_t)n * S;
     auto write_infeasible = [&]() {
         for (int s = lane; s < S; s += 32) { h_o[s] = 0; c_o[s] = 0; b_o[s] = 0; }
@@ -564,7 +572,7 @@ prefix_fronts_kernel(const Params p)
                 if (count[q] == 0) any_empty = 1;
                 else {
                     lmin_sum += (int)(rec_inst[(size_t)s * pitch] & kLowMask);
-                    cheapest[q] = rec_inst[(size_t)s * pitch + count[q] - 1] >> kIdxBits;
+                    cheapest[q] = rec_inst[TH_IDX(707, (size_t)s * pitch + count[q] - 1, (size_t)S * pitch)] >> kIdxBits;
                 }
                 n_of[s] = (uint32_t)count[q];
             }
@@ -600,7 +608,7 @@ prefix_fronts_kernel(const Params p)
             const uint32_t *g_row = rec_inst + (size_t)s * pitch;
             for (int k = lane; k < (int)n_of[s]; k += 32) {
                 const uint32_t w = g_row[k];
-                sf[off[s] + k] = make_float2((float)(w & kLowMask), (float)(w >> kIdxBits));
+                sf[TH_IDX(708, off[s] + k, cap + 1)] = make_float2((float)(w & kLowMask), (float)(w >> kIdxBits));
             }
         }
         __syncwarp();
@@ -645,8 +653,8 @@ prefix_fronts_kernel(const Params p)
             for (int q = 0; q < kLists; ++q) {
                 const int k = lane + 32 * q - first;
                 if (k >= 0 && k < n_fit) {
-                    Fcur[cap - n_fit + k] = gk[q];
-                    g_row[n_fit - 1 - k] = gix[q];
+                    Fcur[TH_IDX(709, cap - n_fit + k, cap)] = gk[q];
+                    g_row[TH_IDX(710, n_fit - 1 - k, pitch)] = gix[q];
                 }
             }
             n_cur = n_fit;
@@ -655,9 +663,9 @@ prefix_fronts_kernel(const Params p)
             const int limit = s == S - 1 ? 1 : cap;
             uint32_t *Ftop = Fcur + cap;
             const uint32_t *Fp = Fprev + (cap - n_prev);
-            n_cur = n_g <= 32 ? merge_fronts<1>(Fp, rank, g_row, gidx_row, n_g, Ftop, bound, stop, limit, lane, &more)
-                  : n_g <= 64 ? merge_fronts<2>(Fp, rank, g_row, gidx_row, n_g, Ftop, bound, stop, limit, lane, &more)
-                              : merge_fronts<kMaxStageFront / 32>(Fp, rank, g_row, gidx_row, n_g, Ftop, bound, stop,
+            n_cur = n_g <= 32 ? merge_fronts<1>(p, Fp, n_prev, rank, g_row, gidx_row, n_g, Ftop, bound, stop, limit, lane, &more)
+                  : n_g <= 64 ? merge_fronts<2>(p, Fp, n_prev, rank, g_row, gidx_row, n_g, Ftop, bound, stop, limit, lane, &more)
+                              : merge_fronts<kMaxStageFront / 32>(p, Fp, n_prev, rank, g_row, gidx_row, n_g, Ftop, bound, stop,
                                                                   limit, lane, &more);
             if (more && s < S - 1) { redo = true; break; }
         }
@@ -669,12 +677,12 @@ prefix_fronts_kernel(const Params p)
 
         // bitmap of the new front's budgets and the running counts, for the next stage
         if (s + 1 < S) {
-            if (lane == 0) { Fprev[cap - n_prev - 1] = kAbsent; pairs[-1] = make_uint2(0u, 0u); }
+            if (lane == 0) { Fprev[TH_IDX(711, cap - n_prev, cap + 1) - 1] = kAbsent; pairs[-1] = make_uint2(0u, 0u); }
             for (int w = lane; w < L.wb; w += 32) pairs[w].x = 0u;
             __syncwarp();
             for (int i = lane; i < n_prev; i += 32) {
-                const uint32_t t = Fprev[cap - n_prev + i] & kLowMask;
-                atomicOr(&pairs[t >> 5].x, 1u << (t & 31));
+                const uint32_t t = Fprev[TH_IDX(712, cap - n_prev + i, cap)] & kLowMask;
+                atomicOr(&pairs[TH_IDX(713, t >> 5, L.wb)].x, 1u << (t & 31));
             }
             __syncwarp();
             uint32_t carry = 0;
@@ -697,7 +705,7 @@ prefix_fronts_kernel(const Params p)
     if (redo) {                                            // front outgrown: the block kernel solves it
         if (lane == 0) {
             p.inst_flag[n] = kFlagRedo;
-            p.redo_list[atomicAdd(p.redo_count, 1)] = n;
+            p.redo_list[TH_IDX(716, atomicAdd(p.redo_count, 1), p.prob.n_instances)] = n;
         }
         return;
     }
@@ -711,8 +719,8 @@ prefix_fronts_kernel(const Params p)
     if (lane == 0) {
         uint32_t q = 0;
         for (int s = S - 1; s >= 0; --s) {
-            const uint32_t r = rec_inst[(size_t)s * pitch + q];
-            idx_of[s] = r & 0xFFFFu;
+            const uint32_t r = rec_inst[TH_IDX(714, (size_t)s * pitch + q, (size_t)S * pitch)];
+            idx_of[TH_IDX(715, s, THEMIS_MAX_STAGES)] = r & 0xFFFFu;
             if (s > 0) q = n_of[s - 1] - (r >> 16);
         }
         p.out.total_cost[n] = (int32_t)(best >> kIdxBits);

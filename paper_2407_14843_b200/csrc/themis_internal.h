@@ -55,6 +55,7 @@ struct Params {
     uint16_t *Garg;
     uint16_t *A;
     int32_t *F;
+    int32_t *check;      // bounds-checked build: {site of the first violation (0 = none), index, limit, 0}
     int32_t *redo_count; // sparse warp kernel: number of instances handed to the block kernel ...
     int32_t *redo_list;  // ... and their indices [N]
     int32_t *inst_flag;  // [N] kFlagBadInput: bad input seen by the scoring kernel; kFlagNeedsWide: see above
@@ -95,6 +96,35 @@ inline cudaError_t allow_max_smem(const void *kernel, std::atomic<uint64_t> &don
     if (e == cudaSuccess) done.fetch_or(bit, std::memory_order_release);
     return e;
 }
+
+// Bounds-checked build (-DTHEMIS_CHECK_BOUNDS; stands in for a memory sanitizer).  Every index
+// into shared or global memory that a kernel computes goes through TH_IDX(site, index, limit):
+// an index outside [0, limit) is recorded once in Params::check (site number, index, limit)
+// and clamped into range, so the access itself stays legal, the kernel runs to its end and the
+// host reads the record (themis_bounds_check_report).  Nothing traps.  Site numbers: 1xx
+// scoring, 2xx packed recurrence, 3xx 32-bit recurrence, 4xx pruned recurrence, 5xx sparse
+// block kernel, 6xx stage fronts, 7xx prefix fronts.  In the normal build TH_IDX is its index.
+#ifdef THEMIS_CHECK_BOUNDS
+#ifdef __CUDACC__
+__device__ __forceinline__ int th_checked_index(int site, long long i, long long n, int32_t *check)
+{
+    if (i >= 0 && i < n) return (int)i;
+    if (atomicCAS(&check[0], 0, site) == 0) {
+        check[1] = (int)i;
+        check[2] = (int)n;
+    }
+    return i < 0 || n < 1 ? 0 : (int)(n - 1);
+}
+#endif
+#define TH_IDX(site, i, n) th_checked_index((site), (long long)(i), (long long)(n), p.check)
+// a pointer that must stay within [base, base + n)
+#define TH_PTR(site, ptr, base, n) ((base) + TH_IDX(site, (ptr) - (base), n))
+constexpr int kBoundsChecked = 1;
+#else
+#define TH_IDX(site, i, n) (i)
+#define TH_PTR(site, ptr, base, n) (ptr)
+constexpr int kBoundsChecked = 0;
+#endif
 
 cudaError_t launch_score(const Params &p, cudaStream_t stream);
 cudaError_t launch_minplus(const Params &p, int tile, cudaStream_t stream);

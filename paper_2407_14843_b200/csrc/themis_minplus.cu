@@ -84,7 +84,9 @@ minplus_kernel(const Params p)
 
     const int tile = ((int)p.warp_group[tid >> 5] << 5) | (tid & 31);                   // groups dealt by assign_warp_groups
     const int t0 = tile * R;
-    uint32_t *my_chunk = Fs + (tile + 1) * CS;
+    const int f_words = (NT + 1) * CS;                  // words of F in shared memory
+    (void)f_words;
+    uint32_t *my_chunk = Fs + TH_IDX(301, tile + 1, NT + 1) * CS;
     const uint32_t row_bytes = (uint32_t)pitch * 4u;
     const int32_t *G_inst = p.G + (size_t)n * S * pitch;
 
@@ -97,7 +99,7 @@ minplus_kernel(const Params p)
         p.out.status[n] = status;
     };
     if (p.only_flagged) {                               // second pass: only what the packed kernel left over
-        if (p.inst_flag[n] != kFlagNeedsWide) return;
+        if (p.inst_flag[TH_IDX(302, n, p.prob.n_instances)] != kFlagNeedsWide) return;
     } else if (p.inst_flag[n] == kFlagBadInput) {       // bad input seen while scoring
         if (tid == 0) write_unsolved(THEMIS_STATUS_BAD_INPUT);
         return;
@@ -111,8 +113,8 @@ minplus_kernel(const Params p)
     // "unreachable" in front of F[0], and behind the loaded part of each G buffer
     if (tid < CS) Fs[tid] = kInfKey;
     for (int l = pitch + tid; l < Tp; l += NT) {
-        Gbuf0[l] = kInfKey | (uint32_t)l;
-        Gbuf1[l] = kInfKey | (uint32_t)l;
+        Gbuf0[TH_IDX(303, l, Tp)] = kInfKey | (uint32_t)l;
+        Gbuf1[TH_IDX(304, l, Tp)] = kInfKey | (uint32_t)l;
     }
     __syncthreads();
     if (tid == 0) {
@@ -131,7 +133,7 @@ minplus_kernel(const Params p)
     if (!mbar_wait(&mbar[0], 0)) failed = 1; else pend0 = -1;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        const uint32_t raw = Gbuf0[t0 + r];              // raw cost, or >= kInfCost when empty/padding
+        const uint32_t raw = Gbuf0[TH_IDX(305, t0 + r, Tp)];   // raw cost, or >= kInfCost when empty/padding
         my_chunk[r] = min(raw, kInfCost) << kIdxBits;
     }
     failed = __syncthreads_or(failed);
@@ -146,8 +148,8 @@ minplus_kernel(const Params p)
         if (t0 < pitch) {
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                const uint32_t raw = Gk[t0 + r];
-                Gk[t0 + r] = (min(raw, kInfCost) << kIdxBits) | (uint32_t)(t0 + r);
+                const uint32_t raw = Gk[TH_IDX(306, t0 + r, Tp)];
+                Gk[TH_IDX(307, t0 + r, Tp)] = (min(raw, kInfCost) << kIdxBits) | (uint32_t)(t0 + r);
             }
         }
         failed = __syncthreads_or(failed);               // keys and F_{s-1} visible to all
@@ -171,8 +173,9 @@ minplus_kernel(const Params p)
         int f_off = tile * CS;                           // word offset of chunk tile-1
         const uint32_t *g = Gk;
         for (int q = 0; q <= q_end; q += 2) {
-            chunk_step<R>(wa, wb, acc, Fs + max(f_off, 0), g);
-            chunk_step<R>(wb, wa, acc, Fs + max(f_off - CS, 0), g + R);
+            chunk_step<R>(wa, wb, acc, Fs + TH_IDX(308, max(f_off, 0), f_words - R + 1), TH_PTR(309, g, Gk, Tp - R + 1));
+            chunk_step<R>(wb, wa, acc, Fs + TH_IDX(310, max(f_off - CS, 0), f_words - R + 1),
+                          TH_PTR(311, g + R, Gk, Tp - R + 1));
             f_off -= 2 * CS;
             g += 2 * R;
         }
@@ -186,7 +189,7 @@ minplus_kernel(const Params p)
             a16[r] = inf ? 0u : (acc[r] & kIdxMask);
         }
         if (t0 + R <= pitch) {
-            uint16_t *A_row = p.A + ((size_t)n * S + s) * pitch + t0;
+            uint16_t *A_row = p.A + TH_IDX(312, ((size_t)n * S + s) * pitch + t0, (size_t)p.prob.n_instances * S * pitch - R + 1);
 #pragma unroll
             for (int v = 0; v < R / 8; ++v) {
                 uint4 o;
@@ -217,10 +220,10 @@ minplus_kernel(const Params p)
         const int t = t0 + r;
         const uint32_t fk = my_chunk[r];
         if (t <= T) best = min(best, fk | (uint32_t)t);
-        if (t < pitch) F_row[t] = fk >= kInfKey ? THEMIS_G_INF : (int32_t)(fk >> kIdxBits);
+        if (t < pitch) F_row[TH_IDX(313, t, pitch)] = fk >= kInfKey ? THEMIS_G_INF : (int32_t)(fk >> kIdxBits);
     }
     best = __reduce_min_sync(0xFFFFFFFFu, best);
-    if ((tid & 31) == 0) red[tid >> 5] = best;
+    if ((tid & 31) == 0) red[TH_IDX(314, tid >> 5, 32)] = best;
     __syncthreads();                                     // also orders this block's A stores
     if (tid == 0) {
         for (int w = 1; w < (NT >> 5); ++w) best = min(best, red[w]);
@@ -232,10 +235,10 @@ minplus_kernel(const Params p)
             const int C = p.prob.c_max, NB = p.prob.n_batch;
             for (int s = S - 1; s >= 0; --s) {
                 const size_t row = ((size_t)n * S + s) * pitch;
-                const int ell = s > 0 ? (int)p.A[row + t] : t;
-                const int idx = (int)p.Garg[row + ell];
+                const int ell = s > 0 ? (int)p.A[TH_IDX(315, row + t, (size_t)p.prob.n_instances * S * pitch)] : t;
+                const int idx = (int)p.Garg[TH_IDX(316, row + ell, (size_t)p.prob.n_instances * S * pitch)];
                 const int bi = idx % NB, rest = idx / NB;
-                b_o[s] = p.prob.batch_sizes[bi];
+                b_o[s] = p.prob.batch_sizes[TH_IDX(317, bi, THEMIS_MAX_BATCH_SIZES)];
                 c_o[s] = rest % C + 1;
                 h_o[s] = p.vertical ? p.replicas[(size_t)n * S + s]
                        : p.horizontal ? G_inst[(size_t)s * pitch + ell] : rest / C + 1;

@@ -138,16 +138,18 @@ minplus16_kernel(const Params p)
     const uint32_t row_bytes = (uint32_t)pitch * 4u;
     const int32_t *G_inst = p.G + (size_t)n * S * pitch;
     uint16_t *F16_inst = p.A + (size_t)n * S * pitch;     // prefix tables F_s as uint16 rows
-    auto chunk_of = [&](int tile) -> uint32_t * { return Fw + (kPadChunks + tile) * CS; };
+    const int f_words = (kPadChunks + n_tiles) * CS;      // words of F in shared memory
+    (void)f_words;
+    auto chunk_of = [&](int tile) -> uint32_t * { return Fw + TH_IDX(201, kPadChunks + tile, kPadChunks + n_tiles) * CS; };
 
     int32_t *h_o = p.out.h + (size_t)n * S, *c_o = p.out.c + (size_t)n * S, *b_o = p.out.b + (size_t)n * S;
     auto write_unsolved = [&](int status) {
         for (int s = 0; s < S; ++s) { h_o[s] = 0; c_o[s] = 0; b_o[s] = 0; }
-        p.out.total_cost[n] = -1;
+        p.out.total_cost[TH_IDX(202, n, p.prob.n_instances)] = -1;
         p.out.latency_buckets[n] = -1;
         p.out.status[n] = status;
     };
-    if (p.inst_flag[n] == kFlagBadInput) {                // bad input seen while scoring (a leftover
+    if (p.inst_flag[TH_IDX(203, n, p.prob.n_instances)] == kFlagBadInput) {   // bad input seen while scoring (a leftover
                                                           // kFlagNeedsWide of an earlier pass is re-decided below)
         if (tid == 0) write_unsolved(THEMIS_STATUS_BAD_INPUT);
         return;
@@ -163,8 +165,8 @@ minplus16_kernel(const Params p)
     for (int i = tid; i < (kPadChunks + n_tiles) * CS; i += NT) Fw[i] = kInf16x2;
     for (int i = tid; i < THEMIS_MAX_STAGES; i += NT) stage_cmin[i] = 0xFFFFFFFFu;
     for (int l = pitch + tid; l < Tp; l += NT) {
-        Gbuf0[l] = kInf16x2;
-        Gbuf1[l] = kInf16x2;
+        Gbuf0[TH_IDX(204, l, Tp)] = kInf16x2;
+        Gbuf1[TH_IDX(205, l, Tp)] = kInf16x2;
     }
     __syncthreads();
     if (tid == 0) {
@@ -190,11 +192,11 @@ minplus16_kernel(const Params p)
         uint32_t first = (uint32_t)T + 1u;
         for (int base = 0; base <= T; base += 32) {
             const int l = base + (tid & 31);
-            const unsigned hit = __ballot_sync(0xFFFFFFFFu, l <= T && row[l] != THEMIS_G_INF);
+            const unsigned hit = __ballot_sync(0xFFFFFFFFu, l <= T && row[TH_IDX(206, l, pitch)] != THEMIS_G_INF);
             if (hit) { first = (uint32_t)(base + __ffs((int)hit) - 1); break; }
         }
         if ((tid & 31) == 0) {
-            later_first[s] = first;
+            later_first[TH_IDX(207, s, THEMIS_MAX_STAGES)] = first;
             stage_lmin[s] = first > (uint32_t)T ? 0xFFFFFFFFu : first;   // also the bound the stage skips by
         }
     }
@@ -214,7 +216,8 @@ minplus16_kernel(const Params p)
     auto blank_unused = [&](int s, int nhg_used) {
         const int t_first = max(0, (nhg_used * 16 - n_dummy) * R);
         uint32_t *row = reinterpret_cast<uint32_t *>(F16_inst + (size_t)s * pitch);
-        for (int w = t_first / 2 + tid; w < pitch / 2; w += NT) row[w] = kInf16x2;
+        for (int w = t_first / 2 + tid; w < pitch / 2; w += NT)
+            row[TH_IDX(208, (size_t)s * (pitch / 2) + w, (size_t)S * (pitch / 2)) - (size_t)s * (pitch / 2)] = kInf16x2;
     };
     // "unreachable" for the cells of a tile above the budget limit (only the last tiles in use reach it)
     auto mask_above = [&](uint32_t (&w)[H], int tile, int t_max) {
@@ -233,7 +236,8 @@ minplus16_kernel(const Params p)
         store_words<H>(w, chunk_of(tile));
         const int t0 = (tile - n_dummy) * R;
         if (t0 >= 0 && t0 + R <= pitch)
-            store_words<H>(w, reinterpret_cast<uint32_t *>(F16_inst + (size_t)s * pitch + t0));
+            store_words<H>(w, reinterpret_cast<uint32_t *>(
+                F16_inst + TH_IDX(209, (size_t)s * pitch + t0, (size_t)S * pitch - R + 1)));
     };
 
     // The kernel works on costs relative to every row's cheapest entry, G_s[l] - min G_s, so that
@@ -243,7 +247,7 @@ minplus16_kernel(const Params p)
     auto note_row_cmin = [&](const uint32_t *Gk, int s) {
         uint32_t m = 0xFFFFFFFFu;
         for (int l4 = tid * 4; l4 < pitch; l4 += NT * 4) {
-            const uint4 v = *reinterpret_cast<const uint4 *>(Gk + l4);
+            const uint4 v = *reinterpret_cast<const uint4 *>(Gk + TH_IDX(210, l4, Tp - 3));
             m = min(m, min(min(v.x, v.y), min(v.z, v.w)));
         }
         m = __reduce_min_sync(0xFFFFFFFFu, m);
@@ -276,8 +280,8 @@ minplus16_kernel(const Params p)
 #pragma unroll
             for (int r = H - 1; r >= 0; --r) {
                 // raw costs; entries beyond the loaded row hold kInf16x2, far above kInf16
-                const uint32_t lo = t0 < 0 ? kInf16 : min(Gbuf0[t0 + 2 * r] - c_off0, kInf16);
-                const uint32_t hi = t0 < 0 ? kInf16 : min(Gbuf0[t0 + 2 * r + 1] - c_off0, kInf16);
+                const uint32_t lo = t0 < 0 ? kInf16 : min(Gbuf0[TH_IDX(211, t0 + 2 * r, Tp)] - c_off0, kInf16);
+                const uint32_t hi = t0 < 0 ? kInf16 : min(Gbuf0[TH_IDX(212, t0 + 2 * r + 1, Tp)] - c_off0, kInf16);
                 w[r] = lo | (hi << 16);
             }
             mask_above(w, tile, t_max);
@@ -286,15 +290,15 @@ minplus16_kernel(const Params p)
         if (has_a) init_tile(tile_a);
         if (has_b) init_tile(tile_b);
         if (tid < n_extra) {
-            const uint32_t v = Tc + tid <= t_max ? min(Gbuf0[Tc + tid] - c_off0, kInf16) : kInf16;
-            fx_prev[tid] = v;
-            F16_inst[Tc + tid] = (uint16_t)v;
+            const uint32_t v = Tc + tid <= t_max ? min(Gbuf0[TH_IDX(213, Tc + tid, Tp)] - c_off0, kInf16) : kInf16;
+            fx_prev[TH_IDX(214, tid, kMaxExtra)] = v;
+            F16_inst[TH_IDX(215, Tc + tid, pitch)] = (uint16_t)v;
         }
     }
     failed = __syncthreads_or(failed);
     // Half-word i (< Tc) of the prefix table in shared memory.
     auto f_at = [&](int i) -> uint32_t {
-        const uint32_t w = Fw[(kPadChunks + n_dummy + i / R) * CS + ((i % R) >> 1)];
+        const uint32_t w = Fw[TH_IDX(216, (kPadChunks + n_dummy + i / R) * CS + ((i % R) >> 1), f_words)];
         return (i & 1) ? (w >> 16) : (w & 0xFFFFu);
     };
     // Lowest budget the prefix F_{s-1} can reach: the sum of the earlier rows' first non-empty
@@ -314,14 +318,14 @@ minplus16_kernel(const Params p)
         cost_offset += c_off;
         {
             for (int l4 = tid * 4; l4 < pitch; l4 += NT * 4) {
-                uint4 v4 = *reinterpret_cast<const uint4 *>(Gk + l4);
+                uint4 v4 = *reinterpret_cast<const uint4 *>(Gk + TH_IDX(217, l4, Tp - 3));
                 uint32_t *v = reinterpret_cast<uint32_t *>(&v4);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const uint32_t c = min(v[i] - c_off, kInf16);
                     v[i] = c * 0x10001u;
                 }
-                *reinterpret_cast<uint4 *>(Gk + l4) = v4;
+                *reinterpret_cast<uint4 *>(Gk + TH_IDX(218, l4, Tp - 3)) = v4;
             }
             if (EXTRA && tid < kMaxExtra) fx_acc[tid] = 0xFFFFFFFFu;
         }
@@ -358,7 +362,7 @@ minplus16_kernel(const Params p)
 #pragma unroll
             for (int r = 0; r < H; ++r) { acc[r] = 0xFFFFFFFFu; accp[r] = 0xFFFFFFFFu; }
             const uint32_t *f_hi = chunk_of(tile) - q_lo * CS;   // chunk tile - q_lo: at worst a pad chunk
-            if (steps_of(tile) > 0) load_words<H>(wa, f_hi);
+            if (steps_of(tile) > 0) load_words<H>(wa, TH_PTR(219, f_hi, Fw, f_words - H + 1));
             f_lo = f_hi - CS;
             g = Gk + q_lo * R;
         };
@@ -370,7 +374,7 @@ minplus16_kernel(const Params p)
 #pragma unroll
             for (int r = 0; r < H; ++r)
                 dst[r] = __vminu2(acc[r], __byte_perm(r == 0 ? 0xFFFFFFFFu : accp[r - 1], accp[r], 0x5432));
-            xchg[tile] = accp[H - 1];
+            xchg[TH_IDX(220, tile, n_tiles)] = accp[H - 1];
         };
         int phase = 0, remaining = steps_a;          // phase 0: first tile, 1: second tile, 2: done
         if (has_a) begin_tile(tile_a);
@@ -393,15 +397,18 @@ minplus16_kernel(const Params p)
                 for (; q + U <= n_seg; q += U) {
 #pragma unroll
                     for (int u = 0; u < U; u += 2) {
-                        chunk_step16<R>(wa, wb, acc, accp, f_lo - u * CS, g + u * R);
-                        chunk_step16<R>(wb, wa, acc, accp, f_lo - (u + 1) * CS, g + (u + 1) * R);
+                        chunk_step16<R>(wa, wb, acc, accp, TH_PTR(221, f_lo - u * CS, Fw, f_words - H + 1),
+                                        TH_PTR(222, g + u * R, Gk, Tp - R + 1));
+                        chunk_step16<R>(wb, wa, acc, accp, TH_PTR(223, f_lo - (u + 1) * CS, Fw, f_words - H + 1),
+                                        TH_PTR(224, g + (u + 1) * R, Gk, Tp - R + 1));
                     }
                     f_lo -= U * CS;
                     g += U * R;
                 }
                 for (; q < n_seg; q += 2) {               // segments are even, not multiples of U
-                    chunk_step16<R>(wa, wb, acc, accp, f_lo, g);
-                    chunk_step16<R>(wb, wa, acc, accp, f_lo - CS, g + R);
+                    chunk_step16<R>(wa, wb, acc, accp, TH_PTR(225, f_lo, Fw, f_words - H + 1), TH_PTR(226, g, Gk, Tp - R + 1));
+                    chunk_step16<R>(wb, wa, acc, accp, TH_PTR(227, f_lo - CS, Fw, f_words - H + 1),
+                                    TH_PTR(228, g + R, Gk, Tp - R + 1));
                     f_lo -= 2 * CS;
                     g += 2 * R;
                 }
@@ -419,12 +426,12 @@ minplus16_kernel(const Params p)
             auto share_of_tile = [&](int tile) {
                 for (int r = 0; r < R; ++r) {
                     const int l = tile * R + r;
-                    const uint32_t gl = Gk[l] & 0xFFFFu;
+                    const uint32_t gl = Gk[TH_IDX(229, l, Tp)] & 0xFFFFu;
 #pragma unroll
                     for (int e = 0; e < kMaxExtra; ++e)
                         if (e < n_extra) {
                             const int i = Tc + e - l;         // >= 1
-                            ex[e] = min(ex[e], (i < Tc ? f_at(i) : fx_prev[i - Tc]) + gl);
+                            ex[e] = min(ex[e], (i < Tc ? f_at(i) : fx_prev[TH_IDX(230, i - Tc, kMaxExtra)]) + gl);
                         }
                 }
             };
@@ -434,7 +441,7 @@ minplus16_kernel(const Params p)
 #pragma unroll
                 for (int e = 0; e < kMaxExtra; ++e)
                     for (int l = Tc; l <= Tc + e && e < n_extra; ++l)
-                        ex[e] = min(ex[e], f_at(Tc + e - l) + (Gk[l] & 0xFFFFu));
+                        ex[e] = min(ex[e], f_at(Tc + e - l) + (Gk[TH_IDX(231, l, Tp)] & 0xFFFFu));
             }
 #pragma unroll
             for (int e = 0; e < kMaxExtra; ++e)
@@ -452,7 +459,7 @@ minplus16_kernel(const Params p)
         __syncthreads();                                  // every read of F_{s-1} is done, every tile parked
 
         auto finish_tile = [&](uint32_t (&w)[H], int tile) {
-            const uint32_t left = tile == 0 ? 0xFFFFFFFFu : xchg[tile - 1];
+            const uint32_t left = tile == 0 ? 0xFFFFFFFFu : xchg[TH_IDX(232, tile - 1, n_tiles)];
             w[0] = __vminu2(w[0], __byte_perm(left, 0xFFFFFFFFu, 0x5432));
 #pragma unroll
             for (int r = 0; r < H; ++r) w[r] = __vminu2(w[r], kInf16x2);
@@ -464,7 +471,7 @@ minplus16_kernel(const Params p)
         if (tid < n_extra) {                              // every share arrived before the barrier above
             const uint32_t v = extra_in_use && Tc + tid <= t_max ? min(fx_acc[tid], kInf16) : kInf16;
             fx_prev[tid] = v;
-            F16_inst[(size_t)s * pitch + Tc + tid] = (uint16_t)v;
+            F16_inst[TH_IDX(233, (size_t)s * pitch + Tc + tid, (size_t)S * pitch)] = (uint16_t)v;
         }
     }
     failed = __syncthreads_or(failed);
@@ -505,7 +512,7 @@ minplus16_kernel(const Params p)
             uint32_t lmin = 0xFFFFFFFFu;
             const int32_t *G_row = G_inst + (size_t)s * pitch;
             for (int l = tid; l <= T; l += NT)
-                if (G_row[l] != THEMIS_G_INF) { lmin = (uint32_t)l; break; }
+                if (G_row[TH_IDX(234, l, pitch)] != THEMIS_G_INF) { lmin = (uint32_t)l; break; }
             lmin = block_min(lmin, red, tid, n_warps);
             fastest += lmin == 0xFFFFFFFFu ? (long long)T + 1 : (long long)lmin;
         }
@@ -526,7 +533,7 @@ minplus16_kernel(const Params p)
                 const uint32_t w = chunk[r];
                 const int t = (tile - n_dummy) * R + 2 * r;
                 if (t >= 0 && t < pitch) {
-                    F_row[t] = (w & 0xFFFFu) >= kInf16 ? THEMIS_G_INF : (int32_t)((w & 0xFFFFu) + cost_offset);
+                    F_row[TH_IDX(235, t, pitch - 1)] = (w & 0xFFFFu) >= kInf16 ? THEMIS_G_INF : (int32_t)((w & 0xFFFFu) + cost_offset);
                     F_row[t + 1] = (w >> 16) >= kInf16 ? THEMIS_G_INF : (int32_t)((w >> 16) + cost_offset);
                 }
             }
@@ -536,7 +543,7 @@ minplus16_kernel(const Params p)
     }
 
     if (tid < n_extra)
-        p.F[(size_t)n * pitch + Tc + tid] =
+        p.F[TH_IDX(236, (size_t)n * pitch + Tc + tid, (size_t)p.prob.n_instances * pitch)] =
             fx_prev[tid] >= kInf16 ? THEMIS_G_INF : (int32_t)(fx_prev[tid] + cost_offset);
 
     // backtrack along the optimal path: lowest l with F_{s-1}[t-l] + G_s[l] == F_s[t].
@@ -561,19 +568,19 @@ minplus16_kernel(const Params p)
             for (int k = kScanGroups - 1; k >= 0; --k) {
                 const int l4 = base + (k * NT + tid) * 4;
                 if (l4 <= t) {
-                    const int4 g4 = *reinterpret_cast<const int4 *>(G_row + l4);   // pitch covers l4 + 3
+                    const int4 g4 = *reinterpret_cast<const int4 *>(G_row + TH_IDX(237, l4, pitch - 3));   // pitch covers l4 + 3
                     const int32_t gv[4] = {g4.x, g4.y, g4.z, g4.w};
 #pragma unroll
                     for (int i = 3; i >= 0; --i)
                         if (l4 + i <= t) {
-                            const uint32_t f = Fprev[t - l4 - i];
+                            const uint32_t f = Fprev[TH_IDX(238, t - l4 - i, pitch)];
                             if (f + min((uint32_t)gv[i] - c_off, kInf16) == target) cand = ((uint32_t)(l4 + i) << 16) | f;
                         }
                 }
             }
             cand = __reduce_min_sync(0xFFFFFFFFu, cand);
             uint32_t *rbuf = (round++ & 1) ? red_alt : red;
-            if ((tid & 31) == 0) rbuf[tid >> 5] = cand;
+            if ((tid & 31) == 0) rbuf[TH_IDX(239, tid >> 5, 32)] = cand;
             __syncthreads();
             key = rbuf[0];
             for (int w = 1; w < n_warps; ++w) key = min(key, rbuf[w]);
@@ -581,7 +588,7 @@ minplus16_kernel(const Params p)
         }
         if (key == 0xFFFFFFFFu) { failed = 1; break; }    // cannot happen for consistent tables
         const int ell = (int)(key >> 16);
-        if (tid == 0) ell_of[s] = (uint32_t)ell;
+        if (tid == 0) ell_of[TH_IDX(240, s, Tp)] = (uint32_t)ell;
         t -= ell;
         target = key & 0xFFFFu;
     }
@@ -594,13 +601,13 @@ minplus16_kernel(const Params p)
     // one thread per stage turns (s, l_s) into the stage's configuration
     for (int s = tid; s < S; s += NT) {
         const int ell = (int)ell_of[s];
-        const int idx = (int)p.Garg[((size_t)n * S + s) * pitch + ell];
+        const int idx = (int)p.Garg[TH_IDX(241, ((size_t)n * S + s) * pitch + ell, (size_t)p.prob.n_instances * S * pitch)];
         const int C = p.prob.c_max, NB = p.prob.n_batch;
         const int bi = idx % NB, rest = idx / NB;
-        b_o[s] = p.prob.batch_sizes[bi];
+        b_o[s] = p.prob.batch_sizes[TH_IDX(242, bi, THEMIS_MAX_BATCH_SIZES)];
         c_o[s] = rest % C + 1;
         h_o[s] = p.vertical ? p.replicas[(size_t)n * S + s]
-                   : p.horizontal ? G_inst[(size_t)s * pitch + ell] : rest / C + 1;
+                   : p.horizontal ? G_inst[TH_IDX(243, (size_t)s * pitch + ell, (size_t)S * pitch)] : rest / C + 1;
     }
     if (tid == 0) {
         p.out.total_cost[n] = (int32_t)(best_cost + cost_offset);

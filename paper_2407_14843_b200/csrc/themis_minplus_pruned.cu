@@ -51,9 +51,10 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t id
 
 // Front of one raw G row (int32 costs, THEMIS_G_INF = empty) as packed keys
 // (cost << 14 | l) in ascending l; returns the entry count.  seg = entries per thread.
-__device__ __forceinline__ int extract_front(const uint32_t *g_row, int n_entries, int seg, uint32_t *front,
-                                             uint32_t *warp_tot, int tid)
+__device__ __forceinline__ int extract_front(const Params &p, const uint32_t *g_row, int n_entries, int seg,
+                                             uint32_t *front, uint32_t *warp_tot, int tid)
 {
+    (void)p;
     const int l0 = tid * seg, l1 = min(l0 + seg, n_entries);
     uint32_t local_min = 0xFFFFFFFFu;
     for (int l = l0; l < l1; ++l) local_min = min(local_min, g_row[l]);
@@ -65,7 +66,11 @@ __device__ __forceinline__ int extract_front(const uint32_t *g_row, int n_entrie
     uint32_t pos = block_exclusive_scan<false>(count, 0u, warp_tot, tid);
     running = min(before, kInfCost);
     for (int l = l0; l < l1; ++l)
-        if (g_row[l] < running) { running = g_row[l]; front[pos++] = (running << kIdxBits) | (uint32_t)l; }
+        if (g_row[TH_IDX(401, l, p.pitch)] < running) {
+            running = g_row[l];
+            front[TH_IDX(402, pos, p.pitch)] = (running << kIdxBits) | (uint32_t)l;
+            ++pos;
+        }
     // total = exclusive prefix of the last thread + its count
     __shared__ uint32_t s_total;
     if (tid == kPrunedThreads - 1) s_total = pos;
@@ -102,7 +107,7 @@ minplus_pruned_kernel(const Params p)
         p.out.latency_buckets[n] = -1;
         p.out.status[n] = status;
     };
-    if (p.inst_flag[n] == kFlagBadInput) {     // bad input seen while scoring
+    if (p.inst_flag[TH_IDX(411, n, p.prob.n_instances)] == kFlagBadInput) {     // bad input seen while scoring
         if (tid == 0) write_unsolved(THEMIS_STATUS_BAD_INPUT);
         return;
     }
@@ -140,10 +145,10 @@ minplus_pruned_kernel(const Params p)
     uint32_t *Fprev = Fa, *Fnew = Fb;
     if (!failed) {
         for (int t = tid; t < pitch; t += kPrunedThreads) Fprev[t] = kInfKey;
-        const int P = extract_front(Gbuf0, T + 1, seg, front, red, tid);   // barriers inside order the fill
+        const int P = extract_front(p, Gbuf0, T + 1, seg, front, red, tid);   // barriers inside order the fill
         for (int k = tid; k < P; k += kPrunedThreads) {
             const uint32_t e = front[k];
-            Fprev[e & kIdxMask] = e & ~kIdxMask;
+            Fprev[TH_IDX(403, e & kIdxMask, pitch)] = e & ~kIdxMask;
         }
     }
     __syncthreads();
@@ -156,7 +161,7 @@ minplus_pruned_kernel(const Params p)
         else if (cur) pend1 = -1; else pend0 = -1;
         failed = __syncthreads_or(failed);
         if (failed) break;
-        const int P = extract_front(Graw, T + 1, seg, front, red, tid);
+        const int P = extract_front(p, Graw, T + 1, seg, front, red, tid);
         uint16_t *A_row = p.A + ((size_t)n * S + s) * pitch;
         // kCellsInFlight cells per thread at a time (independent chains hide the
         // shared-memory latency); cells of one thread are kPrunedThreads apart, so the
@@ -167,13 +172,13 @@ minplus_pruned_kernel(const Params p)
             for (int j = 0; j < kCellsInFlight; ++j) acc[j] = 0xFFFFFFFFu;
             const int t_hi = t0 + kPrunedThreads * (kCellsInFlight - 1);
             for (int k = 0; k < P; ++k) {
-                const uint32_t e = front[k];
+                const uint32_t e = front[TH_IDX(404, k, pitch)];
                 const int l = (int)(e & kIdxMask);
                 if (l > t_hi) break;            // ascending l: nothing further fits any of these cells
 #pragma unroll
                 for (int j = 0; j < kCellsInFlight; ++j) {
                     const int i = t0 + kPrunedThreads * j - l;
-                    const uint32_t f = i >= 0 && i < pitch ? Fprev[i] : kInfKey;
+                    const uint32_t f = i >= 0 && i < pitch ? Fprev[TH_IDX(405, i, pitch)] : kInfKey;
                     acc[j] = __viaddmin_u32(f, e, acc[j]);
                 }
             }
@@ -182,8 +187,8 @@ minplus_pruned_kernel(const Params p)
                 const int t = t0 + kPrunedThreads * j;
                 if (t < pitch) {
                     const bool inf = acc[j] >= kInfKey;
-                    Fnew[t] = inf ? kInfKey : (acc[j] & ~kIdxMask);
-                    A_row[t] = inf ? (uint16_t)0 : (uint16_t)(acc[j] & kIdxMask);
+                    Fnew[TH_IDX(406, t, pitch)] = inf ? kInfKey : (acc[j] & ~kIdxMask);
+                    A_row[TH_IDX(407, t, pitch)] = inf ? (uint16_t)0 : (uint16_t)(acc[j] & kIdxMask);
                 }
             }
         }
@@ -205,7 +210,7 @@ minplus_pruned_kernel(const Params p)
     for (int t = tid; t < pitch; t += kPrunedThreads) {
         const uint32_t fk = Fprev[t];
         if (t <= T) best = min(best, fk | (uint32_t)t);
-        F_row[t] = fk >= kInfKey ? THEMIS_G_INF : (int32_t)(fk >> kIdxBits);
+        F_row[TH_IDX(408, t, pitch)] = fk >= kInfKey ? THEMIS_G_INF : (int32_t)(fk >> kIdxBits);
     }
     best = __reduce_min_sync(0xFFFFFFFFu, best);
     if ((tid & 31) == 0) red[tid >> 5] = best;
@@ -220,8 +225,8 @@ minplus_pruned_kernel(const Params p)
             const int C = p.prob.c_max, NB = p.prob.n_batch;
             for (int s = S - 1; s >= 0; --s) {
                 const size_t row = ((size_t)n * S + s) * pitch;
-                const int ell = s > 0 ? (int)p.A[row + t] : t;
-                const int idx = (int)p.Garg[row + ell];
+                const int ell = s > 0 ? (int)p.A[TH_IDX(409, row + t, (size_t)p.prob.n_instances * S * pitch)] : t;
+                const int idx = (int)p.Garg[TH_IDX(410, row + ell, (size_t)p.prob.n_instances * S * pitch)];
                 const int bi = idx % NB, rest = idx / NB;
                 b_o[s] = p.prob.batch_sizes[bi];
                 c_o[s] = rest % C + 1;

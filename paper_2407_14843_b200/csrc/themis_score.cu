@@ -76,6 +76,25 @@ __device__ __forceinline__ void score_two_entries(uint32_t entries, uint32_t q4,
         : "memory");
 }
 
+#ifdef THEMIS_CHECK_BOUNDS
+// The same step with every address formed in C++ and range-checked (bounds-checked build).
+__device__ __forceinline__ void score_two_entries_checked(const Params &p, uint32_t *smem, int smem_words,
+                                                          int entries_word, uint32_t q4, uint32_t lmax, uint32_t t4,
+                                                          uint32_t key_mul, uint32_t key_add, int keys_word,
+                                                          int idle_word)
+{
+    for (int j = 0; j < 2; ++j) {
+        const uint32_t e0 = smem[TH_IDX(140, entries_word + 2 * j, smem_words)];
+        const uint32_t x = smem[TH_IDX(141, entries_word + 2 * j + 1, smem_words)] + q4;
+        const uint32_t l = x & 0x1FFFCu;
+        const bool ok = e0 <= lmax && l <= t4;
+        const uint32_t key = (x >> 17) * key_mul + key_add;
+        const int word = ok ? keys_word + (int)(l >> 2) : idle_word;
+        atomicMin(&smem[TH_IDX(142, word, smem_words)], key);
+    }
+}
+#endif
+
 __device__ __forceinline__ uint32_t sat_u32(unsigned long long v, uint32_t cap)
 {
     return v > (unsigned long long)cap ? cap : (uint32_t)v;
@@ -107,12 +126,14 @@ score_kernel(const Params p)
     const int lmax_off = q_off + SV * NB * HN;
     const int list_base = (lmax_off + SV * NB * HN + 3) & ~3;
     const int list_off = list_base + warp * kListWords;
+    const int smem_words = list_base + kScoreWarps * kListWords + 32;   // what the launch provides
+    (void)smem_words;
     const uint32_t smem_addr = (uint32_t)__cvta_generic_to_shared(smem);
     const uint32_t idle_addr = smem_addr + 4u * (uint32_t)(list_base + kScoreWarps * kListWords + lane);
     __shared__ int s_bad;
 
-    const uint32_t lambda_m = p.lambda_mrps[n];
-    const int pid = p.profile_id ? p.profile_id[n] : 0;
+    const uint32_t lambda_m = p.lambda_mrps[TH_IDX(101, n, p.prob.n_instances)];
+    const int pid = p.profile_id ? p.profile_id[TH_IDX(102, n, p.prob.n_instances)] : 0;
     const int32_t *rep = p.vertical ? p.replicas + (size_t)n * S : nullptr;
 
     if (tid == 0) {
@@ -128,7 +149,7 @@ score_kernel(const Params p)
         s_bad = bad;
     }
     for (int l4 = tid * 4; l4 < 2 * pitch; l4 += kScoreThreads * 4)
-        *reinterpret_cast<uint4 *>(smem + l4) = make_uint4(kEmptyKey, kEmptyKey, kEmptyKey, kEmptyKey);
+        *reinterpret_cast<uint4 *>(smem + TH_IDX(124, l4, 2 * pitch - 3)) = make_uint4(kEmptyKey, kEmptyKey, kEmptyKey, kEmptyKey);
     __syncthreads();
     const bool skip_all = s_bad != 0;
     const int32_t *lat = p.lat_us + (size_t)(skip_all ? 0 : pid) * S * CB;
@@ -143,12 +164,12 @@ score_kernel(const Params p)
             const int sv = e / (NB * HN);
             const int bi = (e - sv * NB * HN) / HN;
             const int k = e - (sv * NB + bi) * HN;
-            const unsigned long long h = (unsigned long long)((p.vertical ? rep[sv] : 1) + k);
-            const unsigned long long b = (unsigned long long)p.prob.batch_sizes[bi];
+            const unsigned long long h = (unsigned long long)((p.vertical ? rep[TH_IDX(105, sv, S)] : 1) + k);
+            const unsigned long long b = (unsigned long long)p.prob.batch_sizes[TH_IDX(106, bi, NB)];
             const unsigned long long m = (p.prob.flags & THEMIS_QUEUE_PER_REPLICA) ? h : 1ull;
             const unsigned long long q_num = (b - 1ull) * m * 1000000000ull;
-            smem[q_off + e] = sat_u32((q_num + q_den - 1ull) / q_den, (uint32_t)T + 1u);
-            smem[lmax_off + e] = sat_u32(h * b * 1000000000ull / lambda_m, 0x7FFFFFFFu);
+            smem[TH_IDX(103, q_off + e, lmax_off)] = sat_u32((q_num + q_den - 1ull) / q_den, (uint32_t)T + 1u);
+            smem[TH_IDX(104, lmax_off + e, list_base)] = sat_u32(h * b * 1000000000ull / lambda_m, 0x7FFFFFFFu);
         }
     }
     __syncthreads();                            // tables ready, both key rows empty
@@ -181,8 +202,8 @@ score_kernel(const Params p)
                 bool live = cidx < C;
                 uint32_t l_us = 0, l_b = 0;
                 if (live) {
-                    const int32_t v = lat_s[pair];
-                    const int32_t v_prev = cidx > 0 ? lat_s[pair - NB] : 0;
+                    const int32_t v = lat_s[TH_IDX(107, pair, CB)];
+                    const int32_t v_prev = cidx > 0 ? lat_s[TH_IDX(108, pair - NB, CB)] : 0;
                     if (v <= 0) saw_bad_latency = 1;
                     // Same latency with one core fewer: that candidate reaches the same buckets with
                     // the same replica counts at a lower cost, so this one is never a minimum
@@ -205,20 +226,24 @@ score_kernel(const Params p)
                     if (live) {
                         int lo = 0, cnt = HN;
                         if (HN == 1) {                       // vertical variant: the one replica count
-                            lo = smem[lmax_row] < l_us ? 1 : 0;
+                            lo = smem[TH_IDX(109, lmax_row, list_base)] < l_us ? 1 : 0;
                             cnt = 0;
                         }
                         while (cnt > 0) {
                             const int half = cnt >> 1;
-                            if (smem[lmax_row + lo + half] < l_us) { lo += half + 1; cnt -= half + 1; }
+                            if (smem[TH_IDX(110, lmax_row + lo + half, list_base)] < l_us) { lo += half + 1; cnt -= half + 1; }
                             else cnt = half;
                         }
                         if (lo < HN) {
-                            const uint32_t ell = l_b + smem[q_row + lo];
+                            const uint32_t ell = l_b + smem[TH_IDX(111, q_row + lo, lmax_off)];
                             if (ell <= (uint32_t)T) {
                                 const uint32_t cost = (uint32_t)(h_lo + lo) * (uint32_t)(cidx + 1);
                                 const uint32_t idx = (uint32_t)((p.horizontal ? 0 : lo * CB) + pair);
+#ifdef THEMIS_CHECK_BOUNDS
+                                atomicMin(&smem[TH_IDX(112, key_off + (int)ell, key_off + pitch)], (cost << 16) | idx);
+#else
                                 red_min_shared(key_addr + 4u * ell, (cost << 16) | idx);
+#endif
                             }
                         }
                     }
@@ -226,29 +251,36 @@ score_kernel(const Params p)
                     // Joint problem with h_max >= 2 (so c <= 32767: at most 65535 candidates per stage).
                     for (int h0 = 0; h0 < HN; h0 += HNp) {
                         // pairs that still fit the budget at this chunk's first replica count ...
-                        const bool fits = live && l_b + smem[q_row + h0] <= (uint32_t)T;
+                        const bool fits = live && l_b + smem[TH_IDX(113, q_row + h0, lmax_off)] <= (uint32_t)T;
                         if (__ballot_sync(0xFFFFFFFFu, fits) == 0u) break;     // q never shrinks with h
                         // ... and sustain lambda at its last
-                        const bool in = fits && l_us <= smem[lmax_row + min(h0 + HNp, HN) - 1];
+                        const bool in = fits && l_us <= smem[TH_IDX(114, lmax_row + min(h0 + HNp, HN) - 1, list_base)];
                         const uint32_t mask = __ballot_sync(0xFFFFFFFFu, in);
                         const int cnt = __popc(mask);
                         // compacted entries first; the other slots hold a latency no replica count sustains
                         if (lane >= cnt)
-                            *reinterpret_cast<uint2 *>(smem + list_off + 2 * lane) = make_uint2(kNeverFits, 0u);
+                            *reinterpret_cast<uint2 *>(smem + TH_IDX(115, list_off + 2 * lane, smem_words - 1)) = make_uint2(kNeverFits, 0u);
                         if (in)
-                            *reinterpret_cast<uint2 *>(smem + list_off + 2 * __popc(mask & lanemask_lt)) =
+                            *reinterpret_cast<uint2 *>(smem + TH_IDX(116, list_off + 2 * __popc(mask & lanemask_lt), smem_words - 1)) =
                                 make_uint2(l_us, (l_b << 2) | ((uint32_t)(cidx + 1) << 17));
                         __syncwarp();
                         const int k = h0 + hk;                       // this lane's replica count - 1
                         const bool kv = k < HN;
-                        const uint32_t q4 = 4u * (kv ? smem[q_row + k] : (uint32_t)T + 1u);
-                        const uint32_t lmax = kv ? smem[lmax_row + k] : 0u;
+                        const uint32_t q4 = 4u * (kv ? smem[TH_IDX(117, q_row + k, lmax_off)] : (uint32_t)T + 1u);
+                        const uint32_t lmax = kv ? smem[TH_IDX(118, lmax_row + k, list_base)] : 0u;
                         // key = (h * c) << 16 | (h - 1) * CB + (c - 1) * NB + bi  =  c * key_mul + key_add
                         const uint32_t key_mul = ((uint32_t)(k + 1) << 16) + (uint32_t)NB;
                         const uint32_t key_add = (uint32_t)(k * CB - NB + bi);
+#ifdef THEMIS_CHECK_BOUNDS
+                        for (int i = 0; i < cnt; i += 2 * groups)
+                            score_two_entries_checked(p, smem, smem_words, list_off + 4 * group + 2 * i, q4, lmax,
+                                                      4u * (uint32_t)T, key_mul, key_add, key_off,
+                                                      list_base + kScoreWarps * kListWords + lane);
+#else
                         uint32_t entries = list_addr;
                         for (int i = 0; i < cnt; i += 2 * groups, entries += 16u * (uint32_t)groups)
                             score_two_entries(entries, q4, lmax, 4u * (uint32_t)T, key_mul, key_add, key_addr, idle_addr);
+#endif
                         __syncwarp();
                     }
                 }
@@ -262,8 +294,9 @@ score_kernel(const Params p)
         int32_t *G_row = p.G + ((size_t)n * S + s) * pitch;
         uint16_t *Garg_row = p.Garg + ((size_t)n * S + s) * pitch;
         for (int l4 = tid * 4; l4 < pitch; l4 += kScoreThreads * 4) {
-            const uint4 k4 = *reinterpret_cast<const uint4 *>(smem + key_off + l4);
-            *reinterpret_cast<uint4 *>(smem + key_off + l4) = make_uint4(kEmptyKey, kEmptyKey, kEmptyKey, kEmptyKey);
+            const uint4 k4 = *reinterpret_cast<const uint4 *>(smem + TH_IDX(119, key_off + l4, key_off + pitch - 3));
+            *reinterpret_cast<uint4 *>(smem + TH_IDX(120, key_off + l4, key_off + pitch - 3)) =
+                make_uint4(kEmptyKey, kEmptyKey, kEmptyKey, kEmptyKey);
             const uint32_t kk[4] = {k4.x, k4.y, k4.z, k4.w};
             int4 g;
             int32_t *gv = reinterpret_cast<int32_t *>(&g);
@@ -274,13 +307,13 @@ score_kernel(const Params p)
                 gv[i] = empty ? THEMIS_G_INF : (int32_t)(kk[i] >> 16);
                 a[i] = empty ? 0u : kk[i];
             }
-            *reinterpret_cast<int4 *>(G_row + l4) = g;
-            *reinterpret_cast<uint2 *>(Garg_row + l4) =
+            *reinterpret_cast<int4 *>(G_row + TH_IDX(121, l4, pitch - 3)) = g;
+            *reinterpret_cast<uint2 *>(Garg_row + TH_IDX(122, l4, pitch - 3)) =
                 make_uint2(__byte_perm(a[0], a[1], 0x5410), __byte_perm(a[2], a[3], 0x5410));
         }
     }
     const int any_bad = __syncthreads_or(saw_bad_latency);
-    if (tid == 0) p.inst_flag[n] = (skip_all || any_bad) ? kFlagBadInput : 0;
+    if (tid == 0) p.inst_flag[TH_IDX(123, n, p.prob.n_instances)] = (skip_all || any_bad) ? kFlagBadInput : 0;
 }
 
 }  // namespace

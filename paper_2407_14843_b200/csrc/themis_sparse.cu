@@ -59,9 +59,10 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t id
 // is called for each, pos counting from 0 in ascending index order; the row is left
 // empty.  Returns the number of front entries.
 template <int SHIFT, int kThreads, class Emit>
-__device__ __forceinline__ int front_of_row(uint32_t *row, int n_entries, int seg, uint32_t *warp_tot,
-                                            uint32_t *s_total, int tid, Emit emit)
+__device__ __forceinline__ int front_of_row(const Params &p, uint32_t *row, int n_entries, int seg,
+                                            uint32_t *warp_tot, uint32_t *s_total, int tid, Emit emit)
 {
+    (void)p;
     constexpr uint32_t kBig = 0xFFFFFFFFu;
     const int l0 = tid * seg, l1 = min(l0 + seg, n_entries);
     uint32_t local_min = kBig;
@@ -78,7 +79,7 @@ __device__ __forceinline__ int front_of_row(uint32_t *row, int n_entries, int se
     uint32_t pos = block_exclusive_scan<false>(count, 0u, warp_tot, tid);
     running = before;
     for (int l = l0; l < l1; ++l) {
-        const uint32_t key = row[l];
+        const uint32_t key = row[TH_IDX(501, l, p.pitch)];
         row[l] = kEmpty;
         if (key != kEmpty && (key >> SHIFT) < running) { running = key >> SHIFT; emit((int)pos++, l, key); }
     }
@@ -117,9 +118,11 @@ __device__ __forceinline__ void solve_instance_sparse(const Params &p, const int
     __shared__ uint32_t s_total;
     __shared__ int s_bad;
 
-    const uint32_t lambda_m = p.lambda_mrps[n];
+    const uint32_t lambda_m = p.lambda_mrps[TH_IDX(502, n, p.prob.n_instances)];
     const int pid = p.profile_id ? p.profile_id[n] : 0;
     const int32_t *lat = p.lat_us + (size_t)pid * S * CB;
+    const int tab = SV * NB * HN;
+    (void)tab;
     const int32_t *rep = p.vertical ? p.replicas + (size_t)n * S : nullptr;
     int32_t *h_o = p.out.h + (size_t)n * S, *c_o = p.out.c + (size_t)n * S, *b_o = p.out.b + (size_t)n * S;
     auto write_unsolved = [&](int status) {
@@ -157,8 +160,8 @@ __device__ __forceinline__ void solve_instance_sparse(const Params &p, const int
             const unsigned long long b = (unsigned long long)p.prob.batch_sizes[bi];
             const unsigned long long m = (p.prob.flags & THEMIS_QUEUE_PER_REPLICA) ? h : 1ull;
             const unsigned long long q_num = (b - 1ull) * m * 1000000000ull;
-            Q[e] = sat_u32((q_num + q_den - 1ull) / q_den, (uint32_t)T + 1u);
-            Lmax[e] = sat_u32(h * b * 1000000000ull / lambda_m, 0x7FFFFFFFu);
+            Q[TH_IDX(503, e, tab)] = sat_u32((q_num + q_den - 1ull) / q_den, (uint32_t)T + 1u);
+            Lmax[TH_IDX(504, e, tab)] = sat_u32(h * b * 1000000000ull / lambda_m, 0x7FFFFFFFu);
         }
     }
     __syncthreads();
@@ -181,9 +184,9 @@ __device__ __forceinline__ void solve_instance_sparse(const Params &p, const int
             const int c = (task - bi * c_chunks) * 32 + lane + 1;
             if (c > C) continue;
             const int pair = (c - 1) * NB + bi;
-            const int32_t l_us = lat_s[pair];
+            const int32_t l_us = lat_s[TH_IDX(505, pair, CB)];
             if (l_us <= 0) { saw_bad_latency = 1; continue; }
-            if (c > 1 && lat_s[pair - NB] == l_us) continue;       // same buckets, cheaper, one core fewer
+            if (c > 1 && lat_s[TH_IDX(506, pair - NB, CB)] == l_us) continue;   // same buckets, cheaper, one core fewer
             uint32_t l_q = __umulhi((uint32_t)l_us, w_magic);
             uint32_t l_r = (uint32_t)l_us - l_q * w_us;
             while (l_r >= w_us) { l_r -= w_us; ++l_q; }
@@ -194,14 +197,14 @@ __device__ __forceinline__ void solve_instance_sparse(const Params &p, const int
             const float need = (float)l_us * ((float)lambda_m / ((float)b * 1.0e9f)) - (float)h_lo;
             int k = (int)fminf(fmaxf(need, 0.0f), (float)HN) - 1;
             k = max(k, 0);
-            if (k > 0 && (uint32_t)l_us <= lmax_row[k - 1]) k = 0;
-            while (k < HN && (uint32_t)l_us > lmax_row[k]) ++k;
+            if (k > 0 && (uint32_t)l_us <= lmax_row[TH_IDX(507, k - 1, HN)]) k = 0;
+            while (k < HN && (uint32_t)l_us > lmax_row[TH_IDX(508, k, HN)]) ++k;
             if (k >= HN) continue;                                   // no replica count sustains lambda
-            const uint32_t ell = l_b + Q_s[bi * HN + k];
+            const uint32_t ell = l_b + Q_s[TH_IDX(509, bi * HN + k, NB * HN)];
             if (ell > (uint32_t)T) continue;
             const uint32_t cost = (uint32_t)(h_lo + k) * (uint32_t)c;
             const uint32_t idx = (uint32_t)((p.horizontal ? 0 : k * CB) + pair);
-            atomicMin(&keys_g[ell], (cost << 16) | idx);
+            atomicMin(&keys_g[TH_IDX(510, ell, pitch)], (cost << 16) | idx);
         }
         __syncthreads();
 
@@ -209,37 +212,37 @@ __device__ __forceinline__ void solve_instance_sparse(const Params &p, const int
         uint32_t *G_row = reinterpret_cast<uint32_t *>(p.G + ((size_t)n * S + s) * pitch);
         uint16_t *Gc_row = p.Garg + ((size_t)n * S + s) * pitch;
         uint16_t *A_row = p.A + ((size_t)n * S + s) * pitch;
-        const int n_g = front_of_row<16, kThreads>(keys_g, T + 1, seg, warp_tot, &s_total, tid,
+        const int n_g = front_of_row<16, kThreads>(p, keys_g, T + 1, seg, warp_tot, &s_total, tid,
             [&](int pos, int l, uint32_t key) {
-                gf_l[pos] = (uint32_t)l;
-                gf_c[pos] = key >> 16;
-                G_row[pos] = ((uint32_t)l << 16) | (key & 0xFFFFu);
-                Gc_row[pos] = (uint16_t)(key >> 16);
+                gf_l[TH_IDX(511, pos, cap_g)] = (uint32_t)l;
+                gf_c[TH_IDX(512, pos, cap_g)] = key >> 16;
+                G_row[TH_IDX(513, pos, pitch)] = ((uint32_t)l << 16) | (key & 0xFFFFu);
+                Gc_row[TH_IDX(514, pos, pitch)] = (uint16_t)(key >> 16);
                 if (s == 0) {                      // the first stage's front is the first prefix front
-                    ff_t[pos] = (uint32_t)l;
-                    ff_c[pos] = key >> 16;
-                    A_row[l] = (uint16_t)pos;
+                    ff_t[TH_IDX(515, pos, pitch)] = (uint32_t)l;
+                    ff_c[TH_IDX(516, pos, pitch)] = key >> 16;
+                    A_row[TH_IDX(517, l, pitch)] = (uint16_t)pos;
                 }
             });
         if (s == 0) { n_f = n_g; continue; }
 
         // 3. front(F_{s-1}) x front(G_s): each warp takes prefix entries, lanes take stage entries
         for (int i = warp; i < n_f; i += kWarps) {
-            const uint32_t t_i = ff_t[i], c_i = ff_c[i];
+            const uint32_t t_i = ff_t[TH_IDX(518, i, pitch)], c_i = ff_c[TH_IDX(519, i, pitch)];
             for (int k = lane; k < n_g; k += 32) {
-                const uint32_t t = t_i + gf_l[k];
+                const uint32_t t = t_i + gf_l[TH_IDX(520, k, cap_g)];
                 if (t > (uint32_t)T) break;           // ascending l: the rest does not fit either
-                atomicMin(&keys_f[t], ((c_i + gf_c[k]) << kIdxBits) | (uint32_t)k);
+                atomicMin(&keys_f[TH_IDX(521, t, pitch)], ((c_i + gf_c[TH_IDX(522, k, cap_g)]) << kIdxBits) | (uint32_t)k);
             }
         }
         __syncthreads();
 
         // 4. front of F_s; the argmin k of every front cell goes to the workspace
-        n_f = front_of_row<kIdxBits, kThreads>(keys_f, T + 1, seg, warp_tot, &s_total, tid,
+        n_f = front_of_row<kIdxBits, kThreads>(p, keys_f, T + 1, seg, warp_tot, &s_total, tid,
             [&](int pos, int t, uint32_t key) {
-                ff_t[pos] = (uint32_t)t;
-                ff_c[pos] = key >> kIdxBits;
-                A_row[t] = (uint16_t)(key & kIdxMask);
+                ff_t[TH_IDX(523, pos, pitch)] = (uint32_t)t;
+                ff_c[TH_IDX(524, pos, pitch)] = key >> kIdxBits;
+                A_row[TH_IDX(525, t, pitch)] = (uint16_t)(key & kIdxMask);
             });
     }
     const int any_bad = __syncthreads_or(saw_bad_latency);    // also orders this block's global stores
@@ -249,12 +252,12 @@ __device__ __forceinline__ void solve_instance_sparse(const Params &p, const int
     if (n_f == 0) { write_unsolved(THEMIS_STATUS_INFEASIBLE); return; }
     // Costs fall strictly along the front, so its last entry is the cheapest total at
     // the lowest budget that reaches it.
-    const int tstar = (int)ff_t[n_f - 1];
+    const int tstar = (int)ff_t[TH_IDX(526, n_f - 1, pitch)];
     int t = tstar;
     for (int s = S - 1; s >= 0; --s) {
         const size_t row = ((size_t)n * S + s) * pitch;
-        const int k = (int)p.A[row + t];
-        const uint32_t e = reinterpret_cast<const uint32_t *>(p.G)[row + k];
+        const int k = (int)p.A[TH_IDX(527, row + t, (size_t)p.prob.n_instances * S * pitch)];
+        const uint32_t e = reinterpret_cast<const uint32_t *>(p.G)[TH_IDX(528, row + k, (size_t)p.prob.n_instances * S * pitch)];
         const int ell = (int)(e >> 16), idx = (int)(e & 0xFFFFu);
         const int bi = idx % NB, rest = idx / NB;
         b_o[s] = p.prob.batch_sizes[bi];
@@ -281,7 +284,7 @@ solve_sparse_kernel(const Params p)
     }
     const int count = min(*p.redo_count, p.prob.n_instances);
     for (int i = blockIdx.x; i < count; i += gridDim.x) {
-        solve_instance_sparse<kThreads>(p, p.redo_list[i], smem);
+        solve_instance_sparse<kThreads>(p, TH_IDX(529, p.redo_list[TH_IDX(530, i, p.prob.n_instances)], p.prob.n_instances), smem);
         __syncthreads();                 // the last reader of this instance's shared memory is done
     }
 }
@@ -296,8 +299,9 @@ size_t sparse_smem_bytes(const Params &p)
     return sizeof(uint32_t) * (3u * (size_t)p.pitch + 2u * cap_g + 2u * table + 32u);
 }
 
+// (internal linkage: its `ready` word must belong to this copy of the library alone)
 template <int kThreads, bool LISTED>
-cudaError_t launch_sparse_variant(const Params &p, size_t smem, cudaStream_t stream)
+static cudaError_t launch_sparse_variant(const Params &p, size_t smem, cudaStream_t stream)
 {
     static std::atomic<uint64_t> ready{0};
     cudaError_t e = allow_max_smem(reinterpret_cast<const void *>(solve_sparse_kernel<kThreads, LISTED>), ready);

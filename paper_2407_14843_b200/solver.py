@@ -41,7 +41,7 @@ EXPORTS = (
     "themis_fit_profiles_batch", "themis_configs_equal_batch",
 )
 # include/themis_probe.h: measurement probes, not part of the solver
-PROBE_EXPORTS = ("themis_alu_probe", "themis_wait_probe")
+PROBE_EXPORTS = ("themis_alu_probe", "themis_wait_probe", "themis_bounds_check_report")
 
 
 class ThemisError(RuntimeError):
@@ -89,12 +89,12 @@ class WorkspaceLayout(ctypes.Structure):
                 ("row_pitch", ctypes.c_int32), ("T", ctypes.c_int32)]
 
 
-def _load() -> ctypes.CDLL:
-    if not os.path.exists(LIB_PATH):
+def _load(path: str = LIB_PATH) -> ctypes.CDLL:
+    if not os.path.exists(path):
         raise ImportError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2407_14843_b200.build` "
+            f"{path} is missing: build it with `python -m paper_2407_14843_b200.build` "
             "(there is no fallback implementation)")
-    lib = ctypes.CDLL(LIB_PATH)
+    lib = ctypes.CDLL(path)
     PP, vp, sz = ctypes.POINTER(Problem), ctypes.c_void_p, ctypes.c_size_t
     lib.themis_version.restype = ctypes.c_int
     lib.themis_version.argtypes = []
@@ -118,6 +118,7 @@ def _load() -> ctypes.CDLL:
                                               ctypes.c_int32, vp, vp, vp, vp, vp]
     lib.themis_alu_probe.argtypes = [ctypes.c_int] * 4 + [vp, vp]
     lib.themis_wait_probe.argtypes = [ctypes.c_int32, vp, vp, vp, vp]
+    lib.themis_bounds_check_report.argtypes = [PP, ctypes.c_int, vp, sz, ctypes.POINTER(ctypes.c_int32 * 4), vp]
     for name in EXPORTS + PROBE_EXPORTS:
         if name != "themis_strerror":
             getattr(lib, name).restype = ctypes.c_int
@@ -282,6 +283,23 @@ def themis_alu_probe(mode: int, blocks: int, threads: int, iters: int, sink) -> 
         raise ValueError("sink too small")
     _check(_lib.themis_alu_probe(mode, blocks, threads, iters, _dptr(sink, torch.uint32, "sink"), _stream()),
            "themis_alu_probe")
+
+
+def themis_bounds_check_report(problem: Problem, vertical: bool, workspace) -> dict:
+    """Record of the bounds-checked build for the last solve on ``workspace`` (waits for the
+    stream): ``{"site", "index", "limit", "checked"}``; all zero with the normal library."""
+    rep = (ctypes.c_int32 * 4)()
+    _check(_lib.themis_bounds_check_report(ctypes.byref(problem), int(vertical),
+                                           _dptr(workspace, torch.uint8, "workspace"), workspace.numel(),
+                                           ctypes.byref(rep), _stream()), "themis_bounds_check_report")
+    return {"site": rep[0], "index": rep[1], "limit": rep[2], "checked": bool(rep[3])}
+
+
+def use_library(path: str = LIB_PATH) -> None:
+    """Routes every call of this module to the library at ``path`` (the normal one by default;
+    ``build.CHECK_LIB_PATH`` for the bounds-checked build)."""
+    global _lib
+    _lib = _load(path)
 
 
 def themis_wait_probe(max_polls: int, src16, dst16, status) -> None:
