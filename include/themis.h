@@ -72,7 +72,10 @@ extern "C" {
  *      stages of their first non-empty bucket), and 0x7FFF above (such a state is part of
  *      no solution); the backtrack recovers the argmin along the optimal path only.  Instances
  *      whose optimum lies 32767 or more above the sum of the stages' cheapest entries
- *      are redone by the 32-bit kernel in a second launch.
+ *      are redone by the 32-bit kernel in a second launch.  Budgets of up to 1100 cells
+ *      run with one warp per instance, longer ones with one thread block per instance.
+ *   THEMIS_KERNEL_PACKED16_BLOCK  the same with one thread block per instance whatever
+ *      the budget length (same tables, same results).
  *   THEMIS_KERNEL_WIDE32       dense recurrence on 32-bit keys; the A rows hold the
  *      argmin tables.
  *   THEMIS_KERNEL_PRUNED       dense scoring, then the recurrence restricted to the
@@ -100,6 +103,7 @@ extern "C" {
 #define THEMIS_KERNEL_PRUNED       (3u << 8)
 #define THEMIS_KERNEL_SPARSE       (4u << 8)
 #define THEMIS_KERNEL_SPARSE_BLOCK (5u << 8)
+#define THEMIS_KERNEL_PACKED16_BLOCK (6u << 8)
 #define THEMIS_KERNEL_MASK         (15u << 8)
 
 /* themis_problem_t.flags, bits 12..13: consecutive budget cells per thread of the

@@ -52,7 +52,7 @@ int validate(const themis_problem_t *pr, int vertical, int32_t *T_out, int32_t *
         return THEMIS_E_INVALID_ARG;
     if (pr->slo_us < 1 || pr->bucket_us < 1) return THEMIS_E_INVALID_ARG;
     if (pr->flags & ~(THEMIS_QUEUE_PER_REPLICA | THEMIS_KERNEL_MASK | THEMIS_TILE_MASK)) return THEMIS_E_INVALID_ARG;
-    if ((pr->flags & THEMIS_KERNEL_MASK) > THEMIS_KERNEL_SPARSE_BLOCK) return THEMIS_E_INVALID_ARG;
+    if ((pr->flags & THEMIS_KERNEL_MASK) > THEMIS_KERNEL_PACKED16_BLOCK) return THEMIS_E_INVALID_ARG;
     if (!vertical && pr->h_max < 1) return THEMIS_E_INVALID_ARG;
     if (pr->n_batch > THEMIS_MAX_BATCH_SIZES) return THEMIS_E_UNSUPPORTED_SIZE;
     for (int i = 0; i < pr->n_batch; ++i) {
@@ -167,10 +167,13 @@ int minplus_impl(const themis_problem_t *pr, const int32_t *rep, const SolveOpts
     const int tile = tile_of(pr);
     if (kernel == THEMIS_KERNEL_WIDE32) {
         e = launch_minplus(P, tile, st);
-    } else if (kernel >= THEMIS_KERNEL_PRUNED && pruned_smem_bytes(P.pitch) <= kMaxDynamicSmem) {
+    } else if (kernel >= THEMIS_KERNEL_PRUNED && kernel != THEMIS_KERNEL_PACKED16_BLOCK &&
+               pruned_smem_bytes(P.pitch) <= kMaxDynamicSmem) {
         e = launch_minplus_pruned(P, st);
     } else {
-        e = launch_minplus16(P, tile, st);
+        // short budgets: a warp per instance, unless the block kernel is asked for
+        e = kernel != THEMIS_KERNEL_PACKED16_BLOCK && minplus16_warp_fits(P, tile) ? launch_minplus16_warp(P, tile, st)
+                                                                                  : launch_minplus16(P, tile, st);
         // A total can only reach the 16-bit saturation value if the static bound allows it
         // (vertical: the bound depends on replicas[], which lives on the device).
         const bool may_saturate =

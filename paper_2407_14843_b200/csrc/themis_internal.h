@@ -129,6 +129,9 @@ constexpr int kBoundsChecked = 0;
 cudaError_t launch_score(const Params &p, cudaStream_t stream);
 cudaError_t launch_minplus(const Params &p, int tile, cudaStream_t stream);
 cudaError_t launch_minplus16(const Params &p, int tile, cudaStream_t stream);
+// The packed kernel with one warp per instance, for short budgets (tiles of 4 or 8 cells).
+bool minplus16_warp_fits(const Params &p, int tile);
+cudaError_t launch_minplus16_warp(const Params &p, int tile, cudaStream_t stream);
 cudaError_t launch_minplus_pruned(const Params &p, cudaStream_t stream);
 // Scoring and recurrence on undominated entries in one kernel (needs lat_us, lambda, out set),
 // one block per instance; only_listed: a fixed grid works through redo_list instead.

@@ -20,8 +20,8 @@ LIB_PATH = os.path.join(_PKG, "libthemis.so")
 
 QUEUE_PER_REPLICA = 1
 # themis_problem_t.flags: kernel choice of a call (bits 8..11) and cells per thread (bits 12..13)
-KERNEL_DEFAULT, KERNEL_PACKED16, KERNEL_WIDE32, KERNEL_PRUNED, KERNEL_SPARSE, KERNEL_SPARSE_BLOCK = (
-    k << 8 for k in range(6))
+(KERNEL_DEFAULT, KERNEL_PACKED16, KERNEL_WIDE32, KERNEL_PRUNED, KERNEL_SPARSE, KERNEL_SPARSE_BLOCK,
+ KERNEL_PACKED16_BLOCK) = (k << 8 for k in range(7))
 KERNEL_MASK = 15 << 8
 TILE_FLAGS = {0: 0 << 12, 4: 1 << 12, 8: 2 << 12, 16: 3 << 12}
 OK, E_INVALID_ARG, E_UNSUPPORTED_SIZE, E_WORKSPACE_TOO_SMALL, E_CUDA = 0, -1, -2, -3, -4

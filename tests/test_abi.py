@@ -115,10 +115,10 @@ def test_kernel_choice_is_part_of_the_problem_flags(S):
     n = ctypes.c_size_t()
     base = S.themis_workspace_bytes(_good(S), False)
     for kernel in (S.KERNEL_DEFAULT, S.KERNEL_PACKED16, S.KERNEL_WIDE32, S.KERNEL_PRUNED, S.KERNEL_SPARSE,
-                   S.KERNEL_SPARSE_BLOCK):
+                   S.KERNEL_SPARSE_BLOCK, S.KERNEL_PACKED16_BLOCK):
         for tile in (0, 4, 8, 16):
             assert S.themis_workspace_bytes(_good(S, flags=1 | kernel | S.TILE_FLAGS[tile]), False) == base
-    for flags in (6 << 8, 15 << 8, 1 << 14, 2, 1 << 31):
+    for flags in (7 << 8, 15 << 8, 1 << 14, 2, 1 << 31):
         assert S._lib.themis_workspace_bytes(ctypes.byref(_good(S, flags=flags)), 0, ctypes.byref(n)) == S.E_INVALID_ARG
 
 

@@ -12,7 +12,7 @@ from tests.test_gpu_parity import SHAPES, _assert_results_equal
 
 pytestmark = pytest.mark.gpu
 
-KERNEL_IDS = ["packed16", "wide32", "pruned", "sparse", "sparse_block"]
+KERNEL_IDS = ["packed16", "wide32", "pruned", "sparse", "sparse_block", "packed16_block"]
 
 
 @pytest.fixture(scope="module")
@@ -40,7 +40,7 @@ def _checked_solve(S, wl, kernel_id):
     return {k: v.cpu().numpy() for k, v in out.items()}
 
 
-@pytest.mark.parametrize("kernel_id", range(5), ids=KERNEL_IDS)
+@pytest.mark.parametrize("kernel_id", range(6), ids=KERNEL_IDS)
 def test_edge_shapes_raise_no_violation(S, oracle_mod, kernel_id):
     for shape in SHAPES:
         n_stages, c_max, batches, h_max, T, bucket_us, vertical, (lo, hi) = shape
@@ -49,7 +49,7 @@ def test_edge_shapes_raise_no_violation(S, oracle_mod, kernel_id):
         _assert_results_equal(_checked_solve(S, wl, kernel_id), oracle_mod.solve_batch(wl))
 
 
-@pytest.mark.parametrize("kernel_id", range(5), ids=KERNEL_IDS)
+@pytest.mark.parametrize("kernel_id", range(6), ids=KERNEL_IDS)
 def test_budget_lengths_and_stage_counts_raise_no_violation(S, oracle_mod, kernel_id):
     for T in (1, 2, 31, 32, 33, 127, 128, 131, 135, 136, 255, 256, 257, 263, 264, 511, 512, 1024, 1031, 2047, 2048,
               2049, 2055, 2056):
@@ -64,7 +64,7 @@ def test_budget_lengths_and_stage_counts_raise_no_violation(S, oracle_mod, kerne
     _assert_results_equal(_checked_solve(S, wl, kernel_id), oracle_mod.solve_batch(wl))
 
 
-@pytest.mark.parametrize("kernel_id", range(5), ids=KERNEL_IDS)
+@pytest.mark.parametrize("kernel_id", range(6), ids=KERNEL_IDS)
 def test_benchmark_shapes_raise_no_violation(S, oracle_mod, kernel_id):
     """Subsets of the benchmark configurations (the launch shapes the benchmark times)."""
     for cfg, n in ((1, 64), (2, 64), (3, 96), (4, 8), (5, 2)):

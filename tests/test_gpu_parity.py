@@ -63,12 +63,14 @@ def _assert_results_equal(gpu, ref, idx=None):
                                            + _diagnose(gpu, ref, idx))
 
 
-# kernel under test: 0 packed 16-bit (the default), 1 32-bit, 2 pruned, 3 sparse (one warp per
-# instance, block kernel for what outgrows its lists), 4 sparse block kernel; tile: cells per thread
+# kernel under test: 0 packed 16-bit (the default: one warp per instance for short budgets, else
+# a block), 1 32-bit, 2 pruned, 3 sparse (one warp per instance, block kernel for what outgrows
+# its lists), 4 sparse block kernel, 5 packed 16-bit with a block per instance at any budget;
+# tile: cells per thread
 MODE = {"mode": 0, "tile": 0}
 
 
-@pytest.fixture(params=[0, 1, 2, 3, 4], ids=["packed16", "wide32", "pruned", "sparse", "sparse_block"])
+@pytest.fixture(params=[0, 1, 2, 3, 4, 5], ids=["packed16", "wide32", "pruned", "sparse", "sparse_block", "packed16_block"])
 def mode(request, S):
     MODE["mode"] = request.param
     yield request.param
@@ -80,14 +82,14 @@ def _assert_tables_equal(S, gpu, ref):
     32-bit kernel: A where F_s[t] is reachable (0 elsewhere);
     packed kernel: every prefix table F_s[t], saturated at 0x7FFF, up to the budget the
     later stages can still complete."""
-    if MODE["mode"] >= 3:      # one fused kernel: the workspace holds fronts, not the dense tables
+    if MODE["mode"] in (3, 4): # one fused kernel: the workspace holds fronts, not the dense tables
         return
     assert np.array_equal(gpu["G"], ref["G"])
     assert np.array_equal(gpu["Garg"], ref["Garg"])
     assert (gpu["G_pad"] == S.G_INF).all()
     if MODE["mode"] == 2:      # tables of the restricted problem: only the results are comparable
         return
-    if MODE["mode"] == 0:
+    if MODE["mode"] in (0, 5):
         solved = ref["status"] == 0
         assert np.array_equal(gpu["F"][solved], ref["F"][solved, -1, :])
         assert (ref["F"][ref["F"] != S.G_INF] < S.INF16).all(), "use the saturation test for such inputs"
