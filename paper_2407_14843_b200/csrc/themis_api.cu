@@ -78,6 +78,11 @@ int validate(const themis_problem_t *pr, int vertical, int32_t *T_out, int32_t *
     return THEMIS_OK;
 }
 
+inline size_t list_words_of(const themis_problem_t *pr)
+{
+    return (size_t)kListHeaderWords + 4u * (size_t)pr->c_max * pr->n_batch;
+}
+
 int layout_of(const themis_problem_t *pr, int vertical, themis_workspace_layout_t *L)
 {
     int32_t T, K;
@@ -93,6 +98,8 @@ int layout_of(const themis_problem_t *pr, int vertical, themis_workspace_layout_
     L->flag_offset = off; off = align_up(off + (size_t)pr->n_instances * sizeof(int32_t));
     // behind the tables: instances the sparse warp kernel hands to the block kernel (count, then ids)
     off = align_up(off + ((size_t)pr->n_instances + 1) * sizeof(int32_t));
+    // candidate lists of the scoring kernels: per (profile, stage) a header and one uint4 per (cores, batch size)
+    off = align_up(off + (size_t)pr->n_profiles * pr->n_stages * list_words_of(pr) * sizeof(uint32_t));
     // record of the bounds-checked build (four words)
     off = align_up(off + 4 * sizeof(int32_t));
     L->total_bytes = off;
@@ -125,6 +132,9 @@ int make_params(const themis_problem_t *pr, const SolveOpts &opts, void *ws, siz
     P->redo_count = reinterpret_cast<int32_t *>(base + align_up(L.flag_offset + (size_t)pr->n_instances * sizeof(int32_t)));
     P->redo_list = P->redo_count + 1;
     P->check = reinterpret_cast<int32_t *>(base + L.total_bytes - kAlign);
+    P->list_words = (int32_t)list_words_of(pr);
+    P->lists = reinterpret_cast<uint32_t *>(base + L.total_bytes - kAlign -
+                                            align_up((size_t)pr->n_profiles * pr->n_stages * list_words_of(pr) * sizeof(uint32_t)));
     return THEMIS_OK;
 }
 

@@ -36,6 +36,9 @@ constexpr uint32_t kInf16 = 0x7FFFu;
 // bulk copies of whole rows meet the 16-byte rule.
 constexpr int kRowAlign = 32;
 
+// Words in front of the entries of a scoring list (see score_lists_kernel).
+constexpr int kListHeaderWords = 4;
+
 struct Params {
     themis_problem_t prob;
     int32_t T;          // budget in buckets
@@ -55,6 +58,8 @@ struct Params {
     uint16_t *Garg;
     uint16_t *A;
     int32_t *F;
+    uint32_t *lists;     // scoring: one candidate list per (profile, stage), list_words words each
+    int32_t list_words;
     int32_t *check;      // bounds-checked build: {site of the first violation (0 = none), index, limit, 0}
     int32_t *redo_count; // sparse warp kernel: number of instances handed to the block kernel ...
     int32_t *redo_list;  // ... and their indices [N]

@@ -14,16 +14,20 @@
 // min on the packed word (cost << 16 | candidate index), whose ordering gives
 // "cheapest, then lowest index" directly.
 //
-// A warp task is (one batch size) x (32 consecutive core counts).  Its lanes
-// first take one (c, b) pair each: load the latency, drop the pair if one core
-// fewer has the same latency or if the latency alone exceeds the budget, and
-// round it up to buckets.  Then
-//  - where the queuing delay grows with the replica count (joint problem, flag
-//    THEMIS_QUEUE_PER_REPLICA, b > 1), the surviving pairs are compacted into a
-//    warp-private list and the lanes switch to one replica count each: every
-//    list entry is broadcast and each lane scores its (h, c, b);
+// What depends on the latency table alone is done once per (profile, stage) by a
+// small kernel in front (score_lists_kernel): the (cores, batch size) pairs whose
+// latency differs from the one with a core fewer and fits the budget, with the
+// latency rounded up to buckets, as one list sorted by batch size and cores.  Every
+// instance of the profile reads that list instead of the table.
+//
+// A warp task is 32 consecutive list entries.
+//  - Where the queuing delay grows with the replica count (joint problem, flag
+//    THEMIS_QUEUE_PER_REPLICA, b > 1), the entries of one batch size that can
+//    still fit are compacted into a warp-private list and the lanes switch to one
+//    replica count each: every list entry is broadcast and each lane scores its
+//    (h, c, b);
 //  - elsewhere more replicas only cost more in the same bucket, so each lane
-//    looks up the fewest replicas that sustain lambda for its pair (binary
+//    looks up the fewest replicas that sustain lambda for its entry (binary
 //    search in the Lmax row) and scores that one candidate.
 // Two key rows alternate between stages, so a stage costs one block barrier.
 #include "themis_internal.h"
@@ -100,6 +104,63 @@ __device__ __forceinline__ uint32_t sat_u32(unsigned long long v, uint32_t cap)
     return v > (unsigned long long)cap ? cap : (uint32_t)v;
 }
 
+// One list per (profile, stage): kListHeaderWords words {entries, entries of batch size 1
+// (they come first), 1 if a latency is not positive, 0}, then one uint4 per entry
+// {latency [us], latency in buckets, cores, batch index}, sorted by batch index, then cores.
+// One block per (profile, stage), one warp per batch size.
+__global__ void __launch_bounds__(32 * THEMIS_MAX_BATCH_SIZES)
+score_lists_kernel(const Params p)
+{
+    const int C = p.prob.c_max, NB = p.prob.n_batch, CB = C * NB;
+    const int lane = threadIdx.x & 31, bi = threadIdx.x >> 5;
+    const uint32_t w_us = (uint32_t)p.prob.bucket_us;
+    const int32_t *lat_s = p.lat_us + (size_t)blockIdx.x * CB;
+    uint32_t *hdr = p.lists + (size_t)blockIdx.x * p.list_words;
+    uint4 *entries = reinterpret_cast<uint4 *>(hdr + kListHeaderWords);
+    __shared__ int count[THEMIS_MAX_BATCH_SIZES];
+    __shared__ int bad;
+    if (threadIdx.x == 0) bad = 0;
+    __syncthreads();
+    const uint32_t lanemask_lt = (1u << lane) - 1u;
+    int offset = 0;
+    for (int pass = 0; pass < 2; ++pass) {
+        int n = 0, saw_bad = 0;
+        for (int c0 = 0; c0 < C; c0 += 32) {
+            const int cidx = c0 + lane;               // core count - 1
+            int32_t v = 1, v_prev = 0;
+            if (cidx < C) {
+                v = lat_s[TH_IDX(151, cidx * NB + bi, CB)];
+                v_prev = cidx > 0 ? lat_s[TH_IDX(152, (cidx - 1) * NB + bi, CB)] : 0;
+            }
+            if (v <= 0) saw_bad = 1;
+            // Same latency with one core fewer: that candidate reaches the same buckets with the
+            // same replica counts at a lower cost, so this one is never a minimum (latency
+            // tables are flat over long runs of core counts).
+            const uint32_t l_b = v > 0 ? ((uint32_t)v + w_us - 1u) / w_us : 0u;
+            const bool keep = cidx < C && v > 0 && v != v_prev && l_b <= (uint32_t)p.T;
+            const unsigned kept = __ballot_sync(0xFFFFFFFFu, keep);
+            if (pass == 1 && keep)
+                entries[TH_IDX(153, offset + n + __popc(kept & lanemask_lt), CB)] =
+                    make_uint4((uint32_t)v, l_b, (uint32_t)(cidx + 1), (uint32_t)bi);
+            n += __popc(kept);
+        }
+        if (pass == 0) {
+            if (lane == 0) count[bi] = n;
+            if (saw_bad) bad = 1;
+            __syncthreads();
+            for (int j = 0; j < bi; ++j) offset += count[j];
+            if (threadIdx.x == 0) {
+                int total = 0;
+                for (int j = 0; j < NB; ++j) total += count[j];
+                hdr[0] = (uint32_t)total;
+                hdr[1] = p.prob.batch_sizes[0] == 1 ? (uint32_t)count[0] : 0u;
+                hdr[2] = (uint32_t)bad;
+                hdr[3] = 0u;
+            }
+        }
+    }
+}
+
 // THREADS: 256, or 128 for short budgets, where a stage is so little work that the per-warp
 // cost of a stage (loop, barrier, row addresses) shows; registers for 1536 threads per SM.
 template <int THREADS>
@@ -152,12 +213,7 @@ score_kernel(const Params p)
         *reinterpret_cast<uint4 *>(smem + TH_IDX(124, l4, 2 * pitch - 3)) = make_uint4(kEmptyKey, kEmptyKey, kEmptyKey, kEmptyKey);
     __syncthreads();
     const bool skip_all = s_bad != 0;
-    const int32_t *lat = p.lat_us + (size_t)(skip_all ? 0 : pid) * S * CB;
 
-    // This warp's tasks: (batch index, chunk of 32 core counts) number warp, warp + kScoreWarps, ...
-    const int c_chunks = (C + 31) / 32;
-    const int bi_first = warp / c_chunks, ch_first = warp - bi_first * c_chunks;
-    const int bi_step = kScoreWarps / c_chunks, ch_step = kScoreWarps - bi_step * c_chunks;
     if (!skip_all) {
         const unsigned long long q_den = (unsigned long long)lambda_m * w_us;
         for (int e = tid; e < SV * NB * HN; e += kScoreThreads) {
@@ -178,7 +234,6 @@ score_kernel(const Params p)
     // one candidate per (c, b): q does not depend on h, or only one h is a candidate
     const bool single = !q_grows_with_h || p.horizontal || p.vertical || HN == 1;
     int saw_bad_latency = 0;
-    const uint32_t w_magic = 0xFFFFFFFFu / w_us;            // floor((2^32 - 1) / w)
     // In the list loop the lanes of a warp cover HNp replica counts x (32 / HNp) pairs of entries.
     int hn_log = 1;
     while ((1 << hn_log) < HN && hn_log < 5) ++hn_log;
@@ -193,37 +248,27 @@ score_kernel(const Params p)
         const uint32_t key_addr = smem_addr + 4u * (uint32_t)key_off;
         if (!skip_all) {
             const int h_lo = p.vertical ? rep[s] : 1;
-            const int32_t *lat_s = lat + (size_t)s * CB;
             const int row_s = p.vertical ? s * NB : 0;
-            int bi = bi_first, ch = ch_first;
-            while (bi < NB) {
-                const int cidx = ch * 32 + lane;     // core count - 1
-                const int pair = cidx * NB + bi;
-                bool live = cidx < C;
-                uint32_t l_us = 0, l_b = 0;
-                if (live) {
-                    const int32_t v = lat_s[TH_IDX(107, pair, CB)];
-                    const int32_t v_prev = cidx > 0 ? lat_s[TH_IDX(108, pair - NB, CB)] : 0;
-                    if (v <= 0) saw_bad_latency = 1;
-                    // Same latency with one core fewer: that candidate reaches the same buckets with
-                    // the same replica counts at a lower cost, so this one is never a minimum
-                    // (latency tables are flat over long runs of core counts).
-                    live = v > 0 && v != v_prev;
-                    l_us = (uint32_t)v;
-                    // l_b = ceil(l_us / w): the reciprocal's quotient is at most one too small
-                    uint32_t l_q = __umulhi(l_us, w_magic);
-                    uint32_t l_r = l_us - l_q * w_us;
-                    if (l_r >= w_us) { l_r -= w_us; ++l_q; }
-                    if (l_r >= w_us) { l_r -= w_us; ++l_q; }
-                    l_b = l_q + (l_r != 0u);
-                    live = live && l_b <= (uint32_t)T;
-                }
-                const int q_row = q_off + (row_s + bi) * HN;
-                const int lmax_row = lmax_off + (row_s + bi) * HN;
-                if (single || p.prob.batch_sizes[bi] == 1) {
+            const uint32_t *hdr = p.lists + ((size_t)pid * S + s) * p.list_words;
+            const int n_entries = (int)hdr[0];
+            // entries with one candidate each: all of them, or those of batch size 1 (no queue)
+            const int n_single = single ? n_entries : (int)hdr[1];
+            saw_bad_latency |= (int)hdr[2];
+            const uint4 *entries = reinterpret_cast<const uint4 *>(hdr + kListHeaderWords);
+            const int nt_joint = (n_entries - n_single + 31) >> 5;
+            const int nt_single = (n_single + 31) >> 5;
+            for (int t = warp; t < nt_joint + nt_single; t += kScoreWarps) {
+                const int t_now = t;
+                if (t_now >= nt_joint) {
                     // More replicas only cost more in the same bucket: the fewest replicas that
-                    // sustain lambda (feasibility is monotone in h) are the pair's one candidate.
-                    if (live) {
+                    // sustain lambda (feasibility is monotone in h) are the entry's one candidate.
+                    const int e = 32 * (t_now - nt_joint) + lane;
+                    if (e < n_single) {
+                        const uint4 en = entries[TH_IDX(107, e, CB)];
+                        const uint32_t l_us = en.x, l_b = en.y;
+                        const int cidx = (int)en.z - 1, bi = (int)en.w;
+                        const int q_row = q_off + (row_s + bi) * HN;
+                        const int lmax_row = lmax_off + (row_s + bi) * HN;
                         int lo = 0, cnt = HN;
                         if (HN == 1) {                       // vertical variant: the one replica count
                             lo = smem[TH_IDX(109, lmax_row, list_base)] < l_us ? 1 : 0;
@@ -238,7 +283,7 @@ score_kernel(const Params p)
                             const uint32_t ell = l_b + smem[TH_IDX(111, q_row + lo, lmax_off)];
                             if (ell <= (uint32_t)T) {
                                 const uint32_t cost = (uint32_t)(h_lo + lo) * (uint32_t)(cidx + 1);
-                                const uint32_t idx = (uint32_t)((p.horizontal ? 0 : lo * CB) + pair);
+                                const uint32_t idx = (uint32_t)((p.horizontal ? 0 : lo * CB) + cidx * NB + bi);
 #ifdef THEMIS_CHECK_BOUNDS
                                 atomicMin(&smem[TH_IDX(112, key_off + (int)ell, key_off + pitch)], (cost << 16) | idx);
 #else
@@ -247,10 +292,23 @@ score_kernel(const Params p)
                             }
                         }
                     }
-                } else {
-                    // Joint problem with h_max >= 2 (so c <= 32767: at most 65535 candidates per stage).
+                    continue;
+                }
+                // Joint problem with h_max >= 2 (so c <= 32767: at most 65535 candidates per stage).
+                const int e = n_single + 32 * t_now + lane;
+                const bool valid = e < n_entries;
+                uint4 en = make_uint4(0u, 0u, 0u, 0u);
+                if (valid) en = entries[TH_IDX(108, e, CB)];
+                const uint32_t l_us = en.x, l_b = en.y;
+                unsigned rest = __ballot_sync(0xFFFFFFFFu, valid);
+                while (rest != 0u) {                         // one round per batch size among the 32 entries
+                    const int bi = (int)__shfl_sync(0xFFFFFFFFu, en.w, __ffs((int)rest) - 1);
+                    const bool live = valid && (int)en.w == bi;
+                    rest &= ~__ballot_sync(0xFFFFFFFFu, live);
+                    const int q_row = q_off + (row_s + bi) * HN;
+                    const int lmax_row = lmax_off + (row_s + bi) * HN;
                     for (int h0 = 0; h0 < HN; h0 += HNp) {
-                        // pairs that still fit the budget at this chunk's first replica count ...
+                        // entries that still fit the budget at this chunk's first replica count ...
                         const bool fits = live && l_b + smem[TH_IDX(113, q_row + h0, lmax_off)] <= (uint32_t)T;
                         if (__ballot_sync(0xFFFFFFFFu, fits) == 0u) break;     // q never shrinks with h
                         // ... and sustain lambda at its last
@@ -262,7 +320,7 @@ score_kernel(const Params p)
                             *reinterpret_cast<uint2 *>(smem + TH_IDX(115, list_off + 2 * lane, smem_words - 1)) = make_uint2(kNeverFits, 0u);
                         if (in)
                             *reinterpret_cast<uint2 *>(smem + TH_IDX(116, list_off + 2 * __popc(mask & lanemask_lt), smem_words - 1)) =
-                                make_uint2(l_us, (l_b << 2) | ((uint32_t)(cidx + 1) << 17));
+                                make_uint2(l_us, (l_b << 2) | (en.z << 17));
                         __syncwarp();
                         const int k = h0 + hk;                       // this lane's replica count - 1
                         const bool kv = k < HN;
@@ -277,15 +335,13 @@ score_kernel(const Params p)
                                                       4u * (uint32_t)T, key_mul, key_add, key_off,
                                                       list_base + kScoreWarps * kListWords + lane);
 #else
-                        uint32_t entries = list_addr;
-                        for (int i = 0; i < cnt; i += 2 * groups, entries += 16u * (uint32_t)groups)
-                            score_two_entries(entries, q4, lmax, 4u * (uint32_t)T, key_mul, key_add, key_addr, idle_addr);
+                        uint32_t entries_addr = list_addr;
+                        for (int i = 0; i < cnt; i += 2 * groups, entries_addr += 16u * (uint32_t)groups)
+                            score_two_entries(entries_addr, q4, lmax, 4u * (uint32_t)T, key_mul, key_add, key_addr, idle_addr);
 #endif
                         __syncwarp();
                     }
                 }
-                bi += bi_step; ch += ch_step;
-                if (ch >= c_chunks) { ch -= c_chunks; ++bi; }
             }
         }
         __syncthreads();
@@ -327,6 +383,9 @@ cudaError_t launch_score(const Params &p, cudaStream_t stream)
     auto kernel = threads == 128 ? score_kernel<128> : score_kernel<256>;
     static std::atomic<uint64_t> ready128{0}, ready256{0};
     cudaError_t e = allow_max_smem(reinterpret_cast<const void *>(kernel), threads == 128 ? ready128 : ready256);
+    if (e != cudaSuccess) return e;
+    score_lists_kernel<<<p.prob.n_profiles * p.prob.n_stages, 32 * p.prob.n_batch, 0, stream>>>(p);
+    e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     kernel<<<p.prob.n_instances, threads, smem, stream>>>(p);
     return cudaGetLastError();
