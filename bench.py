@@ -574,7 +574,8 @@ def run_ours(args):
     N_total = wl.n_instances * world if not strong else wl_all.n_instances
     # score + min-plus, plus the 32-bit second pass where a total may exceed 15 bits
     second_pass = packed and (wl.vertical or wl.n_stages * wl.h_max * wl.c_max >= 0x7FFF)
-    launches_per_step = 3 if second_pass else 2
+    # score_lists_kernel + score_kernel + the recurrence kernel (+ the 32-bit pass over flagged instances)
+    launches_per_step = 4 if second_pass else 3
     cells_per_launch = wl.n_instances * wl.minplus_cells
     main_r = dense_rooflines(wl, main, packed, probe, counts)
     kernel_name = ("minplus16_warp_kernel" if wl.T + 1 <= 1100 and args.minplus_tile != 16 else "minplus16_kernel") \

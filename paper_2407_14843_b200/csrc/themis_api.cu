@@ -80,7 +80,7 @@ int validate(const themis_problem_t *pr, int vertical, int32_t *T_out, int32_t *
 
 inline size_t list_words_of(const themis_problem_t *pr)
 {
-    return (size_t)kListHeaderWords + 4u * (size_t)pr->c_max * pr->n_batch;
+    return (size_t)score_list_layout(pr->c_max, pr->n_batch).words;
 }
 
 int layout_of(const themis_problem_t *pr, int vertical, themis_workspace_layout_t *L)
@@ -132,7 +132,6 @@ int make_params(const themis_problem_t *pr, const SolveOpts &opts, void *ws, siz
     P->redo_count = reinterpret_cast<int32_t *>(base + align_up(L.flag_offset + (size_t)pr->n_instances * sizeof(int32_t)));
     P->redo_list = P->redo_count + 1;
     P->check = reinterpret_cast<int32_t *>(base + L.total_bytes - kAlign);
-    P->list_words = (int32_t)list_words_of(pr);
     P->lists = reinterpret_cast<uint32_t *>(base + L.total_bytes - kAlign -
                                             align_up((size_t)pr->n_profiles * pr->n_stages * list_words_of(pr) * sizeof(uint32_t)));
     return THEMIS_OK;

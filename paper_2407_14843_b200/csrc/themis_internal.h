@@ -36,8 +36,28 @@ constexpr uint32_t kInf16 = 0x7FFFu;
 // bulk copies of whole rows meet the 16-byte rule.
 constexpr int kRowAlign = 32;
 
-// Words in front of the entries of a scoring list (see score_lists_kernel).
-constexpr int kListHeaderWords = 4;
+// Candidate list of one (profile, stage), built by score_lists_kernel and read by score_kernel,
+// in 32-bit words:
+//   [0] entries  [1] entries of batch size 1 (they come first)  [2] 1 if a latency is not positive
+//   [3] joint tasks
+//   [4 ..)       uint4 per joint task {batch index | first joint entry << 4 | entries << 24,
+//                smallest latency of that batch size in buckets, the same in us, 0}
+//   [single ..)  uint4 per entry {latency [us], latency in buckets, cores, batch index}, sorted by
+//                batch index, then cores
+//   [joint ..)   uint2 per entry {latency [us], latency in buckets << 2 | cores << 17}, the same
+//                order, every batch size padded with entries that never fit to a multiple of the
+//                entries one pass of the scoring loop takes (at most 32)
+struct ScoreListLayout { int tasks, single, joint, words; };
+__host__ __device__ inline ScoreListLayout score_list_layout(int c_max, int n_batch)
+{
+    ScoreListLayout L;
+    const int CB = c_max * n_batch;
+    L.tasks = 4;
+    L.single = L.tasks + 4 * n_batch * (c_max / 32 + 2);
+    L.joint = L.single + 4 * CB;
+    L.words = (L.joint + 2 * (CB + 32 * n_batch) + 3) & ~3;   // every list starts 16-byte aligned
+    return L;
+}
 
 struct Params {
     themis_problem_t prob;
@@ -58,8 +78,7 @@ struct Params {
     uint16_t *Garg;
     uint16_t *A;
     int32_t *F;
-    uint32_t *lists;     // scoring: one candidate list per (profile, stage), list_words words each
-    int32_t list_words;
+    uint32_t *lists;     // scoring: candidate lists per (profile, stage), score_list_layout().words words each
     int32_t *check;      // bounds-checked build: {site of the first violation (0 = none), index, limit, 0}
     int32_t *redo_count; // sparse warp kernel: number of instances handed to the block kernel ...
     int32_t *redo_list;  // ... and their indices [N]

@@ -17,18 +17,16 @@
 // What depends on the latency table alone is done once per (profile, stage) by a
 // small kernel in front (score_lists_kernel): the (cores, batch size) pairs whose
 // latency differs from the one with a core fewer and fits the budget, with the
-// latency rounded up to buckets, as one list sorted by batch size and cores.  Every
-// instance of the profile reads that list instead of the table.
-//
-// A warp task is 32 consecutive list entries.
+// latency rounded up to buckets, as lists sorted by batch size and cores, cut into
+// warp tasks.  Every instance of the profile reads the lists instead of the table.
 //  - Where the queuing delay grows with the replica count (joint problem, flag
-//    THEMIS_QUEUE_PER_REPLICA, b > 1), the entries of one batch size that can
-//    still fit are compacted into a warp-private list and the lanes switch to one
-//    replica count each: every list entry is broadcast and each lane scores its
-//    (h, c, b);
-//  - elsewhere more replicas only cost more in the same bucket, so each lane
-//    looks up the fewest replicas that sustain lambda for its entry (binary
-//    search in the Lmax row) and scores that one candidate.
+//    THEMIS_QUEUE_PER_REPLICA, b > 1), a task is up to 32 entries of one batch
+//    size; the lanes take one replica count each, every entry is read by all of
+//    them (one 16-byte load brings two) and each lane scores its (h, c, b);
+//  - elsewhere more replicas only cost more in the same bucket, so a task is 32
+//    entries, one per lane, and each lane looks up the fewest replicas that
+//    sustain lambda for its entry (binary search in the Lmax row) and scores
+//    that one candidate.
 // Two key rows alternate between stages, so a stage costs one block barrier.
 #include "themis_internal.h"
 
@@ -45,10 +43,11 @@ __device__ __forceinline__ void red_min_shared(uint32_t addr, uint32_t v)
     asm volatile("red.shared.min.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 
-// Two list entries {latency [us], 4 * l_b | c << 17} at `entries` against this lane's replica
-// count: q4 = 4 * Q[b][h], lmax = Lmax[b][h], key = c * key_mul + key_add.  A lane whose
-// candidate is infeasible or over budget sends its word to `idle` (a word nobody reads), so
-// the reduction itself is unconditional and the loop body has no branch.
+// Two list entries {latency [us], 4 * l_b | c << 17} at `entries` (shared memory, 16-byte
+// aligned) against this lane's replica count: q4 = 4 * Q[b][h], lmax = Lmax[b][h],
+// key = c * key_mul + key_add.  A lane whose candidate is infeasible or over budget sends
+// its word to `idle` (a word nobody reads), so the reduction itself is unconditional and
+// the loop body has no branch.
 __device__ __forceinline__ void score_two_entries(uint32_t entries, uint32_t q4, uint32_t lmax, uint32_t t4,
                                                   uint32_t key_mul, uint32_t key_add, uint32_t keys,
                                                   uint32_t idle)
@@ -104,27 +103,41 @@ __device__ __forceinline__ uint32_t sat_u32(unsigned long long v, uint32_t cap)
     return v > (unsigned long long)cap ? cap : (uint32_t)v;
 }
 
-// One list per (profile, stage): kListHeaderWords words {entries, entries of batch size 1
-// (they come first), 1 if a latency is not positive, 0}, then one uint4 per entry
-// {latency [us], latency in buckets, cores, batch index}, sorted by batch index, then cores.
-// One block per (profile, stage), one warp per batch size.
+// In the joint loop the lanes of a warp cover 2^hn_log replica counts x (32 >> hn_log) entry
+// pairs at a time.
+__host__ __device__ inline int joint_hn_log(int HN)
+{
+    int hn_log = 1;
+    while ((1 << hn_log) < HN && hn_log < 5) ++hn_log;
+    return hn_log;
+}
+
+// Builds the candidate lists of one (profile, stage) (layout: score_list_layout).  One block
+// per (profile, stage), one warp per batch size.
 __global__ void __launch_bounds__(32 * THEMIS_MAX_BATCH_SIZES)
-score_lists_kernel(const Params p)
+score_lists_kernel(const Params p, int joint_lists)
 {
     const int C = p.prob.c_max, NB = p.prob.n_batch, CB = C * NB;
     const int lane = threadIdx.x & 31, bi = threadIdx.x >> 5;
     const uint32_t w_us = (uint32_t)p.prob.bucket_us;
     const int32_t *lat_s = p.lat_us + (size_t)blockIdx.x * CB;
-    uint32_t *hdr = p.lists + (size_t)blockIdx.x * p.list_words;
-    uint4 *entries = reinterpret_cast<uint4 *>(hdr + kListHeaderWords);
-    __shared__ int count[THEMIS_MAX_BATCH_SIZES];
+    const ScoreListLayout L = score_list_layout(C, NB);
+    uint32_t *hdr = p.lists + (size_t)blockIdx.x * L.words;
+    uint4 *single = reinterpret_cast<uint4 *>(hdr + L.single);
+    uint2 *joint = reinterpret_cast<uint2 *>(hdr + L.joint);
+    const int joint_cap = CB + 32 * NB;
+    (void)joint_cap;
+    // entries one pass of the joint loop takes: 2 per group of lanes
+    const int M = joint_lists ? 64 >> joint_hn_log(p.prob.h_max) : 1;
+    __shared__ int count[THEMIS_MAX_BATCH_SIZES], padded[THEMIS_MAX_BATCH_SIZES], n_task[THEMIS_MAX_BATCH_SIZES];
     __shared__ int bad;
     if (threadIdx.x == 0) bad = 0;
     __syncthreads();
     const uint32_t lanemask_lt = (1u << lane) - 1u;
-    int offset = 0;
+    int off_single = 0, off_joint = 0, off_task = 0;
     for (int pass = 0; pass < 2; ++pass) {
         int n = 0, saw_bad = 0;
+        uint32_t min_lb = 0xFFFFFFFFu, min_lus = 0xFFFFFFFFu;
         for (int c0 = 0; c0 < C; c0 += 32) {
             const int cidx = c0 + lane;               // core count - 1
             int32_t v = 1, v_prev = 0;
@@ -139,32 +152,59 @@ score_lists_kernel(const Params p)
             const uint32_t l_b = v > 0 ? ((uint32_t)v + w_us - 1u) / w_us : 0u;
             const bool keep = cidx < C && v > 0 && v != v_prev && l_b <= (uint32_t)p.T;
             const unsigned kept = __ballot_sync(0xFFFFFFFFu, keep);
-            if (pass == 1 && keep)
-                entries[TH_IDX(153, offset + n + __popc(kept & lanemask_lt), CB)] =
-                    make_uint4((uint32_t)v, l_b, (uint32_t)(cidx + 1), (uint32_t)bi);
+            if (keep) {
+                min_lb = min(min_lb, l_b);
+                min_lus = min(min_lus, (uint32_t)v);
+                if (pass == 1) {
+                    const int at = n + __popc(kept & lanemask_lt);
+                    single[TH_IDX(153, off_single + at, CB)] = make_uint4((uint32_t)v, l_b, (uint32_t)(cidx + 1), (uint32_t)bi);
+                    if (joint_lists)
+                        joint[TH_IDX(154, off_joint + at, joint_cap)] = make_uint2((uint32_t)v, (l_b << 2) | ((uint32_t)(cidx + 1) << 17));
+                }
+            }
             n += __popc(kept);
         }
         if (pass == 0) {
-            if (lane == 0) count[bi] = n;
+            if (lane == 0) {
+                count[bi] = n;
+                padded[bi] = joint_lists ? (n + M - 1) / M * M : 0;
+                // batch size 1 has no queue: its entries go the one-candidate way
+                n_task[bi] = joint_lists && p.prob.batch_sizes[bi] != 1 ? (padded[bi] + 31) / 32 : 0;
+            }
             if (saw_bad) bad = 1;
             __syncthreads();
-            for (int j = 0; j < bi; ++j) offset += count[j];
-            if (threadIdx.x == 0) {
-                int total = 0;
-                for (int j = 0; j < NB; ++j) total += count[j];
-                hdr[0] = (uint32_t)total;
-                hdr[1] = p.prob.batch_sizes[0] == 1 ? (uint32_t)count[0] : 0u;
-                hdr[2] = (uint32_t)bad;
-                hdr[3] = 0u;
+            for (int j = 0; j < bi; ++j) { off_single += count[j]; off_joint += padded[j]; off_task += n_task[j]; }
+        } else {
+            min_lb = __reduce_min_sync(0xFFFFFFFFu, min_lb);
+            min_lus = __reduce_min_sync(0xFFFFFFFFu, min_lus);
+            // entries that never fit behind the last one, up to the padded count
+            if (lane < padded[bi] - n)
+                joint[TH_IDX(155, off_joint + n + lane, joint_cap)] = make_uint2(kNeverFits, 0u);
+            // this batch size's tasks: equal shares, whole passes of the loop
+            const int nt = n_task[bi];
+            if (lane < nt) {
+                const int share = ((padded[bi] + nt - 1) / nt + M - 1) / M * M;
+                const int first = lane * share;
+                const int len = max(0, min(share, padded[bi] - first));
+                reinterpret_cast<uint4 *>(hdr + L.tasks)[TH_IDX(156, off_task + lane, (L.single - L.tasks) / 4)] =
+                    make_uint4((uint32_t)bi | ((uint32_t)(off_joint + first) << 4) | ((uint32_t)len << 24), min_lb, min_lus, 0u);
             }
         }
+    }
+    if (threadIdx.x == 0) {
+        int total = 0, tasks = 0;
+        for (int j = 0; j < NB; ++j) { total += count[j]; tasks += n_task[j]; }
+        hdr[0] = (uint32_t)total;
+        hdr[1] = p.prob.batch_sizes[0] == 1 ? (uint32_t)count[0] : 0u;
+        hdr[2] = (uint32_t)bad;
+        hdr[3] = (uint32_t)tasks;
     }
 }
 
 // THREADS: 256, or 128 for short budgets, where a stage is so little work that the per-warp
 // cost of a stage (loop, barrier, row addresses) shows; registers for 1536 threads per SM.
 template <int THREADS>
-__global__ void __launch_bounds__(THREADS, 1536 / THREADS)
+__global__ void __launch_bounds__(THREADS, 1280 / THREADS)
 score_kernel(const Params p)
 {
     constexpr int kScoreThreads = THREADS, kScoreWarps = THREADS / 32;
@@ -187,10 +227,11 @@ score_kernel(const Params p)
     const int lmax_off = q_off + SV * NB * HN;
     const int list_base = (lmax_off + SV * NB * HN + 3) & ~3;
     const int list_off = list_base + warp * kListWords;
-    const int smem_words = list_base + kScoreWarps * kListWords + 32;   // what the launch provides
+    const int idle_off = list_base + kScoreWarps * kListWords;
+    const int smem_words = idle_off + 32;           // what the launch provides
     (void)smem_words;
     const uint32_t smem_addr = (uint32_t)__cvta_generic_to_shared(smem);
-    const uint32_t idle_addr = smem_addr + 4u * (uint32_t)(list_base + kScoreWarps * kListWords + lane);
+    const uint32_t idle_addr = smem_addr + 4u * (uint32_t)(idle_off + lane);
     __shared__ int s_bad;
 
     const uint32_t lambda_m = p.lambda_mrps[TH_IDX(101, n, p.prob.n_instances)];
@@ -234,13 +275,12 @@ score_kernel(const Params p)
     // one candidate per (c, b): q does not depend on h, or only one h is a candidate
     const bool single = !q_grows_with_h || p.horizontal || p.vertical || HN == 1;
     int saw_bad_latency = 0;
-    // In the list loop the lanes of a warp cover HNp replica counts x (32 / HNp) pairs of entries.
-    int hn_log = 1;
-    while ((1 << hn_log) < HN && hn_log < 5) ++hn_log;
+    // In the joint loop the lanes of a warp cover HNp replica counts x (32 / HNp) pairs of entries.
+    const int hn_log = joint_hn_log(HN);
     const int HNp = 1 << hn_log;
     const int groups = 32 >> hn_log;
     const int group = lane >> hn_log, hk = lane & (HNp - 1);
-    const uint32_t lanemask_lt = (1u << lane) - 1u;
+    const ScoreListLayout LL = score_list_layout(C, NB);
     const uint32_t list_addr = smem_addr + 4u * (uint32_t)list_off + 16u * (uint32_t)group;
 
     for (int s = 0; s < S; ++s) {
@@ -249,20 +289,23 @@ score_kernel(const Params p)
         if (!skip_all) {
             const int h_lo = p.vertical ? rep[s] : 1;
             const int row_s = p.vertical ? s * NB : 0;
-            const uint32_t *hdr = p.lists + ((size_t)pid * S + s) * p.list_words;
+            const uint32_t *hdr = p.lists + ((size_t)pid * S + s) * LL.words;
             const int n_entries = (int)hdr[0];
             // entries with one candidate each: all of them, or those of batch size 1 (no queue)
             const int n_single = single ? n_entries : (int)hdr[1];
             saw_bad_latency |= (int)hdr[2];
-            const uint4 *entries = reinterpret_cast<const uint4 *>(hdr + kListHeaderWords);
-            const int nt_joint = (n_entries - n_single + 31) >> 5;
+            const int nt_joint = single ? 0 : (int)hdr[3];
             const int nt_single = (n_single + 31) >> 5;
+            const uint4 *entries = reinterpret_cast<const uint4 *>(hdr + LL.single);
+            const uint2 *joint = reinterpret_cast<const uint2 *>(hdr + LL.joint);
+            const uint4 *task_recs = reinterpret_cast<const uint4 *>(hdr + LL.tasks);
+            uint4 recs = make_uint4(0u, 0u, 0u, 0u);         // joint tasks: this warp's next 32 task records, one per lane
+            uint2 ahead = make_uint2(kNeverFits, 0u);        // this lane's entry of the task about to start
             for (int t = warp; t < nt_joint + nt_single; t += kScoreWarps) {
-                const int t_now = t;
-                if (t_now >= nt_joint) {
+                if (t >= nt_joint) {
                     // More replicas only cost more in the same bucket: the fewest replicas that
                     // sustain lambda (feasibility is monotone in h) are the entry's one candidate.
-                    const int e = 32 * (t_now - nt_joint) + lane;
+                    const int e = 32 * (t - nt_joint) + lane;
                     if (e < n_single) {
                         const uint4 en = entries[TH_IDX(107, e, CB)];
                         const uint32_t l_us = en.x, l_b = en.y;
@@ -294,54 +337,53 @@ score_kernel(const Params p)
                     }
                     continue;
                 }
-                // Joint problem with h_max >= 2 (so c <= 32767: at most 65535 candidates per stage).
-                const int e = n_single + 32 * t_now + lane;
-                const bool valid = e < n_entries;
-                uint4 en = make_uint4(0u, 0u, 0u, 0u);
-                if (valid) en = entries[TH_IDX(108, e, CB)];
-                const uint32_t l_us = en.x, l_b = en.y;
-                unsigned rest = __ballot_sync(0xFFFFFFFFu, valid);
-                while (rest != 0u) {                         // one round per batch size among the 32 entries
-                    const int bi = (int)__shfl_sync(0xFFFFFFFFu, en.w, __ffs((int)rest) - 1);
-                    const bool live = valid && (int)en.w == bi;
-                    rest &= ~__ballot_sync(0xFFFFFFFFu, live);
-                    const int q_row = q_off + (row_s + bi) * HN;
-                    const int lmax_row = lmax_off + (row_s + bi) * HN;
-                    for (int h0 = 0; h0 < HN; h0 += HNp) {
-                        // entries that still fit the budget at this chunk's first replica count ...
-                        const bool fits = live && l_b + smem[TH_IDX(113, q_row + h0, lmax_off)] <= (uint32_t)T;
-                        if (__ballot_sync(0xFFFFFFFFu, fits) == 0u) break;     // q never shrinks with h
-                        // ... and sustain lambda at its last
-                        const bool in = fits && l_us <= smem[TH_IDX(114, lmax_row + min(h0 + HNp, HN) - 1, list_base)];
-                        const uint32_t mask = __ballot_sync(0xFFFFFFFFu, in);
-                        const int cnt = __popc(mask);
-                        // compacted entries first; the other slots hold a latency no replica count sustains
-                        if (lane >= cnt)
-                            *reinterpret_cast<uint2 *>(smem + TH_IDX(115, list_off + 2 * lane, smem_words - 1)) = make_uint2(kNeverFits, 0u);
-                        if (in)
-                            *reinterpret_cast<uint2 *>(smem + TH_IDX(116, list_off + 2 * __popc(mask & lanemask_lt), smem_words - 1)) =
-                                make_uint2(l_us, (l_b << 2) | (en.z << 17));
-                        __syncwarp();
-                        const int k = h0 + hk;                       // this lane's replica count - 1
-                        const bool kv = k < HN;
-                        const uint32_t q4 = 4u * (kv ? smem[TH_IDX(117, q_row + k, lmax_off)] : (uint32_t)T + 1u);
-                        const uint32_t lmax = kv ? smem[TH_IDX(118, lmax_row + k, list_base)] : 0u;
-                        // key = (h * c) << 16 | (h - 1) * CB + (c - 1) * NB + bi  =  c * key_mul + key_add
-                        const uint32_t key_mul = ((uint32_t)(k + 1) << 16) + (uint32_t)NB;
-                        const uint32_t key_add = (uint32_t)(k * CB - NB + bi);
-#ifdef THEMIS_CHECK_BOUNDS
-                        for (int i = 0; i < cnt; i += 2 * groups)
-                            score_two_entries_checked(p, smem, smem_words, list_off + 4 * group + 2 * i, q4, lmax,
-                                                      4u * (uint32_t)T, key_mul, key_add, key_off,
-                                                      list_base + kScoreWarps * kListWords + lane);
-#else
-                        uint32_t entries_addr = list_addr;
-                        for (int i = 0; i < cnt; i += 2 * groups, entries_addr += 16u * (uint32_t)groups)
-                            score_two_entries(entries_addr, q4, lmax, 4u * (uint32_t)T, key_mul, key_add, key_addr, idle_addr);
-#endif
-                        __syncwarp();
-                    }
+                // Joint problem with h_max >= 2 (so c <= 32767: at most 65535 candidates per stage):
+                // one batch size, lanes over replica counts.  The task's entries come to the
+                // warp's list in shared memory, the next task's are on their way meanwhile.
+                const int j = (t - warp) / kScoreWarps;      // this warp's j-th task of the stage
+                if ((j & 31) == 0) {                         // lane i: the record of task j + i
+                    const int tj = t + lane * kScoreWarps;
+                    recs = tj < nt_joint ? task_recs[TH_IDX(113, tj, (LL.single - LL.tasks) / 4)] : make_uint4(0u, 0u, 0u, 0u);
+                    const uint32_t task0 = __shfl_sync(0xFFFFFFFFu, recs.x, 0);
+                    const int first0 = (int)((task0 >> 4) & 0xFFFFFu), len0 = (int)(task0 >> 24);
+                    ahead = lane < len0 ? joint[TH_IDX(116, first0 + lane, CB + 32 * NB)] : make_uint2(kNeverFits, 0u);
                 }
+                const uint32_t task = __shfl_sync(0xFFFFFFFFu, recs.x, j & 31);
+                const uint32_t min_lb = __shfl_sync(0xFFFFFFFFu, recs.y, j & 31);
+                const uint32_t min_lus = __shfl_sync(0xFFFFFFFFu, recs.z, j & 31);
+                const int bi = (int)(task & 15u), len = (int)(task >> 24);
+                *reinterpret_cast<uint2 *>(smem + TH_IDX(119, list_off + 2 * lane, smem_words - 1)) = ahead;
+                if (((j + 1) & 31) != 0 && t + kScoreWarps < nt_joint) {
+                    const uint32_t task1 = __shfl_sync(0xFFFFFFFFu, recs.x, (j + 1) & 31);
+                    const int first1 = (int)((task1 >> 4) & 0xFFFFFu), len1 = (int)(task1 >> 24);
+                    ahead = lane < len1 ? joint[TH_IDX(120, first1 + lane, CB + 32 * NB)] : make_uint2(kNeverFits, 0u);
+                }
+                __syncwarp();
+                const int q_row = q_off + (row_s + bi) * HN;
+                const int lmax_row = lmax_off + (row_s + bi) * HN;
+                for (int h0 = 0; h0 < HN; h0 += HNp) {
+                    // no entry fits the budget at this chunk's first replica count: q never shrinks with h
+                    if (min_lb + smem[TH_IDX(114, q_row + h0, lmax_off)] > (uint32_t)T) break;
+                    // no entry sustains lambda at its last
+                    if (min_lus > smem[TH_IDX(115, lmax_row + min(h0 + HNp, HN) - 1, list_base)]) continue;
+                    const int k = h0 + hk;                       // this lane's replica count - 1
+                    const bool kv = k < HN;
+                    const uint32_t q4 = 4u * (kv ? smem[TH_IDX(117, q_row + k, lmax_off)] : (uint32_t)T + 1u);
+                    const uint32_t lmax = kv ? smem[TH_IDX(118, lmax_row + k, list_base)] : 0u;
+                    // key = (h * c) << 16 | (h - 1) * CB + (c - 1) * NB + bi  =  c * key_mul + key_add
+                    const uint32_t key_mul = ((uint32_t)(k + 1) << 16) + (uint32_t)NB;
+                    const uint32_t key_add = (uint32_t)(k * CB - NB + bi);
+#ifdef THEMIS_CHECK_BOUNDS
+                    for (int i = 0; i < len; i += 2 * groups)
+                        score_two_entries_checked(p, smem, smem_words, list_off + 4 * group + 2 * i, q4, lmax,
+                                                  4u * (uint32_t)T, key_mul, key_add, key_off, idle_off + lane);
+#else
+                    uint32_t entries_addr = list_addr;
+                    for (int i = 0; i < len; i += 2 * groups, entries_addr += 16u * (uint32_t)groups)
+                        score_two_entries(entries_addr, q4, lmax, 4u * (uint32_t)T, key_mul, key_add, key_addr, idle_addr);
+#endif
+                }
+                __syncwarp();                                // the list is free for the next task
             }
         }
         __syncthreads();
@@ -384,7 +426,8 @@ cudaError_t launch_score(const Params &p, cudaStream_t stream)
     static std::atomic<uint64_t> ready128{0}, ready256{0};
     cudaError_t e = allow_max_smem(reinterpret_cast<const void *>(kernel), threads == 128 ? ready128 : ready256);
     if (e != cudaSuccess) return e;
-    score_lists_kernel<<<p.prob.n_profiles * p.prob.n_stages, 32 * p.prob.n_batch, 0, stream>>>(p);
+    const bool joint_lists = (p.prob.flags & THEMIS_QUEUE_PER_REPLICA) && !p.horizontal && !p.vertical && p.prob.h_max > 1;
+    score_lists_kernel<<<p.prob.n_profiles * p.prob.n_stages, 32 * p.prob.n_batch, 0, stream>>>(p, joint_lists ? 1 : 0);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     kernel<<<p.prob.n_instances, threads, smem, stream>>>(p);
