@@ -454,7 +454,8 @@ def test_totals_beyond_16_bits_fall_back_to_the_wide_kernel(S, oracle_mod):
     solved = ref["status"] == 0
     assert (solved & (ref["total_cost"] >= S.INF16) & (beyond < S.INF16)).any()
     assert (solved[3::4] & (beyond[3::4] >= S.INF16)).all()
-    _assert_results_equal(_gpu_solve(S, wl, mode=0), ref)
+    _assert_results_equal(_gpu_solve(S, wl, mode=0), ref)     # budget of 420 buckets: one warp per instance
+    _assert_results_equal(_gpu_solve(S, wl, mode=5), ref)     # the same with a block per instance
 
 
 def test_recurrence_step_repeats_on_a_scored_workspace(S, oracle_mod):
@@ -469,7 +470,8 @@ def test_recurrence_step_repeats_on_a_scored_workspace(S, oracle_mod):
     ws = S.alloc_workspace(S.Problem.of_workload(wl), True)
     S.themis_score_batch(S.Problem.of_workload(wl), dev["lat_us"], dev["profile_id"], dev["lambda_mrps"],
                          dev["replicas"], ws)
-    for kernel in (S.KERNEL_PACKED16, S.KERNEL_PACKED16, S.KERNEL_WIDE32, S.KERNEL_PRUNED, S.KERNEL_PACKED16):
+    for kernel in (S.KERNEL_PACKED16, S.KERNEL_PACKED16, S.KERNEL_WIDE32, S.KERNEL_PACKED16_BLOCK, S.KERNEL_PRUNED,
+                   S.KERNEL_PACKED16):
         out = S.alloc_result(wl.n_instances, wl.n_stages)
         for v in out.values():
             v.fill_(-9)
