@@ -52,13 +52,46 @@ HBM_FALLBACK_GBS = 6650.0
 # per instance, no reuse across blocks).  A figure is only reported while the kernel's sources
 # still have the recorded hash.
 NCU_TRAFFIC = {
-    "minplus16": {"config": 4, "bytes_per_instance": (315.842304e6 + 156.111616e6) / 2368,
+    "minplus16": {"config": 4, "bytes_per_instance": (316.776448e6 + 158.014720e6) / 2368,
                   "sources": ("paper_2407_14843_b200/csrc/themis_minplus16.cu",
                               "paper_2407_14843_b200/csrc/themis_minplus16_step.cuh"),
-                  "sha256_16": "1a1de2cc92ace9e8"},
-    "score": {"config": 4, "bytes_per_instance": 0.0,
-              "sources": ("paper_2407_14843_b200/csrc/themis_score.cu",), "sha256_16": "none"},
+                  "sha256_16": "0377121c1eba7f0a"},
+    # score_kernel 2.905 MB read + 399.187 MB written, score_lists_kernel 0.942 MB read, per 2368 instances
+    "score": {"config": 4, "bytes_per_instance": (2.905344e6 + 399.187456e6 + 0.942336e6) / 2368,
+              "sources": ("paper_2407_14843_b200/csrc/themis_score.cu",), "sha256_16": "681354dc7b584f9c"},
 }
+
+# Warp instructions the sparse solver executes per instance (ncu smsp__inst_executed.sum of
+# stage_fronts_kernel + prefix_fronts_kernel on the first instances of a configuration, see
+# profiles/): what its roofline is counted in.  It does no dense table work and moves a few MB,
+# so neither the cell-update rate nor HBM bounds it; instruction issue does (one warp
+# instruction per scheduler and cycle: 148 SMs x 4 schedulers x the SM clock).
+NCU_SPARSE_INSTRUCTIONS = {
+    "sources": ("paper_2407_14843_b200/csrc/themis_front.cu",), "sha256_16": "eb8fa0ae6db90b34",
+    "per_instance": {4: (55839185 + 19486326) / 2368, 3: (117619149 + 44170020) / 9472},
+}
+
+
+def sparse_issue_roofline(cfg: int, instances_per_s: float, sm_mhz: float, sms: int):
+    """Issue-slot roofline of the sparse solver: executed warp instructions per second against
+    one instruction per scheduler and cycle."""
+    import hashlib
+    try:
+        h = hashlib.sha256()
+        for src in NCU_SPARSE_INSTRUCTIONS["sources"]:
+            with open(os.path.join(ROOT, src), "rb") as f:
+                h.update(f.read())
+        if h.hexdigest()[:16] != NCU_SPARSE_INSTRUCTIONS["sha256_16"] or cfg not in NCU_SPARSE_INSTRUCTIONS["per_instance"]:
+            return None
+    except OSError:
+        return None
+    per_instance = NCU_SPARSE_INSTRUCTIONS["per_instance"][cfg]
+    peak = sms * 4 * sm_mhz * 1e6
+    achieved = per_instance * instances_per_s
+    return {"bound": "issue", "achieved": achieved / 1e12, "peak": peak / 1e12, "unit": "T warp instructions/s",
+            "frac": achieved / peak, "warp_instructions_per_instance": per_instance,
+            "peak_kind": f"derived: {sms} SMs x 4 schedulers x {sm_mhz:.0f} MHz (the clock sampled in this run)",
+            "traffic": None}
 
 
 def parse_args():
@@ -559,7 +592,11 @@ def run_ours(args):
                 "ms_per_step": t16["total_ms"] / steps, "instances_per_s": w.n_instances * steps / (t16["total_ms"] * 1e-3),
                 "packed16": dense_rooflines(w, t16, True, probe, cnt),
                 "wide32": dict(dense_rooflines(w, t32, False, probe), same_results=same32),
-                "sparse": {"ms_per_step": sp_ms, "instances_per_s": w.n_instances / (sp_ms * 1e-3), "same_results": same_sp},
+                "sparse": {"ms_per_step": sp_ms, "instances_per_s": w.n_instances / (sp_ms * 1e-3), "same_results": same_sp,
+                           "roofline": sparse_issue_roofline(
+                               cfg, w.n_instances / (sp_ms * 1e-3),
+                               (clocks or {}).get("sm_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0,
+                               torch.cuda.get_device_properties(local_rank).multi_processor_count)},
                 "cell_updates": cnt, "infeasible_instances": int((ref["status"] == 1).sum()),
             }
             del d, wsp, o, ref
@@ -644,6 +681,9 @@ def run_ours(args):
             "ms_per_step": other["total_ms"] / max(1, args.other_kernel_steps), "same_results": other_same,
             "peak_kind": "measured in this run: themis_alu_probe", "traffic": None}
     if pruned is not None:
+        sm_mhz = (clocks or {}).get("sm_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
+        sms = torch.cuda.get_device_properties(local_rank).multi_processor_count
+        pruned["roofline"] = sparse_issue_roofline(args.config, pruned["value"] / world, sm_mhz, sms)
         line["pruned_path"] = pruned
     if sharded_check is not None:
         line["sharded_equals_one_gpu"] = sharded_check
