@@ -179,8 +179,9 @@ typedef struct {
 } themis_workspace_layout_t;
 
 /* Device workspace needed by the d_ entry points for this problem
- * (8 * N * S * row_pitch bytes plus small terms).  vertical != 0 selects the
- * h-fixed variant.  Fails with INVALID_ARG / UNSUPPORTED_SIZE like the solvers. */
+ * (8 * N * S * row_pitch bytes plus small terms, among them the scoring kernels'
+ * candidate lists: about 24 * c_max * n_batch bytes per profile and stage, which is why
+ * n_profiles enters the size).  vertical != 0 selects the h-fixed variant.  Fails with INVALID_ARG / UNSUPPORTED_SIZE like the solvers. */
 int themis_workspace_bytes(const themis_problem_t *problem, int vertical, size_t *out_bytes);
 int themis_workspace_layout(const themis_problem_t *problem, int vertical,
                             themis_workspace_layout_t *out_layout);
@@ -193,7 +194,8 @@ int themis_workspace_layout(const themis_problem_t *problem, int vertical,
  *   d_lambda_mrps  [N] uint32 arrival rate in milli-requests per second, >= 1
  *   out            device result arrays
  *   d_workspace    device scratch, 256-byte aligned, >= themis_workspace_bytes
- * Runs the candidate-scoring kernel, then the min-plus/backtrack kernel.
+ * Runs the candidate-scoring kernels (candidate lists per profile and stage, then the
+ * per-bucket minimum per instance), then the min-plus/backtrack kernel.
  */
 int themis_solve_batch(const themis_problem_t *problem, const int32_t *d_lat_us,
                        const int32_t *d_profile_id, const uint32_t *d_lambda_mrps,

@@ -51,8 +51,8 @@ def test_edge_shapes_raise_no_violation(S, oracle_mod, kernel_id):
 
 @pytest.mark.parametrize("kernel_id", range(6), ids=KERNEL_IDS)
 def test_budget_lengths_and_stage_counts_raise_no_violation(S, oracle_mod, kernel_id):
-    for T in (1, 2, 31, 32, 33, 127, 128, 131, 135, 136, 255, 256, 257, 263, 264, 511, 512, 1024, 1031, 2047, 2048,
-              2049, 2055, 2056):
+    for T in (1, 2, 31, 32, 33, 127, 128, 131, 135, 136, 255, 256, 257, 263, 264, 511, 512, 903, 904, 1024, 1031, 1099,
+              1100, 2047, 2048, 2049, 2055, 2056):
         wl = W.random_tiny_workload(5000 + T, 6, 3, 8, (1, 2, 4), 4, T,
                                     bucket_us=max(1, 400_000 // T) if T < 400 else 1000, rate_lo=20.0, rate_hi=120.0)
         _assert_results_equal(_checked_solve(S, wl, kernel_id), oracle_mod.solve_batch(wl))
@@ -60,6 +60,8 @@ def test_budget_lengths_and_stage_counts_raise_no_violation(S, oracle_mod, kerne
         wl = W.random_tiny_workload(5200 + n_stages, 5, n_stages, 4, (1, 2, 4), 3, 40 * n_stages + 60,
                                     rate_lo=10.0, rate_hi=60.0)
         _assert_results_equal(_checked_solve(S, wl, kernel_id), oracle_mod.solve_batch(wl))
+    wl = W.random_tiny_workload(5300, 12, 64, 4, (1, 2), 3, 700, bucket_us=2000, rate_lo=2.0, rate_hi=30.0)   # 64 stages, short budget
+    _assert_results_equal(_checked_solve(S, wl, kernel_id), oracle_mod.solve_batch(wl))
     wl = W.random_tiny_workload(5100, 2, 3, 16, (1, 2, 4, 8, 16), 8, 16383, bucket_us=100, rate_lo=50.0, rate_hi=400.0)
     _assert_results_equal(_checked_solve(S, wl, kernel_id), oracle_mod.solve_batch(wl))
 

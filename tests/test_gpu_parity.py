@@ -275,7 +275,8 @@ def test_stability_test_of_the_transition_policy(S, oracle_mod):
 
 # ---------------------------------------------------------------- edge cases
 
-@pytest.mark.parametrize("T", [1, 2, 31, 32, 33, 127, 128, 131, 135, 136, 255, 256, 257, 263, 264, 511, 512, 1024, 1031,
+@pytest.mark.parametrize("T", [1, 2, 31, 32, 33, 127, 128, 131, 135, 136, 255, 256, 257, 263, 264, 511, 512, 902, 903, 904,
+                               1024, 1031, 1098, 1099, 1100,        # 903/904: 4 -> 8 cells a tile; 1099/1100: warp -> block kernel
                                2047, 2048, 2049, 2055, 2056])
 def test_budget_lengths_around_tile_boundaries(S, oracle_mod, T, mode):
     wl = W.random_tiny_workload(5000 + T, 6, 3, 8, (1, 2, 4), 4, T, bucket_us=max(1, 400_000 // T) if T < 400 else 1000,
@@ -301,6 +302,24 @@ def test_maximum_budget_length(S, oracle_mod, mode):
 def test_stage_counts(S, oracle_mod, n_stages, mode):
     wl = W.random_tiny_workload(5200 + n_stages, 5, n_stages, 4, (1, 2, 4), 3, 40 * n_stages + 60,
                                 rate_lo=10.0, rate_hi=60.0)
+    ref = oracle_mod.solve_batch(wl, dumps=True)
+    gpu = _gpu_solve(S, wl, tables=True)
+    _assert_tables_equal(S, gpu, ref)
+    _assert_results_equal(gpu, ref)
+
+
+def test_most_stages_on_a_short_budget(S, oracle_mod, mode):
+    """64 stages within 700 buckets: the one-warp-per-instance packed kernel with its per-stage
+    arrays at their largest, on a budget so tight that every instance spends all of it (and a
+    looser one)."""
+    for bucket_us in (2000, 4000):
+        wl = W.random_tiny_workload(5300, 12, 64, 4, (1, 2), 3, 700, bucket_us=bucket_us, rate_lo=2.0, rate_hi=30.0)
+        ref = oracle_mod.solve_batch(wl, dumps=True)
+        assert (ref["status"] == 0).all()
+        gpu = _gpu_solve(S, wl, tables=True)
+        _assert_tables_equal(S, gpu, ref)
+        _assert_results_equal(gpu, ref)
+    wl = W.random_tiny_workload(5300, 12, 64, 4, (1, 2), 3, 700, bucket_us=1000, rate_lo=2.0, rate_hi=30.0)   # all infeasible
     ref = oracle_mod.solve_batch(wl, dumps=True)
     gpu = _gpu_solve(S, wl, tables=True)
     _assert_tables_equal(S, gpu, ref)
