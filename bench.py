@@ -305,9 +305,9 @@ def probe_alu_peak(solver, torch, mode):
 def packed_launch_shape(cells: int, tile: int = 0):
     """Tiling of the packed recurrence kernel for a budget of `cells` = T + 1 cells, as its
     launcher chooses it: cells per tile R, half-groups of 16 tiles, cells left to the
-    block-wide reduction (budgets of up to 1100 cells run with one warp per instance: tiles
+    block-wide reduction (budgets of up to 1900 cells run with one warp per instance: tiles
     of 4 or 8 cells, every cell in a tile)."""
-    if cells <= 1100 and tile != 16:
+    if cells <= 1900 and tile != 16:
         R = tile if tile in (4, 8) else (4 if cells <= 904 else 8)
         return R, ((cells + R - 1) // R + 15) // 16, False
     R = tile if tile in (4, 8, 16) else (4 if cells <= 896 + 8 else 8)
@@ -615,7 +615,7 @@ def run_ours(args):
     launches_per_step = 4 if second_pass else 3
     cells_per_launch = wl.n_instances * wl.minplus_cells
     main_r = dense_rooflines(wl, main, packed, probe, counts)
-    kernel_name = ("minplus16_warp_kernel" if wl.T + 1 <= 1100 and args.minplus_tile != 16 else "minplus16_kernel") \
+    kernel_name = ("minplus16_warp_kernel" if wl.T + 1 <= 1900 and args.minplus_tile != 16 else "minplus16_kernel") \
         if packed else "minplus_kernel"
     measured_peak = probe["int16x2" if packed else "int32"]
     derived_peak = ALU_PEAK_TOPS_INT16X2 if packed else ALU_PEAK_TOPS_INT32

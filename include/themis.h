@@ -72,7 +72,7 @@ extern "C" {
  *      stages of their first non-empty bucket), and 0x7FFF above (such a state is part of
  *      no solution); the backtrack recovers the argmin along the optimal path only.  Instances
  *      whose optimum lies 32767 or more above the sum of the stages' cheapest entries
- *      are redone by the 32-bit kernel in a second launch.  Budgets of up to 1100 cells
+ *      are redone by the 32-bit kernel in a second launch.  Budgets of up to 1900 cells
  *      run with one warp per instance, longer ones with one thread block per instance.
  *   THEMIS_KERNEL_PACKED16_BLOCK  the same with one thread block per instance whatever
  *      the budget length (same tables, same results).

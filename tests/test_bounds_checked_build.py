@@ -51,8 +51,8 @@ def test_edge_shapes_raise_no_violation(S, oracle_mod, kernel_id):
 
 @pytest.mark.parametrize("kernel_id", range(6), ids=KERNEL_IDS)
 def test_budget_lengths_and_stage_counts_raise_no_violation(S, oracle_mod, kernel_id):
-    for T in (1, 2, 31, 32, 33, 127, 128, 131, 135, 136, 255, 256, 257, 263, 264, 511, 512, 903, 904, 1024, 1031, 1099,
-              1100, 2047, 2048, 2049, 2055, 2056):
+    for T in (1, 2, 31, 32, 33, 127, 128, 131, 135, 136, 255, 256, 257, 263, 264, 511, 512, 903, 904, 1024, 1031, 1100,
+              1899, 1900, 2047, 2048, 2049, 2055, 2056):
         wl = W.random_tiny_workload(5000 + T, 6, 3, 8, (1, 2, 4), 4, T,
                                     bucket_us=max(1, 400_000 // T) if T < 400 else 1000, rate_lo=20.0, rate_hi=120.0)
         _assert_results_equal(_checked_solve(S, wl, kernel_id), oracle_mod.solve_batch(wl))

@@ -276,7 +276,7 @@ def test_stability_test_of_the_transition_policy(S, oracle_mod):
 # ---------------------------------------------------------------- edge cases
 
 @pytest.mark.parametrize("T", [1, 2, 31, 32, 33, 127, 128, 131, 135, 136, 255, 256, 257, 263, 264, 511, 512, 902, 903, 904,
-                               1024, 1031, 1098, 1099, 1100,        # 903/904: 4 -> 8 cells a tile; 1099/1100: warp -> block kernel
+                               1024, 1031, 1100, 1898, 1899, 1900,  # 903/904: 4 -> 8 cells a tile; 1899/1900: warp -> block kernel
                                2047, 2048, 2049, 2055, 2056])
 def test_budget_lengths_around_tile_boundaries(S, oracle_mod, T, mode):
     wl = W.random_tiny_workload(5000 + T, 6, 3, 8, (1, 2, 4), 4, T, bucket_us=max(1, 400_000 // T) if T < 400 else 1000,
