@@ -50,7 +50,8 @@ def _both(S, wl, kernel):
     return ({k: v.cpu().numpy() for k, v in got.items()}, {k: v.cpu().numpy() for k, v in ref.items()})
 
 
-@pytest.mark.parametrize("kernel_id", [1, 2, 3, 4, 5], ids=["packed16", "wide32", "pruned", "sparse", "sparse_block"])
+@pytest.mark.parametrize("kernel_id", [1, 2, 3, 4, 5, 6],
+                         ids=["packed16", "wide32", "pruned", "sparse", "sparse_block", "packed16_block"])
 def test_static_scratch_entry_point_matches_workspace_entry_point_and_oracle(S, oracle_mod, kernel_id):
     kernel = kernel_id << 8
     # a throwaway call first, so that the buffer's address is already known when the free
