@@ -616,7 +616,7 @@ def run_ours(args):
     cells_per_launch = wl.n_instances * wl.minplus_cells
     main_r = dense_rooflines(wl, main, packed, probe, counts)
     kernel_name = ("minplus16_warp_kernel" if wl.T + 1 <= 1900 and args.minplus_tile != 16 else "minplus16_kernel") \
-        if packed else "minplus_kernel"
+        if packed else ("minplus_warp_kernel" if wl.T + 1 <= 2800 and args.minplus_tile != 16 else "minplus_kernel")
     measured_peak = probe["int16x2" if packed else "int32"]
     derived_peak = ALU_PEAK_TOPS_INT16X2 if packed else ALU_PEAK_TOPS_INT32
     line = {

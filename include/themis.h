@@ -77,7 +77,8 @@ extern "C" {
  *   THEMIS_KERNEL_PACKED16_BLOCK  the same with one thread block per instance whatever
  *      the budget length (same tables, same results).
  *   THEMIS_KERNEL_WIDE32       dense recurrence on 32-bit keys; the A rows hold the
- *      argmin tables.
+ *      argmin tables.  Budgets of up to 2800 cells run with one warp per instance, longer
+ *      ones (and THEMIS_TILE_16) with one thread block per instance.
  *   THEMIS_KERNEL_PRUNED       dense scoring, then the recurrence restricted to the
  *      undominated entries of every G_s (an entry is dominated when a smaller l has
  *      a cost at most as high; such entries never occur in the returned solution);

@@ -152,6 +152,9 @@ constexpr int kBoundsChecked = 0;
 
 cudaError_t launch_score(const Params &p, cudaStream_t stream);
 cudaError_t launch_minplus(const Params &p, int tile, cudaStream_t stream);
+// The 32-bit kernel with one warp per instance, for short budgets (tiles of 8 cells); launch_minplus uses it.
+bool minplus_warp_fits(const Params &p, int tile);
+cudaError_t launch_minplus_warp(const Params &p, cudaStream_t stream);
 cudaError_t launch_minplus16(const Params &p, int tile, cudaStream_t stream);
 // The packed kernel with one warp per instance, for short budgets (tiles of 4 or 8 cells).
 bool minplus16_warp_fits(const Params &p, int tile);
