@@ -67,7 +67,6 @@ struct Params {
     int32_t horizontal; // 1: Algorithm 2, one candidate per batch size with the fewest replicas
                         //    that sustain lambda; candidate index = batch index, stage cost = h
     int32_t only_flagged;  // wide min-plus kernel: solve only instances flagged kFlagNeedsWide
-    uint8_t warp_group[32];  // 32-bit min-plus kernel: tile group (32 tiles) owned by each warp
     int32_t n_half_groups;   // packed min-plus kernel: half-groups of 16 tiles
     const int32_t *lat_us;
     const int32_t *profile_id;
@@ -85,24 +84,6 @@ struct Params {
     int32_t *inst_flag;  // [N] kFlagBadInput: bad input seen by the scoring kernel; kFlagNeedsWide: see above
     themis_result_t out;
 };
-
-// Deals the tile groups of a min-plus block (group g costs g + 1 units: its columns
-// are that much longer) to the block's warps so that the SM's four warp schedulers,
-// which take a block's warps round-robin, end up with equal shares: longest group
-// first, always to the least loaded scheduler that still has a free warp.
-inline void assign_warp_groups(int n_warps, uint8_t *warp_group)
-{
-    int load[4] = {0, 0, 0, 0}, used[4] = {0, 0, 0, 0}, cap[4];
-    for (int c = 0; c < 4; ++c) cap[c] = (n_warps - c + 3) / 4;
-    for (int g = n_warps - 1; g >= 0; --g) {
-        int best = -1;
-        for (int c = 0; c < 4; ++c)
-            if (used[c] < cap[c] && (best < 0 || load[c] < load[best])) best = c;
-        warp_group[4 * used[best] + best] = (uint8_t)g;
-        load[best] += g + 1;
-        ++used[best];
-    }
-}
 
 constexpr size_t kMaxDynamicSmem = 226u * 1024u;   // 227 KB per block less room for static variables
 
