@@ -79,6 +79,59 @@ __device__ __forceinline__ void score_two_entries(uint32_t entries, uint32_t q4,
         : "memory");
 }
 
+// Four list entries in one go: the two at `entries` and the two at `entries + stride`, both
+// loads issued before any arithmetic so that their latencies overlap.
+__device__ __forceinline__ void score_four_entries(uint32_t entries, uint32_t stride, uint32_t q4, uint32_t lmax,
+                                                   uint32_t t4, uint32_t key_mul, uint32_t key_add, uint32_t keys,
+                                                   uint32_t idle)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q, u, v;\n\t"
+        ".reg .b32 e0, e1, e2, e3, f0, f1, f2, f3, x, y, z, w, l0, l1, l2, l3, c0, c1, c2, c3, k0, k1, k2, k3, a2;\n\t"
+        "add.u32 a2, %0, %8;\n\t"
+        "ld.shared.v4.u32 {e0, e1, e2, e3}, [%0];\n\t"
+        "ld.shared.v4.u32 {f0, f1, f2, f3}, [a2];\n\t"
+        "add.u32 x, e1, %1;\n\t"
+        "add.u32 y, e3, %1;\n\t"
+        "add.u32 z, f1, %1;\n\t"
+        "add.u32 w, f3, %1;\n\t"
+        "and.b32 l0, x, 0x1FFFC;\n\t"
+        "and.b32 l1, y, 0x1FFFC;\n\t"
+        "and.b32 l2, z, 0x1FFFC;\n\t"
+        "and.b32 l3, w, 0x1FFFC;\n\t"
+        "setp.le.u32 p, e0, %2;\n\t"
+        "setp.le.u32 q, e2, %2;\n\t"
+        "setp.le.u32 u, f0, %2;\n\t"
+        "setp.le.u32 v, f2, %2;\n\t"
+        "setp.le.and.u32 p, l0, %3, p;\n\t"
+        "setp.le.and.u32 q, l1, %3, q;\n\t"
+        "setp.le.and.u32 u, l2, %3, u;\n\t"
+        "setp.le.and.u32 v, l3, %3, v;\n\t"
+        "shr.u32 c0, x, 17;\n\t"
+        "shr.u32 c1, y, 17;\n\t"
+        "shr.u32 c2, z, 17;\n\t"
+        "shr.u32 c3, w, 17;\n\t"
+        "mad.lo.u32 k0, c0, %4, %5;\n\t"
+        "mad.lo.u32 k1, c1, %4, %5;\n\t"
+        "mad.lo.u32 k2, c2, %4, %5;\n\t"
+        "mad.lo.u32 k3, c3, %4, %5;\n\t"
+        "add.u32 l0, l0, %6;\n\t"
+        "add.u32 l1, l1, %6;\n\t"
+        "add.u32 l2, l2, %6;\n\t"
+        "add.u32 l3, l3, %6;\n\t"
+        "selp.u32 l0, l0, %7, p;\n\t"
+        "selp.u32 l1, l1, %7, q;\n\t"
+        "selp.u32 l2, l2, %7, u;\n\t"
+        "selp.u32 l3, l3, %7, v;\n\t"
+        "red.shared.min.u32 [l0], k0;\n\t"
+        "red.shared.min.u32 [l1], k1;\n\t"
+        "red.shared.min.u32 [l2], k2;\n\t"
+        "red.shared.min.u32 [l3], k3;\n\t"
+        "}" ::"r"(entries), "r"(q4), "r"(lmax), "r"(t4), "r"(key_mul), "r"(key_add), "r"(keys), "r"(idle), "r"(stride)
+        : "memory");
+}
+
 #ifdef THEMIS_CHECK_BOUNDS
 // The same step with every address formed in C++ and range-checked (bounds-checked build).
 __device__ __forceinline__ void score_two_entries_checked(const Params &p, uint32_t *smem, int smem_words,
@@ -379,8 +432,16 @@ score_kernel(const Params p)
                                                   4u * (uint32_t)T, key_mul, key_add, key_off, idle_off + lane);
 #else
                     uint32_t entries_addr = list_addr;
-                    for (int i = 0; i < len; i += 2 * groups, entries_addr += 16u * (uint32_t)groups)
-                        score_two_entries(entries_addr, q4, lmax, 4u * (uint32_t)T, key_mul, key_add, key_addr, idle_addr);
+                    if (groups <= 8) {
+                        // four entries a pass: a pass never leaves the warp's 32-entry list (len <= 32, the
+                        // list's tail holds entries that never fit)
+                        for (int i = 0; i < len; i += 4 * groups, entries_addr += 32u * (uint32_t)groups)
+                            score_four_entries(entries_addr, 16u * (uint32_t)groups, q4, lmax, 4u * (uint32_t)T, key_mul,
+                                               key_add, key_addr, idle_addr);
+                    } else {
+                        for (int i = 0; i < len; i += 2 * groups, entries_addr += 16u * (uint32_t)groups)
+                            score_two_entries(entries_addr, q4, lmax, 4u * (uint32_t)T, key_mul, key_add, key_addr, idle_addr);
+                    }
 #endif
                 }
                 __syncwarp();                                // the list is free for the next task
