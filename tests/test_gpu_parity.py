@@ -326,6 +326,39 @@ def test_most_stages_on_a_short_budget(S, oracle_mod, mode):
     _assert_results_equal(gpu, ref)
 
 
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_random_shapes_every_kernel_and_tile(S, oracle_mod, seed):
+    """Seeded random problem shapes (stages, cores, batch sizes, replicas, budget lengths on both
+    sides of every kernel and tile switch-over, both queue models, joint and vertical, rates from
+    starved to saturated): every kernel choice with every tile size against the oracle."""
+    import random
+    import torch
+    rng = random.Random(seed)
+    done = 0
+    while done < 60:
+        n_stages = rng.choice([1, 2, 3, 4, 5, 7, 10, 13])
+        c_max = rng.choice([1, 2, 3, 5, 8, 16, 33, 64])
+        batches = tuple(sorted(rng.sample([1, 2, 3, 4, 5, 6, 8, 12, 16, 24, 32, 48, 64], rng.choice([1, 2, 3, 4, 6]))))
+        h_max = rng.choice([1, 2, 3, 8, 16, 31, 33, 64])
+        T = rng.choice([1, 5, 17, 63, 64, 65, 200, 500, 903, 904, 1000, 1500, 1899, 1900, 2300, 2799, 2800, 3100])
+        vertical = rng.random() < 0.3
+        flags = rng.choice([0, W.QUEUE_PER_REPLICA])
+        bucket_us = rng.choice([250, 500, 1000, 2000]) if T >= 100 else max(1, 300_000 // T)
+        lo = rng.choice([2.0, 20.0, 200.0])
+        hi = lo * rng.choice([2, 10, 30])
+        if c_max * len(batches) * (1 if vertical else h_max) > 65535 or n_stages * h_max * c_max > 131070:
+            continue
+        done += 1
+        wl = W.random_tiny_workload(20_000 + 100 * seed + done, rng.choice([3, 9, 33]), n_stages, c_max, batches, h_max, T,
+                                    bucket_us=bucket_us, flags=flags, vertical=vertical, rate_lo=lo, rate_hi=hi)
+        ref = oracle_mod.solve_batch(wl)
+        for kernel_id in range(1, 7):
+            for tile in ((0, 4, 8, 16) if kernel_id in (1, 2, 6) else (0,)):
+                out, _ = S.solve(wl, kernel=kernel_id << 8, tile=tile)
+                torch.cuda.synchronize()
+                _assert_results_equal({k: v.cpu().numpy() for k, v in out.items()}, ref)
+
+
 SHAPES = [  # n_stages, c_max, batch sizes, h_max, T, bucket_us, vertical, rate range (rps)
     (2, 1, tuple(range(1, 17)), 512, 300, 1000, False, (50.0, 4000.0)),      # widest replica table
     (3, 100, (1,), 3, 77, 2000, False, (5.0, 90.0)),                         # one batch size, ragged core count
