@@ -46,7 +46,7 @@ __host__ __device__ inline int warp_words(int R, int n_tiles, int pitch, int S)
 }
 
 template <int R>
-__global__ void __launch_bounds__(128, 8)
+__global__ void __launch_bounds__(128, R == 8 ? 6 : 7)   // 77 and 70 registers: no spills; shared memory allows no more warps anyway
 minplus16_warp_kernel(const Params p)
 {
     extern __shared__ __align__(128) uint32_t smem[];
