@@ -26,11 +26,26 @@ def _nvcc() -> str:
     return cand if os.path.exists(cand) else "nvcc"
 
 
+def _source_digest(check_bounds: bool) -> str:
+    """Digest of everything a library is built from (sources, headers, the variant)."""
+    import hashlib
+    h = hashlib.sha256(b"check" if check_bounds else b"plain")
+    for f in SOURCES + HEADERS:
+        h.update(os.path.basename(f).encode())
+        with open(f, "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
+
+
 def is_stale(path: str = LIB_PATH) -> bool:
-    if not os.path.exists(path):
+    """True if the library is missing or was built from other sources.  The digest of its
+    sources is kept beside it (file times do not survive a copy of the tree)."""
+    try:
+        with open(path + ".sha256") as fh:
+            recorded = fh.read().strip()
+    except OSError:
         return True
-    built = os.path.getmtime(path)
-    return any(os.path.getmtime(f) > built for f in SOURCES + HEADERS)
+    return not os.path.exists(path) or recorded != _source_digest(path == CHECK_LIB_PATH)
 
 
 def build_library(force: bool = False, verbose: bool = False, check_bounds: bool = False) -> str:
@@ -48,6 +63,8 @@ def build_library(force: bool = False, verbose: bool = False, check_bounds: bool
     if proc.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + log)
     os.replace(tmp, path)
+    with open(path + ".sha256", "w") as fh:
+        fh.write(_source_digest(check_bounds) + "\n")
     if verbose:
         print(log)
     return path
